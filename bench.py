@@ -1,0 +1,309 @@
+#!/usr/bin/env python
+"""Benchmark of the pipelined-decoder decode path on B200.
+
+One bench "step" is one whole decode job of the workload's batch: every time-step of
+Algorithm 1 (one pd_step each: embedding, per layer KV-append + pipelined self-attention +
+batched cross-attention + projections, vocabulary projection, fused argmax + scheduler) until
+every sequence has ended.  `value` = decoded tokens (terminators included) per second over
+the pd_step loops, inputs resident in HBM; the context projection (pd_encode_context) is
+timed separately and reported as `encode_ms`.  `e2e` is the same job through pd_generate_host
+from pinned host buffers, copies included.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2506_23431_b200 import workload as W
+
+METRIC = "decoded tokens/s per B200"
+UNIT = "tokens/s"
+DEFAULT_CONFIG = "summarisation"      # the largest configuration (most bytes per step); fits one GPU
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def cpu_baseline(wl: W.Workload, weights, budget_steps: int):
+    """The oracle as it stands, timed on the host cores for a bounded sample: batch row 0,
+    the first `budget_steps` time-steps of its decode."""
+    from oracle.pipelined_decoder import PipelinedDecoderOracle
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    hp = wl.hyper()
+    hp["time_max"] = min(wl.time_max, budget_steps)
+    mem = W.make_encoder_memory(wl, rows=range(1))[0]
+    fl = W.make_forced_len(wl)[0]
+    orc = PipelinedDecoderOracle(weights, hp)
+    t0 = time.perf_counter()
+    r = orc.run(mem, wl.ctx, fl, keep_logits=False)
+    dt = time.perf_counter() - t0
+    toks = sum(len(s["active"]) for s in r["trace"])
+    return {"value": toks / dt, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"batch row 0 of {wl.name}, first {r['steps']} time-steps ({toks} tokens, context projection "
+                      f"included), fp64 numpy, {dt:.1f} s"}, toks, dt
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = W.CONFIGS[args.config]
+    weights = W.make_weights(wl)
+    budget = args.ref_time_steps
+    times, toks = [], 0
+    base = None
+    for k in range(args.warmup + args.steps):
+        base, n, dt = cpu_baseline(wl, weights, budget)
+        if k >= args.warmup:
+            times.append(dt); toks += n
+    total = sum(times)
+    value = toks / total
+    base["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "batch_rows": 1, "time_steps_per_step": budget},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=W.CONFIG_ORDER)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-time-steps", type=int, default=24)
+    ap.add_argument("--cpu-baseline-steps", type=int, default=40)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--self-splits", type=int, default=0)
+    ap.add_argument("--cross-splits", type=int, default=0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wl = W.CONFIGS[args.config]
+    weights = W.make_weights(wl)
+    mem = W.make_encoder_memory(wl)
+    ctx_len = W.make_ctx_len(wl)
+    fl = W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, device=local_rank, use_graph=not args.no_graph,
+                           self_splits=args.self_splits, cross_splits=args.cross_splits)
+    mem_dev = dec.device_memory(mem)
+    host_mem = torch.from_numpy(mem).to(dec.tdtype).pin_memory()
+    e = 2 if wl.dtype == "bf16" else 4
+
+    def one_decode(timed):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(dec.stream)
+        dec.encode_context(mem_dev, ctx_len, fl)
+        ev[1].record(dec.stream)
+        n = dec.run(poll_every=8)
+        ev[2].record(dec.stream)
+        return ev, n
+
+    for _ in range(args.warmup):
+        one_decode(False)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    dec.reset_counters()
+    evs = []
+    barrier()
+    t_wall = time.perf_counter()
+    for _ in range(args.steps):
+        evs.append(one_decode(True))
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    own_launches, gemm_calls = dec.counters()
+    loop_ms = sum(ev[1].elapsed_time(ev[2]) for ev, _ in evs)
+    enc_ms = sum(ev[0].elapsed_time(ev[1]) for ev, _ in evs)
+    st = dec.stats()                          # counters of the last decode
+    res = dec.collect()
+    tokens_per_decode = int(st["tokens"])
+    steps_per_decode = int(st["steps"])
+    assert tokens_per_decode == int((fl + 1).sum()), "decoded token count differs from the forced-length schedule"
+
+    # ---- end to end through pd_generate_host (host buffers, copies inside the timed region)
+    e2e_ev = []
+    for k in range(2 + args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(dec.stream)
+        out = dec.generate_host(host_mem, ctx_len, fl)
+        b.record(dec.stream)
+        if k >= 2:
+            e2e_ev.append((a, b))
+    barrier()
+    clocks = sampler.stop()
+    e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
+    assert np.array_equal(out["tokens"], res["tokens"])
+    h2d = host_mem.numel() * e + ctx_len.nbytes + fl.nbytes
+    d2h = sum(v.nbytes for v in out.values()) + 32 * (steps_per_decode // 8 + 2)
+
+    # ---- per-kernel durations with CUDA events on the library's stream (one more decode)
+    dec.profile_enable(True)
+    dec.encode_context(mem_dev, ctx_len, fl)
+    dec.profile_read()
+    dec.run(poll_every=8)
+    prof = dec.profile_read()
+    dec.profile_enable(False)
+    st_p = dec.stats()
+    L, d = wl.n_layers, wl.d_model
+    cross_bytes = st_p["cross_keys"] * 2 * d * e * L          # every context key and value once per layer
+    self_bytes = st_p["self_entries"] * 2 * d * e * L         # every visible cache entry once per layer
+    peak, peak_src = measured_peaks()
+
+    def roof(name, nbytes):
+        ms, n = prof[name]
+        if n == 0 or ms <= 0:
+            return None
+        ach = nbytes / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "traffic": None, "launches": int(n), "avg_launch_us": 1e3 * ms / n,
+                "bytes_per_launch": nbytes / n, "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0}
+
+    roofline = roof("cross_attn", cross_bytes)
+    roofline_self = roof("self_attn", self_bytes)
+    kernel_ms = {k: round(v[0], 4) for k, v in prof.items()}
+
+    # ---- max over ranks
+    t_loop = torch.tensor([loop_ms, e2e_ms, enc_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t_loop, op=dist.ReduceOp.MAX)
+    loop_ms, e2e_ms, enc_ms = [float(x) for x in t_loop.tolist()]
+    total_tokens = tokens_per_decode * args.steps * world
+    value = total_tokens / (loop_ms * 1e-3)
+    e2e_value = total_tokens / (e2e_ms * 1e-3)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": loop_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "batch": wl.batch, "context": wl.ctx, "sub_max": wl.sub_max,
+                       "delta_t": wl.delta_t, "time_max": wl.time_max, "layers": wl.n_layers, "d_model": wl.d_model,
+                       "vocab": wl.vocab, "step": "one whole decode of the batch (all time-steps of Algorithm 1)",
+                       "timed": "pd_step loops; pd_encode_context separate (encode_ms)",
+                       "l2": "inputs larger than L2 (cross K/V per layer %.0f MB)" % (wl.batch * wl.ctx * 2 * d * e / 1e6),
+                       "parallelism": "replicas (one batch per GPU)" if world > 1 else "single GPU",
+                       "self_splits": args.self_splits, "cross_splits": args.cross_splits, "graph": not args.no_graph},
+            "tokens_per_decode": tokens_per_decode, "time_steps_per_decode": steps_per_decode,
+            "ms_per_time_step": loop_ms / args.steps / max(1, steps_per_decode),
+            "encode_ms": enc_ms / args.steps, "region_wall_ms": 1e3 * t_wall,
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(own_launches), "cublas_gemms": int(gemm_calls),
+            "roofline": roofline, "roofline_self_attn": roofline_self, "kernel_ms_per_decode": kernel_ms}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        base, _, _ = cpu_baseline(wl, weights, args.cpu_baseline_steps)
+        line["cpu_baseline"] = base
+    dec.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

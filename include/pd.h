@@ -1,0 +1,206 @@
+/* pd.h - C ABI of the pipelined-decoder decode path for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the per-time-step decode of the pipelined decoder: up to sub_max
+ * subsequences of one target, each started delta_t steps after the previous one, each
+ * emitting one token per step while attending to the encoder memory H^E and to the earlier
+ * subsequences as generated so far (Section 3.2, Eq. 2-4; Algorithm 1 in Section 3.4).
+ * Encoder memory goes in, per-subsequence token streams come out.
+ *
+ * Conventions
+ *  - Every function returns a pd_status (0 = PD_OK, negative = error) unless stated.  Nothing
+ *    throws, aborts or exits.  pd_last_error() gives a text for the last failure on a handle.
+ *  - "device" pointers are CUDA device memory on cfg.device; "host" pointers are ordinary
+ *    host memory.  The caller owns every buffer it passes, including the workspace and the
+ *    weights, and must keep them alive and unmodified until pd_destroy().  The library owns
+ *    only the host-side handle.  pd_init..pd_step allocate no device memory of their own
+ *    (cuBLAS is given a slice of the workspace).
+ *  - All work is enqueued on the CUDA stream given to pd_init.  pd_step and pd_encode_context
+ *    do not synchronise; pd_done, pd_collect and the pd_get_* readers do.
+ *  - Errors found on the device (page pool exhausted, a bounded wait that expired) are written
+ *    to a status word in the workspace, turn the remaining steps into no-ops and are returned
+ *    by the next synchronising call.
+ *  - Time-steps t and subsequence indices i are 1-based as in the paper.  Subsequence i is
+ *    admitted at step s_i = (i-1)*delta_t + 1.  Its cache entry p (p = 0 is <bos>, p >= 1 the
+ *    p-th content token) carries the timestamp tau = s_i - 1 + p (Eq. 2: token j of
+ *    subsequence i is generated at step (i-1)*delta_t + j) and the position tau + i.
+ */
+#ifndef PD_H_
+#define PD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define PD_API __attribute__((visibility("default")))
+#else
+#define PD_API
+#endif
+
+typedef struct pd_handle pd_handle; /* opaque; host memory owned by the library */
+
+typedef enum {
+  PD_OK = 0,
+  PD_ERR_ARG = -1,            /* null pointer, size out of range, unsupported shape        */
+  PD_ERR_STATE = -2,          /* call out of order (e.g. pd_step before pd_encode_context) */
+  PD_ERR_WORKSPACE = -3,      /* workspace too small or misaligned                         */
+  PD_ERR_POOL_EXHAUSTED = -4, /* the KV page pool ran out (set on the device)              */
+  PD_ERR_CUDA = -5,           /* a CUDA or cuBLAS call failed                              */
+  PD_ERR_TIMEOUT = -6,        /* a bounded device-side wait expired (set on the device)    */
+  PD_ERR_UNSUPPORTED = -7     /* valid request the build does not implement                */
+} pd_status;
+
+enum { PD_DTYPE_FP32 = 0, PD_DTYPE_BF16 = 1 };
+enum { PD_POS_T5_BIAS = 0, PD_POS_ROPE = 1 };
+/* per-subsequence flags returned by pd_collect */
+enum { PD_FLAG_COMPLETE = 1, PD_FLAG_TRUNCATED = 2, PD_FLAG_CAPPED = 4 };
+/* intermediate buffers readable with pd_debug_read (values of the last layer of the last step) */
+enum {
+  PD_BUF_X = 0,        /* residual stream after the last layer, fp32 [rows, d_model]          */
+  PD_BUF_QKV = 1,      /* self-attention projection, fp32 [rows, 3*d_model]                   */
+  PD_BUF_SELF_OUT = 2, /* self-attention output, dtype [rows, d_model]                        */
+  PD_BUF_CROSS_Q = 3,  /* cross-attention queries, dtype [rows, d_model]                      */
+  PD_BUF_CROSS_OUT = 4,/* cross-attention output, dtype [rows, d_model]                       */
+  PD_BUF_STATE = 5     /* the integer decode state block, int32                               */
+};
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, d_head, d_ff, vocab; /* d_head must be 64, n_heads*d_head == d_model */
+  int32_t dtype;          /* PD_DTYPE_FP32 or PD_DTYPE_BF16: storage type of weights, H^E, K/V, GEMM inputs */
+  int32_t max_batch, max_ctx;
+  int32_t sub_max, delta_t, time_max; /* the three parameters of Algorithm 1; sub_max <= 64     */
+  int32_t max_sub_len;    /* cap on content tokens per subsequence; a subsequence that reaches
+                             it ends with sep_id at its next emission (flag PD_FLAG_CAPPED)      */
+  int32_t bos_id, eos_id, sep_id; /* eos_id and sep_id both end a subsequence                   */
+  int32_t pos_mode;       /* PD_POS_T5_BIAS: bucketed bias on the Manhattan distance of
+                             Section 4.3; PD_POS_ROPE: rotary embedding at position tau + i      */
+  int32_t rel_buckets, rel_max_dist; /* T5 causal bucketing (32, 128 in T5)                     */
+  float rope_theta, attn_scale, norm_eps;
+  int32_t page_tokens;    /* KV page size in tokens: 16 or 32                                   */
+  int32_t pool_pages;     /* KV pool size in pages; 0 = worst case (never exhausts)             */
+  int32_t self_splits, cross_splits; /* split-K factors of the two attention kernels; 0 = auto  */
+  int32_t use_graph;      /* 1: pd_step replays a CUDA graph captured at the first step         */
+  int32_t device;         /* CUDA device ordinal                                                */
+} pd_config;
+
+/* Device pointers to the parameters, all of cfg.dtype except rel_bias (fp32).  Linear weights
+ * are row-major [in, out] (y = x W).  Per layer, in this order: norm1 [d], wqkv [d, 3d]
+ * (columns q | k | v, head-major), wo [d, d], norm2 [d], wq_c [d, d], wkv_c [d, 2d] (columns
+ * k | v), wo_c [d, d], norm3 [d], w1 [d, d_ff], w2 [d_ff, d].  The decoder layer is pre-RMSNorm,
+ * bias-free, ReLU feed-forward, untied output head. */
+typedef struct {
+  const void *embed;        /* [vocab, d]                                   */
+  const void *const *layer; /* host array of n_layers*10 device pointers    */
+  const void *final_norm;   /* [d]                                          */
+  const void *lm_head;      /* [vocab, d]                                   */
+  const float *rel_bias;    /* [n_heads, rel_buckets], shared by all layers; may be NULL in RoPE mode */
+} pd_weights;
+
+/* Bytes of device workspace pd_init needs for this configuration (0 if cfg is invalid).
+ * Pure function; no CUDA call. */
+PD_API size_t pd_workspace_bytes(const pd_config *cfg);
+
+/* Creates a handle: validates cfg, carves the workspace (device, 256-byte aligned, at least
+ * pd_workspace_bytes(cfg)), creates the cuBLAS handle and the TMA descriptor.  `cuda_stream`
+ * is a cudaStream_t (NULL = legacy default stream).  Algorithm 1's inputs delta_t, time_max,
+ * sub_max are fixed here. */
+PD_API pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspace, size_t workspace_bytes,
+                  void *cuda_stream, pd_handle **out);
+
+/* Algorithm 1 lines 1-3 with H^E supplied: resets all decode state, projects the encoder
+ * memory to per-layer cross-attention keys/values, admits subsequence 1 of every sequence.
+ * enc_mem: device [batch, max_ctx, d_model] of cfg.dtype (rows at or beyond ctx_len[b] are
+ * ignored).  ctx_len: host [batch], 1..max_ctx.  forced_len: host [batch, sub_max] or NULL;
+ * forced_len[b][i-1] = m >= 0 makes subsequence i hold exactly m content tokens (terminators
+ * are barred from the argmax before that and sep_id is emitted at emission m+1); NULL or a
+ * negative entry = free-running greedy decoding. */
+PD_API pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ctx_len, int32_t batch,
+                            const int32_t *forced_len);
+
+/* One iteration of Algorithm 1's loop (lines 4-13) for every sequence of the batch: one
+ * decoder pass (Eq. 3) for all active subsequences, greedy choice (Eq. 4), append, retire on
+ * eos/sep, stop test, and the admission that line 5-7 would do at the top of the next step.
+ * teacher_tokens: device [batch, sub_max] int32 or NULL; an entry >= 0 replaces the chosen
+ * token of that subsequence as the one appended (the library's own choice is still recorded);
+ * -1 keeps the own choice.  Enqueues only; a no-op for sequences that are done. */
+PD_API pd_status pd_step(pd_handle *h, const int32_t *teacher_tokens);
+
+/* Runs pd_step(NULL) until every sequence is done or time_max is reached, polling the device
+ * every `poll_every` steps (>= 1).  Returns the number of steps enqueued in *steps_run. */
+PD_API pd_status pd_run(pd_handle *h, int32_t poll_every, int32_t *steps_run);
+
+/* Synchronises the stream; *all_done = 1 when every sequence has ended or hit time_max. */
+PD_API pd_status pd_done(pd_handle *h, int32_t *all_done);
+
+/* Algorithm 1 line 14: the subsequences without bos and terminator.  Host outputs (any may be
+ * NULL): tokens [batch, sub_max, max_sub_len] (unused tail = -1), lens [batch, sub_max],
+ * n_sub [batch] (k at the end), flags [batch, sub_max] (PD_FLAG_*), steps [batch] (the step
+ * at which the sequence stopped).  Synchronises; returns a pending device error if any. */
+PD_API pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags,
+                     int32_t *steps);
+
+/* Whole Algorithm 1 from host buffers: copies enc_mem (host [batch, max_ctx, d_model], dtype)
+ * to the device, encodes, decodes until done, copies the streams back.  Output arguments as
+ * in pd_collect.  Synchronises. */
+PD_API pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t *ctx_len, int32_t batch,
+                           const int32_t *forced_len, int32_t *tokens, int32_t *lens, int32_t *n_sub,
+                           int32_t *flags, int32_t *steps);
+
+/* Schedule trace: active_mask[(t-1)*batch + b] has bit i-1 set iff subsequence i of sequence b
+ * emitted a token at step t.  Host [time_max, batch].  Synchronises. */
+PD_API pd_status pd_get_trace(pd_handle *h, uint64_t *active_mask);
+
+/* Parity/debug: fp32 logits of the last executed step, host [rows, vocab] with
+ * rows = batch * pd_rows_per_seq(); row_sub host [rows] = subsequence index (1-based) the row
+ * belonged to in that step, 0 = unused row.  Either may be NULL.  Synchronises. */
+PD_API pd_status pd_get_logits(pd_handle *h, float *logits, int32_t *row_sub);
+
+/* The library's own greedy choices: chosen[b][i-1][n] = token chosen at emission n (0-based)
+ * of subsequence i, -1 where none.  Host [batch, sub_max, max_sub_len + 1].  Synchronises. */
+PD_API pd_status pd_get_chosen(pd_handle *h, int32_t *chosen);
+
+/* Rows per sequence in the step's row block: min(sub_max, floor(max_sub_len/delta_t) + 1), the
+ * largest number of subsequences that can be active at once. */
+PD_API int32_t pd_rows_per_seq(const pd_handle *h);
+
+/* Copies an intermediate buffer (PD_BUF_*) to host; *bytes_out = bytes written (<= max_bytes).
+ * Synchronises.  For tests. */
+PD_API pd_status pd_debug_read(pd_handle *h, int32_t which, void *dst_host, size_t max_bytes, size_t *bytes_out);
+
+/* Counters since pd_init (or the last pd_reset_counters): kernels of this library launched
+ * (graph replays count their kernel nodes) and cuBLAS GEMM calls issued. */
+PD_API pd_status pd_get_counters(const pd_handle *h, int64_t *own_kernel_launches, int64_t *gemm_calls);
+PD_API pd_status pd_reset_counters(pd_handle *h);
+
+/* Per-kernel timing.  pd_profile_enable(h, 1) makes every following pd_step bracket each hot
+ * kernel with CUDA events on the stream (steps then run without the CUDA graph);
+ * pd_profile_read sums them up (synchronises): for kind k in PD_PROF_*, ms[k] = total device
+ * time, launches[k] = launches.  Arrays of PD_PROF_COUNT entries. */
+enum { PD_PROF_APPEND = 0, PD_PROF_SELF_ATTN = 1, PD_PROF_CROSS_ATTN = 2, PD_PROF_ARGMAX_SCHED = 3,
+       PD_PROF_GEMM = 4, PD_PROF_OTHER = 5, PD_PROF_COUNT = 6 };
+PD_API pd_status pd_profile_enable(pd_handle *h, int32_t on);
+PD_API pd_status pd_profile_read(pd_handle *h, double *ms, int64_t *launches);
+
+/* Counters accumulated on the device since the last pd_encode_context, host int64 [PD_STAT_COUNT]:
+ * tokens emitted (terminators included), steps executed, and the two sums the attention
+ * kernels' algorithmic traffic follows from: over all (step, sequence), the number of cache
+ * entries of subsequences 1..max active i (each is read once per layer and head as K and V),
+ * and ctx_len of every sequence that had an active subsequence (each context key/value is read
+ * once per layer).  Synchronises. */
+enum { PD_STAT_TOKENS = 0, PD_STAT_STEPS = 1, PD_STAT_SELF_ENTRIES = 2, PD_STAT_CROSS_KEYS = 3,
+       PD_STAT_PAGES = 4, PD_STAT_COUNT = 8 };
+PD_API pd_status pd_get_stats(pd_handle *h, int64_t *stats);
+
+PD_API const char *pd_last_error(const pd_handle *h);
+PD_API const char *pd_version(void);
+
+/* Frees the host-side handle (cuBLAS handle, graph, events).  The workspace stays the caller's. */
+PD_API void pd_destroy(pd_handle *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PD_H_ */

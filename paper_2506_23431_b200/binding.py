@@ -1,0 +1,293 @@
+"""ctypes binding of the C ABI in include/pd.h.  Argument marshalling only: every step of the
+decode path runs inside libpd.so.  torch is used for device memory and the CUDA stream.
+
+There is no fallback: if libpd.so is missing or does not load, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpd.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it first (python -m paper_2506_23431_b200.build); "
+                      "there is no CPU or PyTorch fallback for the decode path")
+_lib = C.CDLL(LIB_PATH)
+
+PD_OK = 0
+PD_DTYPE_FP32, PD_DTYPE_BF16 = 0, 1
+PD_POS_T5_BIAS, PD_POS_ROPE = 0, 1
+PD_FLAG_COMPLETE, PD_FLAG_TRUNCATED, PD_FLAG_CAPPED = 1, 2, 4
+PD_BUF_X, PD_BUF_QKV, PD_BUF_SELF_OUT, PD_BUF_CROSS_Q, PD_BUF_CROSS_OUT, PD_BUF_STATE = range(6)
+PD_PROF_NAMES = ["append", "self_attn", "cross_attn", "argmax_sched", "gemm", "other"]
+PD_STAT_TOKENS, PD_STAT_STEPS, PD_STAT_SELF_ENTRIES, PD_STAT_CROSS_KEYS, PD_STAT_PAGES = range(5)
+PD_STAT_COUNT = 8
+LAYER_TENSORS = ["norm1", "wqkv", "wo", "norm2", "wq_c", "wkv_c", "wo_c", "norm3", "w1", "w2"]
+
+
+class PdConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "d_head", "d_ff", "vocab", "dtype",
+                                         "max_batch", "max_ctx", "sub_max", "delta_t", "time_max", "max_sub_len",
+                                         "bos_id", "eos_id", "sep_id", "pos_mode", "rel_buckets", "rel_max_dist")] + \
+               [(n, C.c_float) for n in ("rope_theta", "attn_scale", "norm_eps")] + \
+               [(n, C.c_int32) for n in ("page_tokens", "pool_pages", "self_splits", "cross_splits", "use_graph",
+                                         "device")]
+
+
+class PdWeights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("layer", C.POINTER(C.c_void_p)), ("final_norm", C.c_void_p),
+                ("lm_head", C.c_void_p), ("rel_bias", C.c_void_p)]
+
+
+_H = C.c_void_p
+_i32p = C.POINTER(C.c_int32)
+_SIGS = {
+    "pd_workspace_bytes": (C.c_size_t, [C.POINTER(PdConfig)]),
+    "pd_init": (C.c_int, [C.POINTER(PdConfig), C.POINTER(PdWeights), C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]),
+    "pd_encode_context": (C.c_int, [_H, C.c_void_p, _i32p, C.c_int32, _i32p]),
+    "pd_step": (C.c_int, [_H, C.c_void_p]),
+    "pd_run": (C.c_int, [_H, C.c_int32, _i32p]),
+    "pd_done": (C.c_int, [_H, _i32p]),
+    "pd_collect": (C.c_int, [_H, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "pd_generate_host": (C.c_int, [_H, C.c_void_p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "pd_get_trace": (C.c_int, [_H, C.POINTER(C.c_uint64)]),
+    "pd_get_logits": (C.c_int, [_H, C.POINTER(C.c_float), _i32p]),
+    "pd_get_chosen": (C.c_int, [_H, _i32p]),
+    "pd_rows_per_seq": (C.c_int32, [_H]),
+    "pd_debug_read": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]),
+    "pd_get_counters": (C.c_int, [_H, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
+    "pd_reset_counters": (C.c_int, [_H]),
+    "pd_profile_enable": (C.c_int, [_H, C.c_int32]),
+    "pd_profile_read": (C.c_int, [_H, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "pd_get_stats": (C.c_int, [_H, C.POINTER(C.c_int64)]),
+    "pd_last_error": (C.c_char_p, [_H]),
+    "pd_version": (C.c_char_p, []),
+    "pd_destroy": (None, [_H]),
+}
+for _name, (_res, _args) in _SIGS.items():
+    _fn = getattr(_lib, _name)          # AttributeError here = the library does not export the symbol
+    _fn.restype, _fn.argtypes = _res, _args
+EXPORTS = sorted(_SIGS)
+
+
+class PdError(RuntimeError):
+    def __init__(self, status: int, where: str, msg: str = ""):
+        super().__init__(f"{where} failed with pd_status {status}" + (f": {msg}" if msg else ""))
+        self.status = status
+
+
+def _np_i32(a, shape=None) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    if shape is not None and tuple(a.shape) != tuple(shape):
+        raise ValueError(f"expected shape {shape}, got {a.shape}")
+    return a
+
+
+def _p(a: Optional[np.ndarray], typ=_i32p):
+    return None if a is None else a.ctypes.data_as(typ)
+
+
+def make_config(hp: Dict, max_batch: int, device: int = 0, use_graph: bool = True, self_splits: int = 0,
+                cross_splits: int = 0, pool_pages: int = 0) -> PdConfig:
+    """pd_config from a plain hyper-parameter dict (keys as in Workload.hyper())."""
+    c = PdConfig()
+    for k in ("n_layers", "d_model", "n_heads", "d_head", "d_ff", "vocab", "sub_max", "delta_t", "time_max",
+              "max_sub_len", "bos_id", "eos_id", "sep_id", "pos_mode", "rel_buckets", "rel_max_dist", "page_tokens"):
+        setattr(c, k, int(hp[k]))
+    c.dtype = PD_DTYPE_BF16 if hp["dtype"] == "bf16" else PD_DTYPE_FP32
+    c.max_batch, c.max_ctx = int(max_batch), int(hp["ctx"])
+    c.rope_theta, c.attn_scale, c.norm_eps = float(hp["rope_theta"]), float(hp["attn_scale"]), float(hp["norm_eps"])
+    c.pool_pages, c.self_splits, c.cross_splits = pool_pages, self_splits, cross_splits
+    c.use_graph, c.device = int(use_graph), device
+    return c
+
+
+class PipelinedDecoder:
+    """One pd_handle plus the torch tensors (weights, workspace) it points into."""
+
+    def __init__(self, hp: Dict, weights: Dict[str, np.ndarray], max_batch: int, device: int = 0, stream=None,
+                 **cfg_kw):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the pipelined-decoder library needs a CUDA device; there is no CPU path")
+        self.torch = torch
+        self.hp = dict(hp)
+        self.device = torch.device("cuda", device)
+        self.cfg = make_config(hp, max_batch, device, **cfg_kw)
+        self.tdtype = torch.bfloat16 if hp["dtype"] == "bf16" else torch.float32
+        self.np_out_dtype = np.float32
+        nbytes = _lib.pd_workspace_bytes(C.byref(self.cfg))
+        if nbytes == 0:
+            raise PdError(-1, "pd_workspace_bytes", "invalid configuration")
+        self.workspace_bytes = int(nbytes)
+        with torch.cuda.device(self.device):
+            self._w = {}
+            for k, v in weights.items():
+                t = torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32))
+                self._w[k] = t.to(self.device, torch.float32 if k == "rel_bias" else self.tdtype).contiguous()
+            self._ws = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            self.stream = stream if stream is not None else torch.cuda.Stream(device=self.device)
+        ws_ptr = (self._ws.data_ptr() + 255) // 256 * 256
+        L = int(hp["n_layers"])
+        self._layer_ptrs = (C.c_void_p * (L * len(LAYER_TENSORS)))()
+        for l in range(L):
+            for j, name in enumerate(LAYER_TENSORS):
+                self._layer_ptrs[l * len(LAYER_TENSORS) + j] = self._w[f"l{l}.{name}"].data_ptr()
+        w = PdWeights()
+        w.embed = self._w["embed"].data_ptr()
+        w.layer = C.cast(self._layer_ptrs, C.POINTER(C.c_void_p))
+        w.final_norm = self._w["final_norm"].data_ptr()
+        w.lm_head = self._w["lm_head"].data_ptr()
+        w.rel_bias = self._w["rel_bias"].data_ptr() if "rel_bias" in self._w else None
+        self._h = _H()
+        torch.cuda.synchronize(self.device)
+        st = _lib.pd_init(C.byref(self.cfg), C.byref(w), C.c_void_p(ws_ptr), C.c_size_t(self.workspace_bytes),
+                          C.c_void_p(self.stream.cuda_stream), C.byref(self._h))
+        if st != PD_OK:
+            raise PdError(st, "pd_init")
+        self.batch = 0
+        self.rows_per_seq = int(_lib.pd_rows_per_seq(self._h))
+        self._keep = []
+
+    # -- helpers
+    def _check(self, st: int, where: str):
+        if st != PD_OK:
+            raise PdError(st, where, (_lib.pd_last_error(self._h) or b"").decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.torch.cuda.synchronize(self.device)
+            _lib.pd_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def device_memory(self, enc_mem: np.ndarray):
+        """Host float32 [batch, ctx, d] -> device tensor of the configured dtype."""
+        t = self.torch.from_numpy(np.ascontiguousarray(enc_mem, dtype=np.float32))
+        return t.to(self.device, self.tdtype).contiguous()
+
+    # -- the C ABI, one method per entry point
+    def encode_context(self, enc_mem, ctx_len: Sequence[int], forced_len=None):
+        """enc_mem: torch CUDA tensor [batch, ctx, d] of the configured dtype."""
+        batch = int(enc_mem.shape[0])
+        if tuple(enc_mem.shape[1:]) != (self.cfg.max_ctx, self.cfg.d_model) or enc_mem.dtype != self.tdtype \
+                or not enc_mem.is_contiguous() or not enc_mem.is_cuda:
+            raise ValueError("enc_mem must be a contiguous CUDA tensor [batch, max_ctx, d_model] of the model dtype")
+        cl = _np_i32(ctx_len, (batch,))
+        fl = None if forced_len is None else _np_i32(forced_len, (batch, self.cfg.sub_max))
+        self.stream.wait_stream(self.torch.cuda.current_stream(self.device))
+        self._keep = [enc_mem]
+        self._check(_lib.pd_encode_context(self._h, C.c_void_p(enc_mem.data_ptr()), _p(cl), batch, _p(fl)),
+                    "pd_encode_context")
+        self.batch = batch
+
+    def step(self, teacher_tokens=None):
+        """teacher_tokens: torch CUDA int32 tensor [batch, sub_max] or None."""
+        ptr = None
+        if teacher_tokens is not None:
+            if teacher_tokens.dtype != self.torch.int32 or tuple(teacher_tokens.shape) != (self.batch, self.cfg.sub_max) \
+                    or not teacher_tokens.is_contiguous() or not teacher_tokens.is_cuda:
+                raise ValueError("teacher_tokens must be a contiguous CUDA int32 tensor [batch, sub_max]")
+            self.stream.wait_stream(self.torch.cuda.current_stream(self.device))
+            self._keep.append(teacher_tokens)
+            ptr = C.c_void_p(teacher_tokens.data_ptr())
+        self._check(_lib.pd_step(self._h, ptr), "pd_step")
+
+    def run(self, poll_every: int = 8) -> int:
+        n = C.c_int32(0)
+        self._check(_lib.pd_run(self._h, poll_every, C.byref(n)), "pd_run")
+        return n.value
+
+    def done(self) -> bool:
+        d = C.c_int32(0)
+        self._check(_lib.pd_done(self._h, C.byref(d)), "pd_done")
+        return bool(d.value)
+
+    def collect(self):
+        b, sm, msl = self.batch, self.cfg.sub_max, self.cfg.max_sub_len
+        tokens = np.empty((b, sm, msl), np.int32)
+        lens = np.empty((b, sm), np.int32)
+        n_sub = np.empty((b,), np.int32)
+        flags = np.empty((b, sm), np.int32)
+        steps = np.empty((b,), np.int32)
+        self._check(_lib.pd_collect(self._h, _p(tokens), _p(lens), _p(n_sub), _p(flags), _p(steps)), "pd_collect")
+        return {"tokens": tokens, "lens": lens, "n_sub": n_sub, "flags": flags, "steps": steps}
+
+    def generate_host(self, enc_mem_host, ctx_len, forced_len=None):
+        """enc_mem_host: host buffer (torch CPU tensor, ideally pinned, or numpy array) of the model
+        dtype's bit pattern, [batch, ctx, d].  Returns the same dict as collect()."""
+        batch = int(enc_mem_host.shape[0])
+        ptr = enc_mem_host.data_ptr() if hasattr(enc_mem_host, "data_ptr") else enc_mem_host.ctypes.data
+        cl = _np_i32(ctx_len, (batch,))
+        fl = None if forced_len is None else _np_i32(forced_len, (batch, self.cfg.sub_max))
+        sm, msl = self.cfg.sub_max, self.cfg.max_sub_len
+        tokens = np.empty((batch, sm, msl), np.int32)
+        lens = np.empty((batch, sm), np.int32)
+        n_sub = np.empty((batch,), np.int32)
+        flags = np.empty((batch, sm), np.int32)
+        steps = np.empty((batch,), np.int32)
+        self._check(_lib.pd_generate_host(self._h, C.c_void_p(ptr), _p(cl), batch, _p(fl), _p(tokens), _p(lens),
+                                          _p(n_sub), _p(flags), _p(steps)), "pd_generate_host")
+        self.batch = batch
+        return {"tokens": tokens, "lens": lens, "n_sub": n_sub, "flags": flags, "steps": steps}
+
+    def get_trace(self) -> np.ndarray:
+        m = np.zeros((self.cfg.time_max, self.batch), np.uint64)
+        self._check(_lib.pd_get_trace(self._h, m.ctypes.data_as(C.POINTER(C.c_uint64))), "pd_get_trace")
+        return m
+
+    def get_logits(self, want_logits: bool = True):
+        rows = self.batch * self.rows_per_seq
+        lg = np.empty((rows, self.cfg.vocab), np.float32) if want_logits else None
+        rs = np.empty((rows,), np.int32)
+        self._check(_lib.pd_get_logits(self._h, _p(lg, C.POINTER(C.c_float)), _p(rs)), "pd_get_logits")
+        return lg, rs.reshape(self.batch, self.rows_per_seq)
+
+    def get_chosen(self) -> np.ndarray:
+        a = np.empty((self.batch, self.cfg.sub_max, self.cfg.max_sub_len + 1), np.int32)
+        self._check(_lib.pd_get_chosen(self._h, _p(a)), "pd_get_chosen")
+        return a
+
+    def debug_read(self, which: int, dtype, count: int) -> np.ndarray:
+        a = np.empty(count, dtype)
+        n = C.c_size_t(0)
+        self._check(_lib.pd_debug_read(self._h, which, a.ctypes.data_as(C.c_void_p), a.nbytes, C.byref(n)),
+                    "pd_debug_read")
+        return a[: n.value // a.itemsize]
+
+    def counters(self):
+        a, b = C.c_int64(0), C.c_int64(0)
+        self._check(_lib.pd_get_counters(self._h, C.byref(a), C.byref(b)), "pd_get_counters")
+        return a.value, b.value
+
+    def reset_counters(self):
+        self._check(_lib.pd_reset_counters(self._h), "pd_reset_counters")
+
+    def profile_enable(self, on: bool):
+        self._check(_lib.pd_profile_enable(self._h, int(on)), "pd_profile_enable")
+
+    def profile_read(self):
+        ms = (C.c_double * len(PD_PROF_NAMES))()
+        n = (C.c_int64 * len(PD_PROF_NAMES))()
+        self._check(_lib.pd_profile_read(self._h, ms, n), "pd_profile_read")
+        return {k: (ms[i], n[i]) for i, k in enumerate(PD_PROF_NAMES)}
+
+    def stats(self) -> Dict[str, int]:
+        a = (C.c_int64 * PD_STAT_COUNT)()
+        self._check(_lib.pd_get_stats(self._h, a), "pd_get_stats")
+        return {"tokens": a[PD_STAT_TOKENS], "steps": a[PD_STAT_STEPS], "self_entries": a[PD_STAT_SELF_ENTRIES],
+                "cross_keys": a[PD_STAT_CROSS_KEYS], "pages": a[PD_STAT_PAGES]}
+
+
+def version() -> str:
+    return _lib.pd_version().decode()

@@ -1,0 +1,212 @@
+// Small kernels of the decode step: state reset, embedding gather, RMSNorm, ReLU,
+// KV-append with the positional write, and zeroing of context rows beyond ctx_len.
+#include "pd_internal.h"
+
+namespace pd {
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---------------------------------------------------------------------------------------------
+// Reset (Algorithm 1 lines 1-2 plus the admission of subsequence 1 at step 1): clears the
+// whole state block, then gives every sequence its first subsequence, first KV page and row.
+__global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_t *ctx_len,
+                                   const int32_t *forced_len, size_t state_words, int32_t *state_base, int phase) {
+  size_t gid = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  if (phase == 0) {
+    for (size_t i = gid; i < state_words; i += stride) state_base[i] = 0;
+    return;
+  }
+  // phase 1 (after phase 0 has completed on the stream)
+  for (size_t i = gid; i < (size_t)batch * dm.SM; i += stride) {
+    st.forced_len[i] = forced_len ? forced_len[i] : -1;
+    st.last_tok[i] = dm.bos;
+  }
+  for (size_t i = gid; i < (size_t)dm.B * dm.SM * (dm.MSL + 1); i += stride) st.chosen[i] = -1;
+  for (size_t i = gid; i < (size_t)dm.B * dm.SM * dm.MSL; i += stride) st.tokens[i] = -1;
+  for (size_t b = gid; b < (size_t)batch; b += stride) {
+    st.ctx_len[b] = ctx_len[b];
+    st.k[b] = 1;
+    st.n_active[b] = 1;
+    st.start[b * dm.SM] = 1;
+    st.state[b * dm.SM] = SUB_ACTIVE;
+    st.row_sub[b * dm.C] = 1;
+    st.page_table[(size_t)b * dm.SM * dm.PPS] = (int32_t)b;   // pages 0..batch-1 go to the first subsequences
+  }
+  if (gid == 0) {
+    st.hdr[HDR_STEP_T] = 1;
+    st.hdr[HDR_BATCH] = batch;
+    st.hdr[HDR_PAGE_BUMP] = batch;
+    if (batch > dm.pool) st.hdr[HDR_STATUS] = PD_ERR_POOL_EXHAUSTED;
+  }
+}
+
+cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, const int32_t *ctx_len_dev,
+                               const int32_t *forced_len_dev, size_t state_words, int32_t *state_base,
+                               cudaStream_t s) {
+  reset_state_kernel<<<148, 256, 0, s>>>(dm, st, batch, ctx_len_dev, forced_len_dev, state_words, state_base, 0);
+  reset_state_kernel<<<148, 256, 0, s>>>(dm, st, batch, ctx_len_dev, forced_len_dev, state_words, state_base, 1);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Embedding gather: row (b, c) takes the embedding of the last token of its subsequence (the
+// decoder input of Eq. 3); unused rows are zero so that they stay zero through the layer stack.
+template <typename T>
+__global__ void embed_kernel(Dims dm, DecState st, const T *__restrict__ embed, float *__restrict__ x) {
+  int r = blockIdx.x;
+  int b = r / dm.C;
+  int i = st.row_sub[r];
+  float *xr = x + (size_t)r * dm.d;
+  if (i <= 0) {
+    for (int c = threadIdx.x; c < dm.d; c += blockDim.x) xr[c] = 0.f;
+    return;
+  }
+  int tok = st.last_tok[b * dm.SM + i - 1];
+  const T *e = embed + (size_t)tok * dm.d;
+  for (int c = threadIdx.x; c < dm.d; c += blockDim.x) xr[c] = to_f<T>(e[c]);
+}
+
+cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x,
+                         cudaStream_t s) {
+  int rows = batch * dm.C;
+  if (dtype == PD_DTYPE_BF16)
+    embed_kernel<__nv_bfloat16><<<rows, 128, 0, s>>>(dm, st, (const __nv_bfloat16 *)embed, x);
+  else
+    embed_kernel<float><<<rows, 128, 0, s>>>(dm, st, (const float *)embed, x);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm of the fp32 residual stream, output in the GEMM input type.
+template <typename T>
+__global__ void rmsnorm_kernel(int d, float eps, const float *__restrict__ x, const T *__restrict__ gain,
+                               T *__restrict__ out) {
+  __shared__ float red[32];
+  const float *xr = x + (size_t)blockIdx.x * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) { float v = xr[c]; ss += v * v; }
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (threadIdx.x == 0) red[0] = v;
+  }
+  __syncthreads();
+  float inv = rsqrtf(red[0] / (float)d + eps);
+  T *orow = out + (size_t)blockIdx.x * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) orow[c] = from_f<T>(xr[c] * inv * to_f<T>(gain[c]));
+}
+
+cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, const void *gain, void *out,
+                           cudaStream_t s) {
+  if (dtype == PD_DTYPE_BF16)
+    rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(dm.d, dm.eps, x, (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)out);
+  else
+    rmsnorm_kernel<float><<<rows, 256, 0, s>>>(dm.d, dm.eps, x, (const float *)gain, (float *)out);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void relu_kernel(T *buf, size_t n) {
+  size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) { float v = to_f<T>(buf[i]); buf[i] = from_f<T>(v > 0.f ? v : 0.f); }
+}
+
+cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s) {
+  int blocks = (int)((n + 1023) / 1024);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks < 1) blocks = 1;
+  if (dtype == PD_DTYPE_BF16) relu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((__nv_bfloat16 *)buf, n);
+  else relu_kernel<float><<<blocks, 256, 0, s>>>((float *)buf, n);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV-append + positional write.  Row (b, c) belongs to subsequence i; its input token is cache
+// entry p = len (p = 0 is bos) with timestamp tau = s_i - 1 + p (Eq. 2) and position tau + i, so
+// that the difference of two positions is the Manhattan distance of Section 4.3 on every visible
+// pair.  Writes k and v to slot p of the subsequence's page list and q to the query buffer; in
+// RoPE mode q and k are rotated by the position first.  All rows of a step are appended before
+// any attends: tokens fed by earlier subsequences at the same step are visible (tau' <= t - 1).
+template <typename T>
+__global__ void append_kernel(Dims dm, DecState st, int layer, const float *__restrict__ qkv, T *__restrict__ q_out,
+                              T *__restrict__ kv_pool, const float2 *__restrict__ rope_tab) {
+  int r = blockIdx.x;
+  int b = r / dm.C;
+  int i = st.row_sub[r];
+  if (i <= 0) return;
+  int sidx = b * dm.SM + i - 1;
+  int p = st.len[sidx];
+  int tau = st.start[sidx] - 1 + p;
+  int pos = tau + i;
+  int page = st.page_table[(size_t)sidx * dm.PPS + p / dm.P];
+  int slot = p % dm.P;
+  const float *row = qkv + (size_t)r * 3 * dm.d;
+  for (int j = threadIdx.x; j < dm.d / 2; j += blockDim.x) {
+    int col = 2 * j;
+    int h = col / kDh, dd = col % kDh;
+    float q0 = row[col], q1 = row[col + 1];
+    float k0 = row[dm.d + col], k1 = row[dm.d + col + 1];
+    float v0 = row[2 * dm.d + col], v1 = row[2 * dm.d + col + 1];
+    if (dm.pos_mode == PD_POS_ROPE) {
+      float2 cs = rope_tab[(size_t)pos * (kDh / 2) + dd / 2];
+      float a = q0 * cs.x - q1 * cs.y, c2 = q0 * cs.y + q1 * cs.x;
+      q0 = a; q1 = c2;
+      a = k0 * cs.x - k1 * cs.y; c2 = k0 * cs.y + k1 * cs.x;
+      k0 = a; k1 = c2;
+    }
+    q_out[(size_t)r * dm.d + col] = from_f<T>(q0);
+    q_out[(size_t)r * dm.d + col + 1] = from_f<T>(q1);
+    size_t base = ((((size_t)layer * dm.pool + page) * 2) * dm.H + h) * dm.P * kDh + (size_t)slot * kDh + dd;
+    size_t vofs = (size_t)dm.H * dm.P * kDh;
+    kv_pool[base] = from_f<T>(k0);
+    kv_pool[base + 1] = from_f<T>(k1);
+    kv_pool[base + vofs] = from_f<T>(v0);
+    kv_pool[base + vofs + 1] = from_f<T>(v1);
+  }
+}
+
+cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
+                          void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s) {
+  int rows = batch * dm.C;
+  int threads = dm.d / 2 < 256 ? dm.d / 2 : 256;
+  if (dtype == PD_DTYPE_BF16)
+    append_kernel<__nv_bfloat16><<<rows, threads, 0, s>>>(dm, st, layer, qkv, (__nv_bfloat16 *)q_out,
+                                                         (__nv_bfloat16 *)kv_pool, rope_tab);
+  else
+    append_kernel<float><<<rows, threads, 0, s>>>(dm, st, layer, qkv, (float *)q_out, (float *)kv_pool, rope_tab);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Context rows at or beyond ctx_len[b] never take part in cross-attention; zero their projected
+// keys/values so that a masked weight of exactly 0 never multiplies a non-finite value.
+template <typename T>
+__global__ void zero_ctx_pad_kernel(Dims dm, DecState st, T *kv_c) {
+  int b = blockIdx.y, l = blockIdx.z;
+  int cl = st.ctx_len[b];
+  size_t w = 2 * (size_t)dm.d;
+  for (int pos = cl + blockIdx.x; pos < dm.ctx; pos += gridDim.x) {
+    T *row = kv_c + (((size_t)l * dm.B + b) * dm.ctx + pos) * w;
+    for (size_t c = threadIdx.x; c < w; c += blockDim.x) row[c] = from_f<T>(0.f);
+  }
+}
+
+cudaError_t launch_zero_ctx_pad(const Dims &dm, const DecState &st, int batch, int dtype, void *kv_c, cudaStream_t s) {
+  dim3 grid(32, batch, dm.L);
+  if (dtype == PD_DTYPE_BF16) zero_ctx_pad_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(dm, st, (__nv_bfloat16 *)kv_c);
+  else zero_ctx_pad_kernel<float><<<grid, 256, 0, s>>>(dm, st, (float *)kv_c);
+  return cudaGetLastError();
+}
+
+}  // namespace pd

@@ -1,0 +1,636 @@
+// Host side of the C ABI: configuration checks, workspace carving, the per-step launch
+// sequence (own kernels + cuBLAS projections) and its CUDA-graph replay, result readers.
+#include <cublas_v2.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "pd_internal.h"
+
+using namespace pd;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kCublasWs = 64u << 20;
+
+struct Region { size_t off = 0, bytes = 0; };
+
+struct Layout {
+  // integer state (offsets in int32 words from the start of the state block)
+  size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
+      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, state_words;
+  Region state, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
+      ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, cublas_ws;
+  size_t total = 0;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
+  if (c.n_layers < 1 || c.d_model < 64 || c.n_heads < 1 || c.d_head != kDh || c.n_heads * c.d_head != c.d_model) return false;
+  if (c.d_ff < 8 || c.vocab < 4 || (c.d_model % 8) || (c.d_ff % 8)) return false;
+  if (c.dtype != PD_DTYPE_FP32 && c.dtype != PD_DTYPE_BF16) return false;
+  if (c.max_batch < 1 || c.max_ctx < 1 || c.sub_max < 1 || c.sub_max > 64 || c.delta_t < 1 || c.time_max < 1) return false;
+  if (c.max_sub_len < 1 || (c.page_tokens != 16 && c.page_tokens != 32)) return false;
+  if (c.pos_mode != PD_POS_T5_BIAS && c.pos_mode != PD_POS_ROPE) return false;
+  if (c.pos_mode == PD_POS_T5_BIAS && (c.rel_buckets < 2 || c.rel_buckets > 256 || (c.rel_buckets & 1) || c.rel_max_dist <= c.rel_buckets / 2)) return false;
+  const int ids[3] = {c.bos_id, c.eos_id, c.sep_id};
+  for (int v : ids) if (v < 0 || v >= c.vocab) return false;
+  if (c.self_splits < 0 || c.self_splits > 32 || c.cross_splits < 0 || c.cross_splits > 32) return false;
+  if (!(c.attn_scale > 0.f) || !(c.norm_eps >= 0.f)) return false;
+  dm.L = c.n_layers; dm.d = c.d_model; dm.H = c.n_heads; dm.ff = c.d_ff; dm.V = c.vocab;
+  dm.B = c.max_batch; dm.ctx = c.max_ctx; dm.SM = c.sub_max; dm.dt = c.delta_t; dm.T = c.time_max;
+  dm.MSL = c.max_sub_len;
+  int conc = c.max_sub_len / c.delta_t + 1;   // subsequences that can be open at the same step
+  dm.C = conc < c.sub_max ? conc : c.sub_max;
+  dm.P = c.page_tokens;
+  dm.PPS = (c.max_sub_len + 1 + dm.P - 1) / dm.P;
+  long long worst = (long long)c.max_batch * c.sub_max * dm.PPS;
+  dm.pool = c.pool_pages > 0 ? c.pool_pages : (int)worst;
+  if (c.pool_pages < 0 || worst > 0x7fffffffLL) return false;
+  dm.bos = c.bos_id; dm.eos = c.eos_id; dm.sep = c.sep_id;
+  dm.pos_mode = c.pos_mode;
+  dm.n_dist = c.time_max + c.sub_max + 2;
+  if (c.pos_mode == PD_POS_T5_BIAS && dm.n_dist > 512) return false;
+  dm.scale_log2e = c.attn_scale * 1.4426950408889634f;
+  dm.eps = c.norm_eps;
+  max_splits = 32;
+  return true;
+}
+
+void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) {
+  const size_t B = dm.B, SM = dm.SM, C = dm.C;
+  size_t w = 0;
+  auto take = [&](size_t n) { size_t o = w; w += n; return o; };
+  L.w_hdr = take(HDR_WORDS);
+  L.w_stats = take(2 * PD_STAT_COUNT);            // 64-bit counters, 8-byte aligned (HDR_WORDS is even)
+  L.w_trace = take(2 * (size_t)dm.T * B);         // 64-bit masks
+  L.w_k = take(B); L.w_done = take(B); L.w_steps = take(B); L.w_nact = take(B); L.w_ctx = take(B); L.w_ticket = take(B);
+  L.w_start = take(B * SM); L.w_len = take(B * SM); L.w_state = take(B * SM); L.w_flag = take(B * SM);
+  L.w_last = take(B * SM); L.w_forced = take(B * SM);
+  L.w_row = take(B * C); L.w_prow = take(B * C); L.w_rtok = take(B * C);
+  L.w_ptab = take(B * SM * dm.PPS);
+  L.w_tokens = take(B * SM * dm.MSL);
+  L.w_chosen = take(B * SM * (dm.MSL + 1));
+  L.state_words = w;
+
+  size_t off = 0;
+  auto reg = [&](Region &r, size_t bytes) { r.off = off; r.bytes = bytes; off = align_up(off + bytes, kAlign); };
+  const size_t e = c.dtype == PD_DTYPE_BF16 ? 2 : 4;
+  const size_t M = B * C;
+  reg(L.state, L.state_words * 4);
+  reg(L.ctx_len_in, B * 4);
+  reg(L.forced_in, B * SM * 4);
+  reg(L.teacher, B * SM * 4);
+  reg(L.dist_bucket, (size_t)dm.n_dist * 4);
+  reg(L.rope_tab, (size_t)dm.n_dist * (kDh / 2) * sizeof(float2));
+  reg(L.x, M * dm.d * 4);
+  reg(L.hbuf, M * dm.d * e);
+  reg(L.qkv, M * 3 * dm.d * 4);
+  reg(L.qbuf, M * dm.d * e);
+  reg(L.self_out, M * dm.d * e);
+  reg(L.cq, M * dm.d * e);
+  reg(L.cross_out, M * dm.d * e);
+  reg(L.ffn, M * dm.ff * e);
+  reg(L.logits, M * (size_t)dm.V * 4);
+  reg(L.part_o, M * dm.H * max_splits * kDh * 4);
+  reg(L.part_ml, M * dm.H * max_splits * 2 * 4);
+  reg(L.kv_c, (size_t)dm.L * B * dm.ctx * 2 * dm.d * e);
+  reg(L.kv_pool, (size_t)dm.L * dm.pool * 2 * dm.H * dm.P * kDh * e);
+  reg(L.enc_stage, B * dm.ctx * dm.d * e);
+  reg(L.cublas_ws, kCublasWs);
+  L.total = off;
+}
+
+struct ProfRec { int kind; cudaEvent_t a, b; };
+
+}  // namespace
+
+struct pd_handle {
+  pd_config cfg;
+  Dims dm;
+  Layout lay;
+  int max_splits = 32;
+  uint8_t *ws = nullptr;
+  cudaStream_t stream = nullptr;
+  cublasHandle_t blas = nullptr;
+  DecState st;
+  std::vector<const void *> layer_w;
+  pd_weights w;
+  CUtensorMap tmap_kvc;
+  bool have_tmap = false;
+  int batch = 0;
+  bool encoded = false;
+  int self_splits = 1, cross_splits = 1;
+  int steps_enqueued = 0;
+  bool teacher_clear = false;
+  // graph
+  cudaGraphExec_t graph_exec = nullptr;
+  int graph_batch = -1;
+  long long graph_own = 0, graph_gemm = 0;
+  // counters / profiling
+  long long own_launches = 0, gemm_calls = 0;
+  bool profiling = false;
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> ev_pool;
+  int32_t *pinned_flag = nullptr;
+  std::string err;
+  template <typename T> T *ptr(const Region &r) const { return reinterpret_cast<T *>(ws + r.off); }
+};
+
+namespace {
+
+pd_status fail(pd_handle *h, pd_status s, const std::string &msg) {
+  if (h) h->err = msg;
+  return s;
+}
+#define CU_TRY(h, expr)                                                                                   \
+  do {                                                                                                    \
+    cudaError_t e__ = (expr);                                                                             \
+    if (e__ != cudaSuccess) return fail(h, PD_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+  } while (0)
+#define PD_TRY(expr)                         \
+  do {                                       \
+    pd_status s__ = (expr);                  \
+    if (s__ != PD_OK) return s__;            \
+  } while (0)
+
+cudaEvent_t get_event(pd_handle *h) {
+  if (!h->ev_pool.empty()) { cudaEvent_t e = h->ev_pool.back(); h->ev_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct ProfScope {
+  pd_handle *h; int kind; cudaEvent_t a = nullptr;
+  ProfScope(pd_handle *h_, int k) : h(h_), kind(k) {
+    if (h->profiling) { a = get_event(h); cudaEventRecord(a, h->stream); }
+  }
+  ~ProfScope() {
+    if (h->profiling) { cudaEvent_t b = get_event(h); cudaEventRecord(b, h->stream); h->prof.push_back({kind, a, b}); }
+  }
+};
+
+// row-major C[M,N] (+)= A[M,K] * W, with W row-major [K,N] (w_is_nk = false) or [N,K] (true)
+pd_status gemm(pd_handle *h, bool w_is_nk, int M, int N, int K, const void *A, const void *W, void *Cmat,
+               bool c_is_f32, float beta) {
+  ProfScope ps(h, PD_PROF_GEMM);
+  const bool bf = h->cfg.dtype == PD_DTYPE_BF16;
+  cudaDataType in_t = bf ? CUDA_R_16BF : CUDA_R_32F;
+  cudaDataType c_t = (c_is_f32 || !bf) ? CUDA_R_32F : CUDA_R_16BF;
+  cublasComputeType_t comp = bf ? CUBLAS_COMPUTE_32F : CUBLAS_COMPUTE_32F_PEDANTIC;
+  float alpha = 1.f;
+  cublasStatus_t s = cublasGemmEx(h->blas, w_is_nk ? CUBLAS_OP_T : CUBLAS_OP_N, CUBLAS_OP_N, N, M, K, &alpha, W, in_t,
+                                  w_is_nk ? K : N, A, in_t, K, &beta, Cmat, c_t, N, comp, CUBLAS_GEMM_DEFAULT);
+  if (s != CUBLAS_STATUS_SUCCESS) return fail(h, PD_ERR_CUDA, "cublasGemmEx failed with status " + std::to_string((int)s));
+  h->gemm_calls++;
+  return PD_OK;
+}
+
+#define OWN(h, kind, expr)                          \
+  do {                                              \
+    ProfScope ps__(h, kind);                        \
+    CU_TRY(h, expr);                                \
+    h->own_launches++;                              \
+  } while (0)
+
+AttnArgs attn_args(pd_handle *h, int layer, bool self) {
+  AttnArgs a;
+  a.dm = h->dm; a.st = h->st; a.layer = layer; a.batch = h->batch;
+  a.splits = self ? h->self_splits : h->cross_splits;
+  a.q = self ? h->ptr<void>(h->lay.qbuf) : h->ptr<void>(h->lay.cq);
+  a.kv = self ? h->ptr<void>(h->lay.kv_pool) : h->ptr<void>(h->lay.kv_c);
+  a.out = self ? h->ptr<void>(h->lay.self_out) : h->ptr<void>(h->lay.cross_out);
+  a.part_o = h->ptr<float>(h->lay.part_o);
+  a.part_ml = h->ptr<float>(h->lay.part_ml);
+  a.dist_bucket = h->ptr<int32_t>(h->lay.dist_bucket);
+  a.rel_bias = h->w.rel_bias;
+  a.rel_buckets = h->cfg.rel_buckets;
+  return a;
+}
+
+// The launch sequence of one decode step (one pass of Eq. 3 for all active rows + Algorithm 1's bookkeeping).
+pd_status enqueue_step(pd_handle *h) {
+  const Dims &dm = h->dm;
+  const int dt = h->cfg.dtype;
+  const int M = h->batch * dm.C;
+  cudaStream_t s = h->stream;
+  float *x = h->ptr<float>(h->lay.x);
+  void *hb = h->ptr<void>(h->lay.hbuf);
+  float *qkv = h->ptr<float>(h->lay.qkv);
+  void *ffn = h->ptr<void>(h->lay.ffn);
+  float *logits = h->ptr<float>(h->lay.logits);
+  const bool tma_cross = dt == PD_DTYPE_BF16 && h->have_tmap && dm.C <= 32;
+
+  OWN(h, PD_PROF_OTHER, launch_embed(dm, h->st, h->batch, dt, h->w.embed, x, s));
+  for (int l = 0; l < dm.L; ++l) {
+    const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
+    PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, true, 0.f));
+    OWN(h, PD_PROF_APPEND, launch_append(dm, h->st, h->batch, l, dt, qkv, h->ptr<void>(h->lay.qbuf),
+                                         h->ptr<void>(h->lay.kv_pool), h->ptr<float2>(h->lay.rope_tab), s));
+    {
+      AttnArgs a = attn_args(h, l, true);
+      ProfScope ps(h, PD_PROF_SELF_ATTN);
+      CU_TRY(h, launch_attn_core(a, dt, true, s));
+      h->own_launches++;
+      if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, s)); h->own_launches++; }
+    }
+    PD_TRY(gemm(h, false, M, dm.d, dm.d, h->ptr<void>(h->lay.self_out), lw[2], x, true, 1.f));
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[3], hb, s));
+    PD_TRY(gemm(h, false, M, dm.d, dm.d, hb, lw[4], h->ptr<void>(h->lay.cq), false, 0.f));
+    {
+      AttnArgs a = attn_args(h, l, false);
+      ProfScope ps(h, PD_PROF_CROSS_ATTN);
+      if (tma_cross) CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, s));
+      else CU_TRY(h, launch_attn_core(a, dt, false, s));
+      h->own_launches++;
+      if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, s)); h->own_launches++; }
+    }
+    PD_TRY(gemm(h, false, M, dm.d, dm.d, h->ptr<void>(h->lay.cross_out), lw[6], x, true, 1.f));
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[7], hb, s));
+    PD_TRY(gemm(h, false, M, dm.ff, dm.d, hb, lw[8], ffn, false, 0.f));
+    OWN(h, PD_PROF_OTHER, launch_relu(dt, ffn, (size_t)M * dm.ff, s));
+    PD_TRY(gemm(h, false, M, dm.d, dm.ff, ffn, lw[9], x, true, 1.f));
+  }
+  OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, h->w.final_norm, hb, s));
+  PD_TRY(gemm(h, true, M, dm.V, dm.d, hb, h->w.lm_head, logits, true, 0.f));
+  OWN(h, PD_PROF_ARGMAX_SCHED, launch_argmax_sched(dm, h->st, h->batch, logits, h->ptr<int32_t>(h->lay.teacher), s));
+  return PD_OK;
+}
+
+int t5_bucket(int dist, int num_buckets, int max_dist) {
+  int exact = num_buckets / 2;
+  if (dist < exact) return dist;
+  int b = exact + (int)floor(log((double)dist / exact) / log((double)max_dist / exact) * (num_buckets - exact));
+  return b < num_buckets - 1 ? b : num_buckets - 1;
+}
+
+pd_status make_tensor_map(pd_handle *h) {
+  typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CU_TRY(h, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return fail(h, PD_ERR_CUDA, "cuTensorMapEncodeTiled not available");
+  const Dims &dm = h->dm;
+  cuuint64_t gdim[2] = {(cuuint64_t)2 * dm.d, (cuuint64_t)dm.L * dm.B * dm.ctx};
+  cuuint64_t gstride[1] = {(cuuint64_t)2 * dm.d * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kDh, 128u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = ((EncodeFn)fn)(&h->tmap_kvc, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ptr<void>(h->lay.kv_c), gdim, gstride, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(h, PD_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+  h->have_tmap = true;
+  return PD_OK;
+}
+
+void drop_graph(pd_handle *h) {
+  if (h->graph_exec) { cudaGraphExecDestroy(h->graph_exec); h->graph_exec = nullptr; }
+  h->graph_batch = -1;
+}
+
+pd_status device_status(pd_handle *h) {
+  int32_t hdr[HDR_WORDS];
+  CU_TRY(h, cudaMemcpyAsync(hdr, h->st.hdr, sizeof(hdr), cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  if (hdr[HDR_STATUS] != 0) return fail(h, (pd_status)hdr[HDR_STATUS], "device-side error " + std::to_string(hdr[HDR_STATUS]));
+  return PD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t pd_workspace_bytes(const pd_config *cfg) {
+  if (!cfg) return 0;
+  Dims dm; int ms; Layout L;
+  if (!make_dims(*cfg, dm, ms)) return 0;
+  make_layout(*cfg, dm, ms, L);
+  return L.total;
+}
+
+pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspace, size_t workspace_bytes,
+                  void *cuda_stream, pd_handle **out) {
+  if (!cfg || !weights || !workspace || !out) return PD_ERR_ARG;
+  *out = nullptr;
+  Dims dm; int ms;
+  if (!make_dims(*cfg, dm, ms)) return PD_ERR_ARG;
+  if (!weights->embed || !weights->layer || !weights->final_norm || !weights->lm_head) return PD_ERR_ARG;
+  if (cfg->pos_mode == PD_POS_T5_BIAS && !weights->rel_bias) return PD_ERR_ARG;
+  for (int i = 0; i < cfg->n_layers * kLayerTensors; ++i) if (!weights->layer[i]) return PD_ERR_ARG;
+  pd_handle *h = new pd_handle();
+  h->cfg = *cfg; h->dm = dm; h->max_splits = ms;
+  make_layout(*cfg, dm, ms, h->lay);
+  if (workspace_bytes < h->lay.total || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) { delete h; return PD_ERR_WORKSPACE; }
+  h->ws = reinterpret_cast<uint8_t *>(workspace);
+  h->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  h->w = *weights;
+  h->layer_w.assign(weights->layer, weights->layer + (size_t)cfg->n_layers * kLayerTensors);
+  h->w.layer = h->layer_w.data();
+  auto bail = [&](pd_status s) { pd_destroy(h); return s; };
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return bail(PD_ERR_CUDA);
+  if (cublasCreate(&h->blas) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
+  if (cublasSetStream(h->blas, h->stream) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
+  if (cublasSetWorkspace(h->blas, h->ptr<void>(h->lay.cublas_ws), kCublasWs) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
+  if (cublasSetMathMode(h->blas, CUBLAS_DEFAULT_MATH) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
+  if (cudaHostAlloc((void **)&h->pinned_flag, 64, cudaHostAllocDefault) != cudaSuccess) return bail(PD_ERR_CUDA);
+
+  int32_t *sb = h->ptr<int32_t>(h->lay.state);
+  const Layout &L = h->lay;
+  DecState &st = h->st;
+  st.hdr = sb + L.w_hdr; st.stats = reinterpret_cast<unsigned long long *>(sb + L.w_stats);
+  st.trace = reinterpret_cast<unsigned long long *>(sb + L.w_trace);
+  st.k = sb + L.w_k; st.done = sb + L.w_done; st.steps = sb + L.w_steps; st.n_active = sb + L.w_nact;
+  st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket;
+  st.start = sb + L.w_start; st.len = sb + L.w_len; st.state = sb + L.w_state; st.flag = sb + L.w_flag;
+  st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced;
+  st.row_sub = sb + L.w_row; st.prev_row_sub = sb + L.w_prow; st.row_tok = sb + L.w_rtok;
+  st.page_table = sb + L.w_ptab; st.tokens = sb + L.w_tokens; st.chosen = sb + L.w_chosen;
+
+  // tables: distance -> bucket (T5 causal bucketing) and (cos, sin) per position and frequency
+  std::vector<int32_t> lut(dm.n_dist, 0);
+  if (cfg->pos_mode == PD_POS_T5_BIAS)
+    for (int d0 = 0; d0 < dm.n_dist; ++d0) lut[d0] = t5_bucket(d0, cfg->rel_buckets, cfg->rel_max_dist);
+  std::vector<float2> rope((size_t)dm.n_dist * (kDh / 2));
+  for (int p = 0; p < dm.n_dist; ++p)
+    for (int j = 0; j < kDh / 2; ++j) {
+      double ang = (double)p * pow((double)cfg->rope_theta, -2.0 * j / kDh);
+      rope[(size_t)p * (kDh / 2) + j] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+  if (cudaMemcpyAsync(h->ptr<void>(L.dist_bucket), lut.data(), lut.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaMemcpyAsync(h->ptr<void>(L.rope_tab), rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaMemsetAsync(h->ptr<void>(L.state), 0, L.state.bytes, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return bail(PD_ERR_CUDA);
+  if (cfg->dtype == PD_DTYPE_BF16 && dm.C <= 32) {
+    pd_status s = make_tensor_map(h);
+    if (s != PD_OK) return bail(s);
+    if (cross_attn_tma_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
+  }
+  *out = h;
+  return PD_OK;
+}
+
+pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ctx_len, int32_t batch,
+                            const int32_t *forced_len) {
+  if (!h) return PD_ERR_ARG;
+  if (!enc_mem || !ctx_len || batch < 1 || batch > h->dm.B) return fail(h, PD_ERR_ARG, "pd_encode_context: bad argument");
+  const Dims &dm = h->dm;
+  for (int b = 0; b < batch; ++b)
+    if (ctx_len[b] < 1 || ctx_len[b] > dm.ctx) return fail(h, PD_ERR_ARG, "pd_encode_context: ctx_len out of range");
+  if (forced_len)
+    for (int i = 0; i < batch * dm.SM; ++i)
+      if (forced_len[i] > dm.MSL) return fail(h, PD_ERR_ARG, "pd_encode_context: forced_len exceeds max_sub_len");
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  cudaStream_t s = h->stream;
+  const Layout &L = h->lay;
+  CU_TRY(h, cudaMemcpyAsync(h->ptr<void>(L.ctx_len_in), ctx_len, (size_t)batch * 4, cudaMemcpyHostToDevice, s));
+  if (forced_len)
+    CU_TRY(h, cudaMemcpyAsync(h->ptr<void>(L.forced_in), forced_len, (size_t)batch * dm.SM * 4, cudaMemcpyHostToDevice, s));
+  CU_TRY(h, cudaMemsetAsync(h->ptr<void>(L.teacher), 0xFF, L.teacher.bytes, s));
+  h->teacher_clear = true;
+  if (batch != h->batch) drop_graph(h);
+  h->batch = batch;
+  // split-K factors
+  auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
+  const int bh = batch * dm.H;
+  int ss = h->cfg.self_splits > 0 ? h->cfg.self_splits : cdiv(2 * 148, bh);
+  if (ss > 8 && h->cfg.self_splits == 0) ss = 8;
+  int cs = h->cfg.cross_splits;
+  if (cs == 0) {
+    int tiles = cdiv(dm.ctx, 128);
+    cs = cdiv(4 * 148, bh);
+    int cap = tiles / 2 > 1 ? tiles / 2 : 1;
+    if (cs > cap) cs = cap;
+  }
+  if (ss > h->max_splits) ss = h->max_splits;
+  if (cs > h->max_splits) cs = h->max_splits;
+  if (ss != h->self_splits || cs != h->cross_splits) drop_graph(h);
+  h->self_splits = ss < 1 ? 1 : ss;
+  h->cross_splits = cs < 1 ? 1 : cs;
+
+  OWN(h, PD_PROF_OTHER, launch_reset_state(dm, h->st, batch, h->ptr<int32_t>(L.ctx_len_in),
+                                           forced_len ? h->ptr<int32_t>(L.forced_in) : nullptr, L.state_words,
+                                           h->ptr<int32_t>(L.state), s));
+  h->own_launches++;   // the reset is two launches
+  const size_t e = h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4;
+  for (int l = 0; l < dm.L; ++l) {
+    uint8_t *dst = h->ptr<uint8_t>(L.kv_c) + (size_t)l * dm.B * dm.ctx * 2 * dm.d * e;
+    PD_TRY(gemm(h, false, batch * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5], dst, false, 0.f));
+  }
+  OWN(h, PD_PROF_OTHER, launch_zero_ctx_pad(dm, h->st, batch, h->cfg.dtype, h->ptr<void>(L.kv_c), s));
+  h->encoded = true;
+  h->steps_enqueued = 0;
+  return PD_OK;
+}
+
+pd_status pd_step(pd_handle *h, const int32_t *teacher_tokens) {
+  if (!h) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_step before pd_encode_context");
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  const Layout &L = h->lay;
+  if (teacher_tokens) {
+    CU_TRY(h, cudaMemcpyAsync(h->ptr<void>(L.teacher), teacher_tokens, (size_t)h->batch * h->dm.SM * 4,
+                              cudaMemcpyDeviceToDevice, h->stream));
+    h->teacher_clear = false;
+  } else if (!h->teacher_clear) {
+    CU_TRY(h, cudaMemsetAsync(h->ptr<void>(L.teacher), 0xFF, L.teacher.bytes, h->stream));
+    h->teacher_clear = true;
+  }
+  if (h->cfg.use_graph && !h->profiling) {
+    if (!h->graph_exec) {
+      cudaGraph_t g = nullptr;
+      long long own0 = h->own_launches, gemm0 = h->gemm_calls;
+      CU_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+      pd_status s = enqueue_step(h);
+      cudaError_t ce = cudaStreamEndCapture(h->stream, &g);
+      h->graph_own = h->own_launches - own0; h->graph_gemm = h->gemm_calls - gemm0;
+      h->own_launches = own0; h->gemm_calls = gemm0;
+      if (s != PD_OK) { if (g) cudaGraphDestroy(g); return s; }
+      CU_TRY(h, ce);
+      cudaError_t ie = cudaGraphInstantiate(&h->graph_exec, g, 0);
+      cudaGraphDestroy(g);
+      CU_TRY(h, ie);
+      h->graph_batch = h->batch;
+    }
+    CU_TRY(h, cudaGraphLaunch(h->graph_exec, h->stream));
+    h->own_launches += h->graph_own; h->gemm_calls += h->graph_gemm;
+  } else {
+    PD_TRY(enqueue_step(h));
+  }
+  h->steps_enqueued++;
+  return PD_OK;
+}
+
+pd_status pd_done(pd_handle *h, int32_t *all_done) {
+  if (!h || !all_done) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_done before pd_encode_context");
+  CU_TRY(h, cudaMemcpyAsync(h->pinned_flag, h->st.hdr, 8 * sizeof(int32_t), cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  *all_done = h->pinned_flag[HDR_ALL_DONE];
+  if (h->pinned_flag[HDR_STATUS] != 0)
+    return fail(h, (pd_status)h->pinned_flag[HDR_STATUS], "device-side error " + std::to_string(h->pinned_flag[HDR_STATUS]));
+  return PD_OK;
+}
+
+pd_status pd_run(pd_handle *h, int32_t poll_every, int32_t *steps_run) {
+  if (!h || poll_every < 1) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_run before pd_encode_context");
+  int n = 0;
+  int32_t done = 0;
+  while (h->steps_enqueued < h->dm.T) {
+    PD_TRY(pd_step(h, nullptr));
+    ++n;
+    if (n % poll_every == 0) {
+      PD_TRY(pd_done(h, &done));
+      if (done) break;
+    }
+  }
+  if (!done) PD_TRY(pd_done(h, &done));
+  if (steps_run) *steps_run = n;
+  return PD_OK;
+}
+
+pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags, int32_t *steps) {
+  if (!h) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_collect before pd_encode_context");
+  const Dims &dm = h->dm;
+  const size_t nb = h->batch;
+  cudaStream_t s = h->stream;
+  if (tokens) CU_TRY(h, cudaMemcpyAsync(tokens, h->st.tokens, nb * dm.SM * dm.MSL * 4, cudaMemcpyDeviceToHost, s));
+  if (lens) CU_TRY(h, cudaMemcpyAsync(lens, h->st.len, nb * dm.SM * 4, cudaMemcpyDeviceToHost, s));
+  if (n_sub) CU_TRY(h, cudaMemcpyAsync(n_sub, h->st.k, nb * 4, cudaMemcpyDeviceToHost, s));
+  if (flags) CU_TRY(h, cudaMemcpyAsync(flags, h->st.flag, nb * dm.SM * 4, cudaMemcpyDeviceToHost, s));
+  if (steps) CU_TRY(h, cudaMemcpyAsync(steps, h->st.steps, nb * 4, cudaMemcpyDeviceToHost, s));
+  return device_status(h);
+}
+
+pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t *ctx_len, int32_t batch,
+                           const int32_t *forced_len, int32_t *tokens, int32_t *lens, int32_t *n_sub,
+                           int32_t *flags, int32_t *steps) {
+  if (!h || !enc_mem_host) return PD_ERR_ARG;
+  if (batch < 1 || batch > h->dm.B) return fail(h, PD_ERR_ARG, "pd_generate_host: bad batch");
+  const size_t e = h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4;
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  CU_TRY(h, cudaMemcpyAsync(h->ptr<void>(h->lay.enc_stage), enc_mem_host, (size_t)batch * h->dm.ctx * h->dm.d * e,
+                            cudaMemcpyHostToDevice, h->stream));
+  PD_TRY(pd_encode_context(h, h->ptr<void>(h->lay.enc_stage), ctx_len, batch, forced_len));
+  int32_t n = 0;
+  PD_TRY(pd_run(h, 8, &n));
+  return pd_collect(h, tokens, lens, n_sub, flags, steps);
+}
+
+pd_status pd_get_trace(pd_handle *h, uint64_t *active_mask) {
+  if (!h || !active_mask) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_get_trace before pd_encode_context");
+  const Dims &dm = h->dm;
+  std::vector<uint64_t> tmp((size_t)dm.T * dm.B);
+  CU_TRY(h, cudaMemcpyAsync(tmp.data(), h->st.trace, tmp.size() * 8, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  for (int t = 0; t < dm.T; ++t)
+    for (int b = 0; b < h->batch; ++b) active_mask[(size_t)t * h->batch + b] = tmp[(size_t)t * dm.B + b];
+  return PD_OK;
+}
+
+pd_status pd_get_logits(pd_handle *h, float *logits, int32_t *row_sub) {
+  if (!h) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_get_logits before pd_encode_context");
+  const size_t rows = (size_t)h->batch * h->dm.C;
+  if (logits) CU_TRY(h, cudaMemcpyAsync(logits, h->ptr<void>(h->lay.logits), rows * h->dm.V * 4, cudaMemcpyDeviceToHost, h->stream));
+  if (row_sub) CU_TRY(h, cudaMemcpyAsync(row_sub, h->st.prev_row_sub, rows * 4, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  return PD_OK;
+}
+
+pd_status pd_get_chosen(pd_handle *h, int32_t *chosen) {
+  if (!h || !chosen) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_get_chosen before pd_encode_context");
+  CU_TRY(h, cudaMemcpyAsync(chosen, h->st.chosen, (size_t)h->batch * h->dm.SM * (h->dm.MSL + 1) * 4, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  return PD_OK;
+}
+
+int32_t pd_rows_per_seq(const pd_handle *h) { return h ? h->dm.C : 0; }
+
+pd_status pd_debug_read(pd_handle *h, int32_t which, void *dst_host, size_t max_bytes, size_t *bytes_out) {
+  if (!h || !dst_host) return PD_ERR_ARG;
+  const Layout &L = h->lay;
+  const Region *r = nullptr;
+  switch (which) {
+    case PD_BUF_X: r = &L.x; break;
+    case PD_BUF_QKV: r = &L.qkv; break;
+    case PD_BUF_SELF_OUT: r = &L.self_out; break;
+    case PD_BUF_CROSS_Q: r = &L.cq; break;
+    case PD_BUF_CROSS_OUT: r = &L.cross_out; break;
+    case PD_BUF_STATE: r = &L.state; break;
+    default: return fail(h, PD_ERR_ARG, "pd_debug_read: unknown buffer");
+  }
+  size_t n = r->bytes < max_bytes ? r->bytes : max_bytes;
+  CU_TRY(h, cudaMemcpyAsync(dst_host, h->ws + r->off, n, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  if (bytes_out) *bytes_out = n;
+  return PD_OK;
+}
+
+pd_status pd_get_counters(const pd_handle *h, int64_t *own_kernel_launches, int64_t *gemm_calls) {
+  if (!h) return PD_ERR_ARG;
+  if (own_kernel_launches) *own_kernel_launches = h->own_launches;
+  if (gemm_calls) *gemm_calls = h->gemm_calls;
+  return PD_OK;
+}
+
+pd_status pd_reset_counters(pd_handle *h) {
+  if (!h) return PD_ERR_ARG;
+  h->own_launches = 0; h->gemm_calls = 0;
+  return PD_OK;
+}
+
+pd_status pd_profile_enable(pd_handle *h, int32_t on) {
+  if (!h) return PD_ERR_ARG;
+  h->profiling = on != 0;
+  return PD_OK;
+}
+
+pd_status pd_profile_read(pd_handle *h, double *ms, int64_t *launches) {
+  if (!h || !ms || !launches) return PD_ERR_ARG;
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  for (int k = 0; k < PD_PROF_COUNT; ++k) { ms[k] = 0.0; launches[k] = 0; }
+  for (const ProfRec &r : h->prof) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) { ms[r.kind] += t; launches[r.kind]++; }
+    h->ev_pool.push_back(r.a); h->ev_pool.push_back(r.b);
+  }
+  h->prof.clear();
+  return PD_OK;
+}
+
+pd_status pd_get_stats(pd_handle *h, int64_t *stats) {
+  if (!h || !stats) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_get_stats before pd_encode_context");
+  CU_TRY(h, cudaMemcpyAsync(stats, h->st.stats, PD_STAT_COUNT * 8, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  return PD_OK;
+}
+
+const char *pd_last_error(const pd_handle *h) { return h ? h->err.c_str() : "null handle"; }
+const char *pd_version(void) { return "pd-b200 0.1 (sm_100a)"; }
+
+void pd_destroy(pd_handle *h) {
+  if (!h) return;
+  drop_graph(h);
+  for (const ProfRec &r : h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+  if (h->pinned_flag) cudaFreeHost(h->pinned_flag);
+  if (h->blas) cublasDestroy(h->blas);
+  delete h;
+}
+
+}  // extern "C"

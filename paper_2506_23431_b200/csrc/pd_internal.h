@@ -1,0 +1,89 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pd.h"
+
+namespace pd {
+
+constexpr int kDh = 64;          // head width the kernels are written for
+constexpr int kMaxRows = 64;     // most subsequences active at once per sequence (sub_max <= 64)
+constexpr int kLayerTensors = 10;
+
+// header words of the state block
+enum { HDR_STEP_T = 0, HDR_ALL_DONE = 1, HDR_STATUS = 2, HDR_PAGE_BUMP = 3, HDR_BATCH = 4, HDR_N_DONE = 5,
+       HDR_TICKET = 6, HDR_WORDS = 16 };
+enum { SUB_NONE = 0, SUB_ACTIVE = 1, SUB_ENDED = 2 };
+
+// Shapes and rule parameters every kernel may need; passed by value.
+struct Dims {
+  int L, d, H, ff, V;
+  int B;        // max_batch
+  int ctx;      // max_ctx
+  int SM;       // sub_max
+  int dt;       // delta_t
+  int T;        // time_max
+  int MSL;      // max_sub_len
+  int C;        // rows per sequence
+  int P;        // page_tokens
+  int PPS;      // pages per subsequence
+  int pool;     // pool pages
+  int bos, eos, sep;
+  int pos_mode;
+  int n_dist;   // entries of the distance -> bucket table
+  float scale_log2e;  // attn_scale * log2(e)
+  float eps;
+};
+
+// Device pointers into the integer state block (all int32 unless noted).
+struct DecState {
+  int32_t *hdr;                 // [HDR_WORDS]
+  unsigned long long *stats;    // [PD_STAT_COUNT]
+  int32_t *k, *done, *steps, *n_active, *ctx_len, *seq_ticket;        // [B]
+  int32_t *start, *len, *state, *flag, *last_tok, *forced_len;        // [B*SM]
+  int32_t *row_sub, *prev_row_sub, *row_tok;                          // [B*C]
+  int32_t *page_table;          // [B*SM*PPS]
+  int32_t *tokens;              // [B*SM*MSL]
+  int32_t *chosen;              // [B*SM*(MSL+1)]
+  unsigned long long *trace;    // [T*B]
+};
+
+// Arguments of the attention kernels (self and cross share the struct).
+struct AttnArgs {
+  Dims dm;
+  DecState st;
+  int layer, batch, splits;
+  const void *q;            // [rows, d] dtype
+  const void *kv;           // self: page pool base; cross: kv_c base [L][B*ctx][2d]
+  void *out;                // [rows, d] dtype
+  float *part_o;            // [rows, H, splits, 64]
+  float *part_ml;           // [rows, H, splits, 2]
+  const int32_t *dist_bucket;  // [n_dist]
+  const float *rel_bias;       // [H, rel_buckets]
+  int rel_buckets;
+};
+
+// ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
+cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, const int32_t *ctx_len_dev,
+                               const int32_t *forced_len_dev, size_t state_words, int32_t *state_base, cudaStream_t s);
+cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x,
+                         cudaStream_t s);
+cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, const void *gain, void *out,
+                           cudaStream_t s);
+cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s);
+cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
+                          void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s);
+cudaError_t launch_zero_ctx_pad(const Dims &dm, const DecState &st, int batch, int dtype, void *kv_c, cudaStream_t s);
+cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
+cudaError_t launch_attn_merge(const AttnArgs &a, int dtype, cudaStream_t s);
+cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, cudaStream_t s);
+cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
+                                const int32_t *teacher, cudaStream_t s);
+int cross_attn_tma_smem_bytes();
+cudaError_t cross_attn_tma_prepare();   // once per device, outside any stream capture
+
+}  // namespace pd

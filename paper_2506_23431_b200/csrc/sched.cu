@@ -1,0 +1,169 @@
+// Fused logits-argmax + scheduler.  One CTA per row scans the row's fp32 logits for the
+// greedy choice of Eq. 4 (ties to the lowest id); the CTA that finishes a sequence's last row
+// then runs that sequence's part of Algorithm 1 for the step: append the tokens (lines 9-11),
+// retire subsequences on eos/sep, the stop test (lines 12-13), the admission that lines 5-7
+// perform at the top of the next step, and the compaction of the active rows for it.  No CTA
+// ever waits for another: the hand-over is an atomic ticket after a memory fence.
+#include <limits.h>
+
+#include "pd_internal.h"
+
+namespace pd {
+
+constexpr int AT = 256;
+
+__device__ __forceinline__ void better(float &bv, int &bi, float v, int i) {
+  if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+}
+
+__device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch, int b, const int32_t *teacher) {
+  const int t = st.hdr[HDR_STEP_T];
+  const int C = dm.C, SM = dm.SM;
+  int nact = st.n_active[b];
+  int k = st.k[b];
+  for (int c = 0; c < C; ++c) st.prev_row_sub[b * C + c] = st.row_sub[b * C + c];
+  if (st.done[b] || st.hdr[HDR_STATUS] != 0) {
+    if (!st.done[b]) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
+    for (int c = 0; c < C; ++c) st.row_sub[b * C + c] = 0;
+    st.n_active[b] = 0;
+    return;
+  }
+  // traffic counters of the step just executed (before any length changes)
+  int i_max = 0;
+  for (int c = 0; c < nact; ++c) i_max = max(i_max, st.row_sub[b * C + c]);
+  unsigned long long nvis = 0;
+  for (int i = 1; i <= i_max; ++i) nvis += (unsigned long long)(st.len[b * SM + i - 1] + 1);
+  atomicAdd(&st.stats[PD_STAT_SELF_ENTRIES], nvis);
+  if (nact > 0) atomicAdd(&st.stats[PD_STAT_CROSS_KEYS], (unsigned long long)st.ctx_len[b]);
+  atomicAdd(&st.stats[PD_STAT_TOKENS], (unsigned long long)nact);
+
+  unsigned long long mask = 0ull;
+  for (int c = 0; c < nact; ++c) {
+    const int i = st.row_sub[b * C + c];
+    const int sidx = b * SM + i - 1;
+    const int len = st.len[sidx];
+    const int fl = st.forced_len[sidx];
+    int own = __ldcg(&st.row_tok[b * C + c]);
+    if (fl >= 0) { if (len >= fl) own = dm.sep; }
+    else if (len >= dm.MSL) own = dm.sep;
+    st.chosen[(size_t)sidx * (dm.MSL + 1) + len] = own;
+    int tok = own;
+    if (teacher != nullptr) { int tt = teacher[sidx]; if (tt >= 0) tok = tt; }
+    if (len >= dm.MSL) { tok = dm.sep; if (fl < 0) st.flag[sidx] |= PD_FLAG_CAPPED; }
+    if (tok == dm.eos || tok == dm.sep) {
+      st.state[sidx] = SUB_ENDED;
+      st.flag[sidx] |= PD_FLAG_COMPLETE;
+    } else {
+      st.tokens[(size_t)sidx * dm.MSL + len] = tok;
+      st.len[sidx] = len + 1;
+      st.last_tok[sidx] = tok;
+    }
+    mask |= 1ull << (i - 1);
+  }
+  st.trace[(size_t)(t - 1) * dm.B + b] = mask;
+
+  int ended = 0;
+  for (int i = 1; i <= k; ++i) ended += st.state[b * SM + i - 1] == SUB_ENDED;
+  bool done = false;
+  if (ended == k) {
+    done = true;                                   // every subsequence has produced its terminator
+  } else if (t >= dm.T) {
+    done = true;                                   // time_max reached with subsequences still open
+    for (int i = 1; i <= k; ++i)
+      if (st.state[b * SM + i - 1] == SUB_ACTIVE) st.flag[b * SM + i - 1] |= PD_FLAG_TRUNCATED;
+  } else if (t % dm.dt == 0 && k < SM) {           // step t+1 satisfies (t+1-1) mod delta_t == 0
+    const int sidx = b * SM + k;
+    k += 1;
+    st.k[b] = k;
+    st.start[sidx] = t + 1;
+    st.len[sidx] = 0;
+    st.state[sidx] = SUB_ACTIVE;
+    st.flag[sidx] = 0;
+    st.last_tok[sidx] = dm.bos;
+  }
+  int n = 0;
+  if (done) {
+    st.done[b] = 1;
+    st.steps[b] = t;
+    atomicAdd(&st.hdr[HDR_N_DONE], 1);
+  } else {
+    for (int i = 1; i <= k; ++i) {
+      const int sidx = b * SM + i - 1;
+      if (st.state[sidx] != SUB_ACTIVE) continue;
+      if (n >= C) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_STATE); break; }
+      st.row_sub[b * C + n++] = i;
+      const int p = st.len[sidx];                  // entry the next step will write
+      if (p % dm.P == 0) {
+        int pg = atomicAdd(&st.hdr[HDR_PAGE_BUMP], 1);
+        if (pg >= dm.pool) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_POOL_EXHAUSTED); pg = 0; }
+        st.page_table[(size_t)sidx * dm.PPS + p / dm.P] = pg;
+        atomicAdd(&st.stats[PD_STAT_PAGES], 1ull);
+      }
+    }
+  }
+  for (int c = n; c < C; ++c) st.row_sub[b * C + c] = 0;
+  st.n_active[b] = n;
+}
+
+__global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, int batch, const float *__restrict__ logits,
+                                                          const int32_t *__restrict__ teacher) {
+  __shared__ float sv[AT / 32];
+  __shared__ int si[AT / 32];
+  __shared__ int is_last;
+  const int r = blockIdx.x, tid = threadIdx.x;
+  const int b = r / dm.C;
+  const int i = st.row_sub[r];
+  if (i > 0) {
+    const int sidx = b * dm.SM + i - 1;
+    const int fl = st.forced_len[sidx];
+    const bool bar = fl >= 0 && st.len[sidx] < fl;     // terminators cannot win before the forced length
+    const float *row = logits + (size_t)r * dm.V;
+    float bv = -INFINITY;
+    int bi = INT_MAX;
+    for (int v = tid; v < dm.V; v += AT) {
+      float x = __ldcs(row + v);
+      if (bar && (v == dm.eos || v == dm.sep)) continue;
+      better(bv, bi, x, v);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      better(bv, bi, ov, oi);
+    }
+    if ((tid & 31) == 0) { sv[tid >> 5] = bv; si[tid >> 5] = bi; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < AT / 32; ++w) better(bv, bi, sv[w], si[w]);
+      st.row_tok[r] = bi == INT_MAX ? 0 : bi;
+    }
+  }
+  if (tid == 0) {
+    __threadfence();
+    int ticket = atomicAdd(&st.seq_ticket[b], 1);
+    is_last = ticket == dm.C - 1;
+  }
+  __syncthreads();
+  if (!is_last || tid != 0) return;
+  __threadfence();
+  st.seq_ticket[b] = 0;
+  schedule_sequence(dm, st, batch, b, teacher);
+  __threadfence();
+  if (atomicAdd(&st.hdr[HDR_TICKET], 1) == batch - 1) {   // last sequence of the step
+    __threadfence();
+    st.hdr[HDR_TICKET] = 0;
+    const int n_done = atomicAdd(&st.hdr[HDR_N_DONE], 0);
+    if (st.hdr[HDR_ALL_DONE] == 0) {
+      atomicAdd(&st.stats[PD_STAT_STEPS], 1ull);
+      if (n_done >= batch) st.hdr[HDR_ALL_DONE] = 1;
+      else st.hdr[HDR_STEP_T] = st.hdr[HDR_STEP_T] + 1;
+    }
+  }
+}
+
+cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
+                                const int32_t *teacher, cudaStream_t s) {
+  argmax_sched_kernel<<<batch * dm.C, AT, 0, s>>>(dm, st, batch, logits, teacher);
+  return cudaGetLastError();
+}
+
+}  // namespace pd

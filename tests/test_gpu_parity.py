@@ -1,0 +1,181 @@
+"""GPU parity tests: the CUDA library, called through the C ABI, against the CPU fp64 oracle on
+the same seeded inputs.  Bars: schedule / active sets / streams bit-exact; logits within
+1e-4 (fp32 storage) or 2e-2 (bf16 storage) max-abs; greedy ids identical wherever the oracle's
+top-2 margin exceeds 5e-2."""
+import numpy as np
+import pytest
+
+from paper_2506_23431_b200 import workload as W
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def make(wl, rows=None, ragged=False, **dec_kw):
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    weights = W.make_weights(wl)
+    mem = W.make_encoder_memory(wl)
+    ctx_len = W.make_ctx_len(wl, ragged=ragged)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, **dec_kw)
+    rows = list(range(wl.batch)) if rows is None else rows
+    return weights, mem, ctx_len, dec, rows
+
+
+def check(wl, rows=None, ragged=False, forced=True, free_run=True, **dec_kw):
+    weights, mem, ctx_len, dec, rows = make(wl, rows, ragged, **dec_kw)
+    fl = W.make_forced_len(wl) if forced else None
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, fl)
+    mem_dev = dec.device_memory(mem)
+    stats = parity.replay_compare(dec, wl, mem_dev, ctx_len, fl, runs)
+    assert stats["logits"] > 0 and stats["choices"] > 0
+    if free_run:
+        parity.free_run_compare(dec, wl, mem_dev, ctx_len, fl, runs)
+    dec.close()
+    return stats
+
+
+TINY = W.CONFIGS["tiny"]
+# scaled-down relatives of the bf16 configs: several tiles, ragged tails, page crossings
+SMALL_BF16 = dict(n_layers=2, d_model=128, n_heads=2, d_ff=256, vocab=1000, norm_gain_std=0.1)
+
+
+def test_tiny_fp32_t5_bias_full_config():
+    s = check(TINY)
+    assert s["max_err"] < 1e-4
+
+
+def test_tiny_fp32_rope():
+    check(TINY.scaled(pos_mode=W.POS_ROPE, norm_gain_std=0.1))
+
+
+def test_tiny_fp32_without_graph_and_with_splits():
+    check(TINY.scaled(norm_gain_std=0.1), use_graph=False, self_splits=3, cross_splits=2)
+
+
+def test_fp32_batch_ragged_context_page_size_32():
+    wl = TINY.scaled(batch=3, ctx=200, page_tokens=32, sub_max=5, delta_t=3, max_sub_len=40,
+                     length_dist=("uniform", 1, 40), time_max=80, norm_gain_std=0.1, vocab=777)
+    check(wl, ragged=True, self_splits=2, cross_splits=3)
+
+
+def test_fp32_free_running_cap_and_time_max():
+    # no forced lengths: random weights almost never emit a terminator, so subsequences run into
+    # the max_sub_len cap; time_max then cuts the rest
+    wl = TINY.scaled(batch=2, sub_max=6, delta_t=2, max_sub_len=7, time_max=15, vocab=300)
+    weights, mem, ctx_len, dec, rows = make(wl)
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, None)
+    assert any(f & 4 for r in runs.values() for f in r["flags"])
+    assert any(f & 2 for r in runs.values() for f in r["flags"])
+    parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, None, runs)
+    dec.close()
+
+
+def test_fp32_sub_max_1_is_sequential_decoding():
+    wl = TINY.scaled(sub_max=1, max_sub_len=30, length_dist=("uniform", 30, 30), time_max=40)
+    check(wl)
+
+
+@pytest.mark.parametrize("pos_mode", [W.POS_T5_BIAS, W.POS_ROPE])
+def test_small_bf16_tma_cross_attention(pos_mode):
+    wl = W.CONFIGS["bart_base"].scaled(name="small_bf16", batch=3, ctx=300, sub_max=6, delta_t=2, max_sub_len=20,
+                                       length_dist=("uniform", 1, 20), time_max=48, pos_mode=pos_mode, **SMALL_BF16)
+    s = check(wl, ragged=True, cross_splits=2, self_splits=2)
+    assert s["max_err"] < 2e-2
+
+
+def test_small_bf16_many_short_subsequences_two_query_tiles():
+    # 20 rows per sequence: exercises the two-tile (32-row) tensor-core variant
+    wl = W.CONFIGS["keyphrase"].scaled(name="small_kp", batch=2, ctx=130, sub_max=24, delta_t=1, max_sub_len=19,
+                                       length_dist=("uniform", 3, 19), time_max=48, **SMALL_BF16)
+    check(wl, ragged=True)
+
+
+def test_small_bf16_wide_rows_use_cuda_core_cross_attention():
+    # more than 32 rows per sequence: falls back to the CUDA-core cross-attention kernel
+    wl = W.CONFIGS["keyphrase"].scaled(name="small_wide", batch=1, ctx=64, sub_max=40, delta_t=1, max_sub_len=36,
+                                       length_dist=("uniform", 30, 36), time_max=80, **SMALL_BF16)
+    check(wl, free_run=False)
+
+
+def test_batch_independence():
+    """B sequences share a step clock and nothing else: decoding a row alone gives its streams."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = TINY.scaled(batch=4, ctx=96, vocab=500)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch)
+    dec.encode_context(dec.device_memory(mem), ctx_len, fl)
+    dec.run()
+    full = dec.collect()
+    for b in (0, 3):
+        dec.encode_context(dec.device_memory(mem[b:b + 1]), ctx_len[b:b + 1], fl[b:b + 1])
+        dec.run()
+        one = dec.collect()
+        assert np.array_equal(one["tokens"][0], full["tokens"][b])
+        assert one["steps"][0] == full["steps"][b]
+    dec.close()
+
+
+def test_pool_exhaustion_is_reported_not_faulted():
+    from paper_2506_23431_b200.binding import PipelinedDecoder, PdError
+    wl = TINY.scaled(batch=2, vocab=300)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, pool_pages=3)
+    dec.encode_context(dec.device_memory(mem), ctx_len, W.make_forced_len(wl))
+    with pytest.raises(PdError) as e:
+        dec.run()
+        dec.collect()
+    assert e.value.status == -4
+    dec.close()
+
+
+def test_call_order_and_argument_errors():
+    from paper_2506_23431_b200.binding import PipelinedDecoder, PdError
+    wl = TINY.scaled(vocab=300)
+    weights, mem = W.make_weights(wl), W.make_encoder_memory(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, 1)
+    with pytest.raises(PdError) as e:
+        dec.step()
+    assert e.value.status == -2
+    with pytest.raises(PdError) as e:
+        dec.encode_context(dec.device_memory(mem), [wl.ctx + 1], None)
+    assert e.value.status == -1
+    with pytest.raises(PdError) as e:
+        dec.encode_context(dec.device_memory(mem), [wl.ctx], np.full((1, wl.sub_max), wl.max_sub_len + 1))
+    assert e.value.status == -1
+    dec.close()
+
+
+def test_generate_host_matches_stepwise_run():
+    import torch
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = TINY.scaled(batch=2, vocab=400)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl)
+    fl = W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch)
+    dec.encode_context(dec.device_memory(mem), ctx_len, fl)
+    dec.run()
+    a = dec.collect()
+    host = torch.from_numpy(mem).pin_memory()
+    b = dec.generate_host(host, ctx_len, fl)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+    own, gemms = dec.counters()
+    assert own > 0 and gemms > 0
+    st = dec.stats()
+    assert st["tokens"] == int((fl + 1).sum()) and st["steps"] == int(a["steps"].max())
+    dec.close()
+
+
+FULL = [("bart_base", 2e-2), ("long_context", 2e-2), ("summarisation", 2e-2), ("keyphrase", 2e-2)]
+
+
+@pytest.mark.parametrize("name,tol", FULL)
+def test_full_size_configs_on_sampled_rows(name, tol):
+    """The four bf16 configurations at full size, in the launch configuration the benchmark
+    times (CUDA graph, automatic splits); the oracle decodes batch rows 0 and B-1."""
+    wl = W.CONFIGS[name]
+    s = check(wl, rows=[0, wl.batch - 1], free_run=True)
+    assert s["max_err"] <= tol
+    print(f"{name}: max logit error {s['max_err']:.3e} over {s['logits']} logits, "
+          f"{s['choices']} choices compared, {s['low_margin']} below margin")
