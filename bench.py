@@ -158,6 +158,10 @@ def main():
     ap.add_argument("--cpu-baseline-steps", type=int, default=40)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--single-decode", action="store_true",
+                    help="run exactly one encode + decode and exit (no timing): the command profilers are pointed at")
+    ap.add_argument("--time-steps", type=int, default=0,
+                    help="with --single-decode: stop after this many time-steps (0 = until done)")
     ap.add_argument("--self-splits", type=int, default=0)
     ap.add_argument("--cross-splits", type=int, default=0)
     args = ap.parse_args()
@@ -194,6 +198,20 @@ def main():
     mem_dev = dec.device_memory(mem)
     host_mem = torch.from_numpy(mem).to(dec.tdtype).pin_memory()
     e = 2 if wl.dtype == "bf16" else 4
+
+    if args.single_decode:
+        dec.encode_context(mem_dev, ctx_len, fl)
+        if args.time_steps > 0:
+            for _ in range(args.time_steps):
+                dec.step()
+            dec.done()
+        else:
+            dec.run(poll_every=8)
+        own, gemms = dec.counters()
+        print(json.dumps({"single_decode": wl.name, "time_steps": int(dec.stats()["steps"]), "own_launches": own,
+                          "cublas_gemms": gemms}))
+        dec.close()
+        return
 
     def one_decode(timed):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]

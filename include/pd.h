@@ -194,6 +194,32 @@ enum { PD_STAT_TOKENS = 0, PD_STAT_STEPS = 1, PD_STAT_SELF_ENTRIES = 2, PD_STAT_
        PD_STAT_PAGES = 4, PD_STAT_COUNT = 8 };
 PD_API pd_status pd_get_stats(pd_handle *h, int64_t *stats);
 
+/* The batched cross-attention step alone (Section 3.2: every generated token attends to all
+ * context tokens; Eq. 3's Decoder(G, H^E) reads H^E only through this step), on caller-supplied
+ * tensors and without a handle: the kernels are the ones pd_step launches.  For sequence b,
+ * rows b*rows_per_seq .. b*rows_per_seq + n_rows[b] - 1 of q are the queries of its active
+ * subsequences; each attends, per head, to context positions 0 .. ctx_len[b]-1 with weights
+ * softmax(attn_scale * q.k) and no positional term:  out = softmax(attn_scale * q K^T) V.
+ *   dtype        PD_DTYPE_FP32 or PD_DTYPE_BF16: element type of q, kv and out
+ *   q, out       device [batch*rows_per_seq, n_heads*64]; rows at or beyond n_rows[b] of a
+ *                sequence are not read and come back as zeros
+ *   kv           device [batch, max_ctx, 2*n_heads*64], 16-byte aligned: per context position
+ *                the keys of all heads, then the values of all heads; positions at or beyond
+ *                ctx_len[b] are ignored (they may hold anything)
+ *   n_rows       device int32 [batch], 0..rows_per_seq;  ctx_len  device int32 [batch], 1..max_ctx
+ *   splits       1..32: split-K factor over the context (partials are merged by a second kernel)
+ *   scratch      device, 256-byte aligned, at least pd_cross_attention_scratch_bytes(...): a
+ *                256-byte header the call clears (int32 word 2 receives PD_ERR_TIMEOUT if a
+ *                bounded wait inside the kernel expired), then the split-K partials
+ * rows_per_seq <= 64.  Enqueues on cuda_stream (a cudaStream_t) and returns; allocates nothing on
+ * the device.  The caller owns every buffer and keeps it alive until the stream has passed the
+ * call.  PD_ERR_ARG for null pointers or sizes out of range, PD_ERR_WORKSPACE for a scratch
+ * that is too small, PD_ERR_CUDA if a launch fails. */
+PD_API size_t pd_cross_attention_scratch_bytes(int32_t batch, int32_t rows_per_seq, int32_t n_heads, int32_t splits);
+PD_API pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_per_seq, int32_t n_heads, int32_t max_ctx,
+                             float attn_scale, int32_t splits, const void *q, const void *kv, const int32_t *n_rows,
+                             const int32_t *ctx_len, void *out, void *scratch, size_t scratch_bytes, void *cuda_stream);
+
 PD_API const char *pd_last_error(const pd_handle *h);
 PD_API const char *pd_version(void);
 

@@ -65,6 +65,9 @@ _SIGS = {
     "pd_profile_enable": (C.c_int, [_H, C.c_int32]),
     "pd_profile_read": (C.c_int, [_H, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "pd_get_stats": (C.c_int, [_H, C.POINTER(C.c_int64)]),
+    "pd_cross_attention_scratch_bytes": (C.c_size_t, [C.c_int32] * 4),
+    "pd_cross_attention": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p, C.c_size_t,
+                                                                                                  C.c_void_p]),
     "pd_last_error": (C.c_char_p, [_H]),
     "pd_version": (C.c_char_p, []),
     "pd_destroy": (None, [_H]),
@@ -287,6 +290,50 @@ class PipelinedDecoder:
         self._check(_lib.pd_get_stats(self._h, a), "pd_get_stats")
         return {"tokens": a[PD_STAT_TOKENS], "steps": a[PD_STAT_STEPS], "self_entries": a[PD_STAT_SELF_ENTRIES],
                 "cross_keys": a[PD_STAT_CROSS_KEYS], "pages": a[PD_STAT_PAGES]}
+
+
+def _attention_call(fn_name: str, q, kv, n_rows, ctx_len, attn_scale: float, splits: int, scratch):
+    """Shared marshalling of the stand-alone cross-attention entry points.  q [batch, rows, heads*64],
+    kv [batch, ctx, 2*heads*64] CUDA tensors of one dtype (float32 or bfloat16); n_rows, ctx_len CUDA
+    int32 [batch].  Runs on torch's current stream; returns out (same shape as q)."""
+    import torch
+    if q.dtype not in (torch.float32, torch.bfloat16) or kv.dtype != q.dtype:
+        raise ValueError("q and kv must both be float32 or both bfloat16")
+    for t in (q, kv, n_rows, ctx_len):
+        if not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+    batch, rows, hd = q.shape
+    heads = hd // 64
+    if hd % 64 or kv.shape[0] != batch or kv.shape[2] != 2 * hd or n_rows.dtype != torch.int32 \
+            or ctx_len.dtype != torch.int32 or n_rows.numel() != batch or ctx_len.numel() != batch:
+        raise ValueError("shape mismatch")
+    out = torch.empty_like(q)
+    dt = PD_DTYPE_BF16 if q.dtype == torch.bfloat16 else PD_DTYPE_FP32
+    stream = torch.cuda.current_stream(q.device).cuda_stream
+    args = [dt, batch, rows, heads, int(kv.shape[1]), float(attn_scale), int(splits), C.c_void_p(q.data_ptr()),
+            C.c_void_p(kv.data_ptr()), C.c_void_p(n_rows.data_ptr()), C.c_void_p(ctx_len.data_ptr()),
+            C.c_void_p(out.data_ptr())]
+    if scratch is not None:
+        args += [C.c_void_p(scratch.data_ptr()), C.c_size_t(scratch.numel() * scratch.element_size())]
+    args.append(C.c_void_p(stream))
+    st = getattr(_lib, fn_name)(*args)
+    if st != PD_OK:
+        raise PdError(st, fn_name)
+    return out
+
+
+def cross_attention_scratch_bytes(batch: int, rows_per_seq: int, n_heads: int, splits: int) -> int:
+    return int(_lib.pd_cross_attention_scratch_bytes(batch, rows_per_seq, n_heads, splits))
+
+
+def cross_attention(q, kv, n_rows, ctx_len, attn_scale: float, splits: int = 1, scratch=None):
+    """pd_cross_attention on torch CUDA tensors; `scratch` (uint8 CUDA tensor, 256-byte aligned) is
+    allocated here when not given."""
+    import torch
+    if scratch is None:
+        n = cross_attention_scratch_bytes(q.shape[0], q.shape[1], q.shape[2] // 64, splits)
+        scratch = torch.empty(max(n, 256), dtype=torch.uint8, device=q.device)
+    return _attention_call("pd_cross_attention", q, kv, n_rows, ctx_len, attn_scale, splits, scratch)
 
 
 def version() -> str:

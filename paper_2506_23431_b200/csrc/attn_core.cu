@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
   const int tid = threadIdx.x;
   const int S = a.st.n_active[b];
   const int row0 = b * dm.C;
-  const int t = a.st.hdr[HDR_STEP_T];
+  const int t = SELF ? a.st.hdr[HDR_STEP_T] : 0;
   const T *qbuf = (const T *)a.q;
   T *out = (T *)a.out;
 
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
   }
   if (tid < kMaxRows) {
     m_s[tid] = -INFINITY; l_s[tid] = 0.f; corr_s[tid] = 1.f;
-    sub_s[tid] = tid < S ? a.st.row_sub[row0 + tid] : 0;
+    sub_s[tid] = (SELF && tid < S) ? a.st.row_sub[row0 + tid] : 0;
   }
   const bool use_bias = SELF && dm.pos_mode == PD_POS_T5_BIAS;
   if (use_bias)
@@ -92,9 +92,8 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
       n_valid = min(dm.P, n_entries - e0);
       if (n_valid <= 0) continue;
       int page = a.st.page_table[(size_t)sidx * dm.PPS + j];
-      size_t base = ((((size_t)a.layer * dm.pool + page) * 2) * dm.H + h) * dm.P * kDh;
-      kp = (const T *)a.kv + base;
-      vp = kp + (size_t)dm.H * dm.P * kDh;
+      kp = (const T *)a.kv + kv_block_offset(a.layer, dm.pool, page, dm.H, h, dm.P);
+      vp = kp + (size_t)dm.P * kDh;
       kstride = kDh;
       k_sub = ksub;
       k_tau0 = a.st.start[sidx] - 1 + e0;  // timestamp of the tile's first entry
@@ -109,8 +108,9 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
     __syncthreads();   // previous tile fully consumed
     for (int idx = tid; idx < n_valid * kDh; idx += NT) {
       int e = idx / kDh, c = idx % kDh;
-      Ks[e][c] = ld_f<T>(kp + e * kstride + c);
-      Vs[e][c] = ld_f<T>(vp + e * kstride + c);
+      size_t off = SELF ? kv_entry_offset<T>(e, c) : e * kstride + c;
+      Ks[e][c] = ld_f<T>(kp + off);
+      Vs[e][c] = ld_f<T>(vp + off);
     }
     __syncthreads();
     // scores in the log2 domain

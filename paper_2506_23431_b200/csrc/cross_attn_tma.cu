@@ -173,6 +173,19 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
       break;
     }
     const uint32_t kbase = base + s * XSTAGE_BYTES, vbase = kbase + XTILE_BYTES;
+    const int key0 = (t0 + it) * XK + kb;          // context position of this warp's first key
+    const bool ragged = key0 + 32 > ctx_len;
+    if (ragged) {
+      // Rows at or beyond ctx_len hold whatever follows in memory (or the fill value).  Their
+      // weights are exactly 0 below; zero the value rows so that 0 never multiplies a non-finite.
+      if (key0 + lane >= ctx_len) {
+        uint4 *vrow = reinterpret_cast<uint4 *>(smem_al + (vbase - base) + (kb + lane) * 128);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage's next bulk copy
+      }
+      __syncwarp();
+    }
 
     // ---- scores: S[mt][nt] = Q (16 x 64) . K^T (64 x 8 keys)
     float sc[MT][4][4];
@@ -196,8 +209,6 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
       }
     }
     // ---- scale, mask the ragged end of the context, online softmax
-    const int key0 = (t0 + it) * XK + kb;          // context position of this warp's first key
-    const bool ragged = key0 + 32 > ctx_len;
     uint32_t pf[MT][2][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
@@ -310,6 +321,31 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
       if (col == 0) { a.part_ml[pi * 2] = M; a.part_ml[pi * 2 + 1] = L; }
     }
   }
+}
+
+// Tensor map of the projected context keys/values seen as a 2-D bf16 array [rows, 2*d] (row =
+// one context position of one sequence and layer; columns k | v, head-major): boxes of 128 rows
+// x 64 columns (one head's keys or values of one tile), 128-byte swizzle.  *driver_code gets the
+// CUresult when the encode itself fails.
+cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int d, int *driver_code) {
+  typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  if (driver_code) *driver_code = 0;
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+  cuuint64_t gdim[2] = {(cuuint64_t)2 * d, (cuuint64_t)rows};
+  cuuint64_t gstride[1] = {(cuuint64_t)2 * d * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kDh, (cuuint32_t)XK};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = ((EncodeFn)fn)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { if (driver_code) *driver_code = (int)r; return cudaErrorInvalidValue; }
+  return cudaSuccess;
 }
 
 cudaError_t cross_attn_tma_prepare() {

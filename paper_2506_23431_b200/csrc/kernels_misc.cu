@@ -1,5 +1,5 @@
 // Small kernels of the decode step: state reset, embedding gather, RMSNorm, ReLU,
-// KV-append with the positional write, and zeroing of context rows beyond ctx_len.
+// KV-append with the positional write.
 #include "pd_internal.h"
 
 namespace pd {
@@ -167,8 +167,8 @@ __global__ void append_kernel(Dims dm, DecState st, int layer, const float *__re
     }
     q_out[(size_t)r * dm.d + col] = from_f<T>(q0);
     q_out[(size_t)r * dm.d + col + 1] = from_f<T>(q1);
-    size_t base = ((((size_t)layer * dm.pool + page) * 2) * dm.H + h) * dm.P * kDh + (size_t)slot * kDh + dd;
-    size_t vofs = (size_t)dm.H * dm.P * kDh;
+    size_t base = kv_block_offset(layer, dm.pool, page, dm.H, h, dm.P) + kv_entry_offset<T>(slot, dd);
+    size_t vofs = (size_t)dm.P * kDh;
     kv_pool[base] = from_f<T>(k0);
     kv_pool[base + 1] = from_f<T>(k1);
     kv_pool[base + vofs] = from_f<T>(v0);
@@ -185,27 +185,6 @@ cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int lay
                                                          (__nv_bfloat16 *)kv_pool, rope_tab);
   else
     append_kernel<float><<<rows, threads, 0, s>>>(dm, st, layer, qkv, (float *)q_out, (float *)kv_pool, rope_tab);
-  return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------------------------
-// Context rows at or beyond ctx_len[b] never take part in cross-attention; zero their projected
-// keys/values so that a masked weight of exactly 0 never multiplies a non-finite value.
-template <typename T>
-__global__ void zero_ctx_pad_kernel(Dims dm, DecState st, T *kv_c) {
-  int b = blockIdx.y, l = blockIdx.z;
-  int cl = st.ctx_len[b];
-  size_t w = 2 * (size_t)dm.d;
-  for (int pos = cl + blockIdx.x; pos < dm.ctx; pos += gridDim.x) {
-    T *row = kv_c + (((size_t)l * dm.B + b) * dm.ctx + pos) * w;
-    for (size_t c = threadIdx.x; c < w; c += blockDim.x) row[c] = from_f<T>(0.f);
-  }
-}
-
-cudaError_t launch_zero_ctx_pad(const Dims &dm, const DecState &st, int batch, int dtype, void *kv_c, cudaStream_t s) {
-  dim3 grid(32, batch, dm.L);
-  if (dtype == PD_DTYPE_BF16) zero_ctx_pad_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(dm, st, (__nv_bfloat16 *)kv_c);
-  else zero_ctx_pad_kernel<float><<<grid, 256, 0, s>>>(dm, st, (float *)kv_c);
   return cudaGetLastError();
 }
 

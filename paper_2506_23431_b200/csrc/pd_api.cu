@@ -226,6 +226,7 @@ pd_status enqueue_step(pd_handle *h) {
   void *ffn = h->ptr<void>(h->lay.ffn);
   float *logits = h->ptr<float>(h->lay.logits);
   const bool tma_cross = dt == PD_DTYPE_BF16 && h->have_tmap && dm.C <= 32;
+  const bool tc_self = dt == PD_DTYPE_BF16 && self_attn_tc_supported(dm);
 
   OWN(h, PD_PROF_OTHER, launch_embed(dm, h->st, h->batch, dt, h->w.embed, x, s));
   for (int l = 0; l < dm.L; ++l) {
@@ -237,7 +238,8 @@ pd_status enqueue_step(pd_handle *h) {
     {
       AttnArgs a = attn_args(h, l, true);
       ProfScope ps(h, PD_PROF_SELF_ATTN);
-      CU_TRY(h, launch_attn_core(a, dt, true, s));
+      if (tc_self) CU_TRY(h, launch_self_attn_tc(a, s));
+      else CU_TRY(h, launch_attn_core(a, dt, true, s));
       h->own_launches++;
       if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, s)); h->own_launches++; }
     }
@@ -272,22 +274,11 @@ int t5_bucket(int dist, int num_buckets, int max_dist) {
 }
 
 pd_status make_tensor_map(pd_handle *h) {
-  typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  void *fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  CU_TRY(h, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-  if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return fail(h, PD_ERR_CUDA, "cuTensorMapEncodeTiled not available");
   const Dims &dm = h->dm;
-  cuuint64_t gdim[2] = {(cuuint64_t)2 * dm.d, (cuuint64_t)dm.L * dm.B * dm.ctx};
-  cuuint64_t gstride[1] = {(cuuint64_t)2 * dm.d * 2};
-  cuuint32_t box[2] = {(cuuint32_t)kDh, 128u};
-  cuuint32_t estr[2] = {1u, 1u};
-  CUresult r = ((EncodeFn)fn)(&h->tmap_kvc, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->ptr<void>(h->lay.kv_c), gdim, gstride, box,
-                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return fail(h, PD_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+  int code = 0;
+  cudaError_t e = encode_ctx_kv_tensor_map(&h->tmap_kvc, h->ptr<void>(h->lay.kv_c), (uint64_t)dm.L * dm.B * dm.ctx, dm.d, &code);
+  if (e != cudaSuccess) return fail(h, PD_ERR_CUDA, std::string("tensor map for the context keys/values: ") + cudaGetErrorString(e) +
+                                                    " (driver code " + std::to_string(code) + ")");
   h->have_tmap = true;
   return PD_OK;
 }
@@ -375,6 +366,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
     if (s != PD_OK) return bail(s);
     if (cross_attn_tma_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
   }
+  if (cfg->dtype == PD_DTYPE_BF16 && self_attn_tc_supported(dm) && self_attn_tc_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
   *out = h;
   return PD_OK;
 }
@@ -426,7 +418,6 @@ pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ct
     uint8_t *dst = h->ptr<uint8_t>(L.kv_c) + (size_t)l * dm.B * dm.ctx * 2 * dm.d * e;
     PD_TRY(gemm(h, false, batch * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5], dst, false, 0.f));
   }
-  OWN(h, PD_PROF_OTHER, launch_zero_ctx_pad(dm, h->st, batch, h->cfg.dtype, h->ptr<void>(L.kv_c), s));
   h->encoded = true;
   h->steps_enqueued = 0;
   return PD_OK;

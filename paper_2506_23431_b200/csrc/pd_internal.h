@@ -13,6 +13,21 @@ namespace pd {
 constexpr int kDh = 64;          // head width the kernels are written for
 constexpr int kMaxRows = 64;     // most subsequences active at once per sequence (sub_max <= 64)
 constexpr int kLayerTensors = 10;
+constexpr size_t kOpHeaderBytes = 256;   // header (HDR_* words) at the start of a stand-alone op's scratch
+
+// KV pool layout: [layer][page][head][K | V][page_tokens][64].  The keys of one (page, head) are
+// page_tokens * 64 contiguous elements, followed by its values.  With 2-byte elements the eight
+// 16-byte chunks of an entry are stored swizzled (chunk c of entry e at chunk c ^ (e & 7)), so a
+// linear copy of a block into shared memory is already in the layout ldmatrix reads without
+// bank conflicts.  Offset of element (entry e, column c) inside a block's keys (or values):
+template <typename T>
+__host__ __device__ __forceinline__ size_t kv_entry_offset(int e, int c) {
+  if (sizeof(T) == 2) return (size_t)e * kDh + ((((c >> 3) ^ (e & 7)) << 3) | (c & 7));
+  return (size_t)e * kDh + c;
+}
+__host__ __device__ __forceinline__ size_t kv_block_offset(int layer, int pool, int page, int H, int h, int P) {
+  return ((((size_t)layer * pool + page) * H + h) * 2) * P * kDh;
+}
 
 // header words of the state block
 enum { HDR_STEP_T = 0, HDR_ALL_DONE = 1, HDR_STATUS = 2, HDR_PAGE_BUMP = 3, HDR_BATCH = 4, HDR_N_DONE = 5,
@@ -77,13 +92,25 @@ cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, 
 cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s);
 cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
                           void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s);
-cudaError_t launch_zero_ctx_pad(const Dims &dm, const DecState &st, int batch, int dtype, void *kv_c, cudaStream_t s);
 cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
 cudaError_t launch_attn_merge(const AttnArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, cudaStream_t s);
+bool self_attn_tc_supported(const Dims &dm);
+cudaError_t self_attn_tc_prepare();     // once per device, outside any stream capture
+cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s);
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
                                 const int32_t *teacher, cudaStream_t s);
+cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int d, int *driver_code);
 int cross_attn_tma_smem_bytes();
 cudaError_t cross_attn_tma_prepare();   // once per device, outside any stream capture
+
+
+// ---- stand-alone cross-attention (attn_ops.cu) ---------------------------------------------
+size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_part_o,
+                                      size_t *off_part_ml);
+bool cross_attention_args_ok(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale, int splits);
+pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale,
+                                  int splits, const void *q, const void *kv, const int32_t *n_rows, const int32_t *ctx_len,
+                                  void *out, void *scratch, cudaStream_t s);
 
 }  // namespace pd
