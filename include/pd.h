@@ -220,6 +220,34 @@ PD_API pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_p
                              float attn_scale, int32_t splits, const void *q, const void *kv, const int32_t *n_rows,
                              const int32_t *ctx_len, void *out, void *scratch, size_t scratch_bytes, void *cuda_stream);
 
+/* pd_cross_attention without a scratch argument (an addition of this library; the paper has no
+ * counterpart).  Some callers have no way to obtain device memory at the moment they need the
+ * op: a plug-in that runs inside a host framework which owns the whole device heap and hands
+ * out no raw allocations; a serving loop that must not call cudaMalloc/cudaFree because those
+ * synchronise the device and stall every stream; a process started with all memory already
+ * reserved by another pool.  For them the split-K partials live in a fixed 8 MiB array inside
+ * the library image (pd_cross_attention_static_max_bytes()), which every GPU that loads the
+ * library carries until the process exits.  The caller still passes q, kv, n_rows, ctx_len and
+ * out exactly as for pd_cross_attention; results are the same.
+ *  - Sizes whose partials would not fit (pd_cross_attention_scratch_bytes(...) above the
+ *    maximum) are refused with PD_ERR_WORKSPACE and a message in pd_static_last_error(); use
+ *    fewer splits, a smaller batch, or pd_cross_attention with a buffer of your own.
+ *  - Calls no cudaMalloc, cudaFree or any other allocating routine.  The first call on a device
+ *    looks up the array's device address (cudaGetSymbolAddress, with the current device, which
+ *    must be the device of the stream and of the buffers); make that first call before any
+ *    stream capture begins.
+ *  - All calls on a device share the one array.  The call clears the header it needs at zero
+ *    and overwrites the partials it reads, so stale contents of earlier calls never matter, but
+ *    two calls that may overlap on the GPU (different streams, no dependency) race on it:
+ *    order them on one stream or with events.
+ * pd_static_last_error() returns the calling thread's message of the last failed
+ * pd_cross_attention_static (empty after a success). */
+PD_API size_t pd_cross_attention_static_max_bytes(void);
+PD_API pd_status pd_cross_attention_static(int32_t dtype, int32_t batch, int32_t rows_per_seq, int32_t n_heads,
+                                    int32_t max_ctx, float attn_scale, int32_t splits, const void *q, const void *kv,
+                                    const int32_t *n_rows, const int32_t *ctx_len, void *out, void *cuda_stream);
+PD_API const char *pd_static_last_error(void);
+
 PD_API const char *pd_last_error(const pd_handle *h);
 PD_API const char *pd_version(void);
 

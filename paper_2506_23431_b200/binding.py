@@ -68,6 +68,9 @@ _SIGS = {
     "pd_cross_attention_scratch_bytes": (C.c_size_t, [C.c_int32] * 4),
     "pd_cross_attention": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p, C.c_size_t,
                                                                                                   C.c_void_p]),
+    "pd_cross_attention_static_max_bytes": (C.c_size_t, []),
+    "pd_cross_attention_static": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p]),
+    "pd_static_last_error": (C.c_char_p, []),
     "pd_last_error": (C.c_char_p, [_H]),
     "pd_version": (C.c_char_p, []),
     "pd_destroy": (None, [_H]),
@@ -318,7 +321,8 @@ def _attention_call(fn_name: str, q, kv, n_rows, ctx_len, attn_scale: float, spl
     args.append(C.c_void_p(stream))
     st = getattr(_lib, fn_name)(*args)
     if st != PD_OK:
-        raise PdError(st, fn_name)
+        msg = (_lib.pd_static_last_error() or b"").decode() if fn_name == "pd_cross_attention_static" else ""
+        raise PdError(st, fn_name, msg)
     return out
 
 
@@ -334,6 +338,17 @@ def cross_attention(q, kv, n_rows, ctx_len, attn_scale: float, splits: int = 1, 
         n = cross_attention_scratch_bytes(q.shape[0], q.shape[1], q.shape[2] // 64, splits)
         scratch = torch.empty(max(n, 256), dtype=torch.uint8, device=q.device)
     return _attention_call("pd_cross_attention", q, kv, n_rows, ctx_len, attn_scale, splits, scratch)
+
+
+def cross_attention_static(q, kv, n_rows, ctx_len, attn_scale: float, splits: int = 1):
+    """pd_cross_attention_static: the same op with the split-K partials in the library's built-in
+    scratch array, for callers that cannot allocate device memory.  Calls sharing a device must not
+    overlap on the GPU."""
+    return _attention_call("pd_cross_attention_static", q, kv, n_rows, ctx_len, attn_scale, splits, None)
+
+
+def cross_attention_static_max_bytes() -> int:
+    return int(_lib.pd_cross_attention_static_max_bytes())
 
 
 def version() -> str:
