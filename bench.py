@@ -158,6 +158,7 @@ def main():
     ap.add_argument("--cpu-baseline-steps", type=int, default=40)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
     ap.add_argument("--single-decode", action="store_true",
                     help="run exactly one encode + decode and exit (no timing): the command profilers are pointed at")
     ap.add_argument("--time-steps", type=int, default=0,
@@ -189,6 +190,8 @@ def main():
         torch.cuda.synchronize()
 
     wl = W.CONFIGS[args.config]
+    if args.batch > 0:
+        wl = wl.scaled(batch=args.batch)
     weights = W.make_weights(wl)
     mem = W.make_encoder_memory(wl)
     ctx_len = W.make_ctx_len(wl)
