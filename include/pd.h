@@ -184,6 +184,16 @@ enum { PD_PROF_APPEND = 0, PD_PROF_SELF_ATTN = 1, PD_PROF_CROSS_ATTN = 2, PD_PRO
 PD_API pd_status pd_profile_enable(pd_handle *h, int32_t on);
 PD_API pd_status pd_profile_read(pd_handle *h, double *ms, int64_t *launches);
 
+/* Times one attention step in isolation on the decoder's current state: enqueues the
+ * self-attention (which = PD_PROF_SELF_ATTN) or cross-attention (PD_PROF_CROSS_ATTN) launches of
+ * all layers, one layer after the other, `reps` times back to back after one warm-up pass,
+ * between two CUDA events, and returns the average device time per layer launch (merge kernel
+ * included when the step is split) in microseconds.  Successive layers read different memory, so
+ * with per-layer keys/values beyond the L2 size the launches stay HBM-bound.  The decode state is
+ * not changed (the attention outputs of the last layer are rewritten with the same values).
+ * Synchronises. */
+PD_API pd_status pd_time_attention(pd_handle *h, int32_t which, int32_t reps, float *avg_us);
+
 /* Counters accumulated on the device since the last pd_encode_context, host int64 [PD_STAT_COUNT]:
  * tokens emitted (terminators included), steps executed, and the two sums the attention
  * kernels' algorithmic traffic follows from: over all (step, sequence), the number of cache

@@ -64,6 +64,7 @@ _SIGS = {
     "pd_reset_counters": (C.c_int, [_H]),
     "pd_profile_enable": (C.c_int, [_H, C.c_int32]),
     "pd_profile_read": (C.c_int, [_H, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "pd_time_attention": (C.c_int, [_H, C.c_int32, C.c_int32, C.POINTER(C.c_float)]),
     "pd_get_stats": (C.c_int, [_H, C.POINTER(C.c_int64)]),
     "pd_cross_attention_scratch_bytes": (C.c_size_t, [C.c_int32] * 4),
     "pd_cross_attention": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p, C.c_size_t,
@@ -287,6 +288,12 @@ class PipelinedDecoder:
         n = (C.c_int64 * len(PD_PROF_NAMES))()
         self._check(_lib.pd_profile_read(self._h, ms, n), "pd_profile_read")
         return {k: (ms[i], n[i]) for i, k in enumerate(PD_PROF_NAMES)}
+
+    def time_attention(self, which: str, reps: int = 5) -> float:
+        """Average device microseconds per layer launch of 'self_attn' or 'cross_attn' on the current state."""
+        us = C.c_float(0)
+        self._check(_lib.pd_time_attention(self._h, PD_PROF_NAMES.index(which), reps, C.byref(us)), "pd_time_attention")
+        return us.value
 
     def stats(self) -> Dict[str, int]:
         a = (C.c_int64 * PD_STAT_COUNT)()

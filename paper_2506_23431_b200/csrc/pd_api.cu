@@ -214,6 +214,28 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   return a;
 }
 
+// Pipelined self-attention of one layer (attention kernel + split-K merge when split).
+pd_status enqueue_self_attention(pd_handle *h, int layer) {
+  const int dt = h->cfg.dtype;
+  AttnArgs a = attn_args(h, layer, true);
+  if (dt == PD_DTYPE_BF16 && self_attn_tc_supported(h->dm)) CU_TRY(h, launch_self_attn_tc(a, h->stream));
+  else CU_TRY(h, launch_attn_core(a, dt, true, h->stream));
+  h->own_launches++;
+  if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, h->stream)); h->own_launches++; }
+  return PD_OK;
+}
+
+// Batched cross-attention of one layer.
+pd_status enqueue_cross_attention(pd_handle *h, int layer) {
+  const int dt = h->cfg.dtype;
+  AttnArgs a = attn_args(h, layer, false);
+  if (dt == PD_DTYPE_BF16 && h->have_tmap && h->dm.C <= 32) CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, h->stream));
+  else CU_TRY(h, launch_attn_core(a, dt, false, h->stream));
+  h->own_launches++;
+  if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, h->stream)); h->own_launches++; }
+  return PD_OK;
+}
+
 // The launch sequence of one decode step (one pass of Eq. 3 for all active rows + Algorithm 1's bookkeeping).
 pd_status enqueue_step(pd_handle *h) {
   const Dims &dm = h->dm;
@@ -225,8 +247,6 @@ pd_status enqueue_step(pd_handle *h) {
   float *qkv = h->ptr<float>(h->lay.qkv);
   void *ffn = h->ptr<void>(h->lay.ffn);
   float *logits = h->ptr<float>(h->lay.logits);
-  const bool tma_cross = dt == PD_DTYPE_BF16 && h->have_tmap && dm.C <= 32;
-  const bool tc_self = dt == PD_DTYPE_BF16 && self_attn_tc_supported(dm);
 
   OWN(h, PD_PROF_OTHER, launch_embed(dm, h->st, h->batch, dt, h->w.embed, x, s));
   for (int l = 0; l < dm.L; ++l) {
@@ -236,23 +256,15 @@ pd_status enqueue_step(pd_handle *h) {
     OWN(h, PD_PROF_APPEND, launch_append(dm, h->st, h->batch, l, dt, qkv, h->ptr<void>(h->lay.qbuf),
                                          h->ptr<void>(h->lay.kv_pool), h->ptr<float2>(h->lay.rope_tab), s));
     {
-      AttnArgs a = attn_args(h, l, true);
       ProfScope ps(h, PD_PROF_SELF_ATTN);
-      if (tc_self) CU_TRY(h, launch_self_attn_tc(a, s));
-      else CU_TRY(h, launch_attn_core(a, dt, true, s));
-      h->own_launches++;
-      if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, s)); h->own_launches++; }
+      PD_TRY(enqueue_self_attention(h, l));
     }
     PD_TRY(gemm(h, false, M, dm.d, dm.d, h->ptr<void>(h->lay.self_out), lw[2], x, true, 1.f));
     OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[3], hb, s));
     PD_TRY(gemm(h, false, M, dm.d, dm.d, hb, lw[4], h->ptr<void>(h->lay.cq), false, 0.f));
     {
-      AttnArgs a = attn_args(h, l, false);
       ProfScope ps(h, PD_PROF_CROSS_ATTN);
-      if (tma_cross) CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, s));
-      else CU_TRY(h, launch_attn_core(a, dt, false, s));
-      h->own_launches++;
-      if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, s)); h->own_launches++; }
+      PD_TRY(enqueue_cross_attention(h, l));
     }
     PD_TRY(gemm(h, false, M, dm.d, dm.d, h->ptr<void>(h->lay.cross_out), lw[6], x, true, 1.f));
     OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[7], hb, s));
@@ -600,6 +612,30 @@ pd_status pd_profile_read(pd_handle *h, double *ms, int64_t *launches) {
     h->ev_pool.push_back(r.a); h->ev_pool.push_back(r.b);
   }
   h->prof.clear();
+  return PD_OK;
+}
+
+pd_status pd_time_attention(pd_handle *h, int32_t which, int32_t reps, float *avg_us) {
+  if (!h || !avg_us || reps < 1 || (which != PD_PROF_SELF_ATTN && which != PD_PROF_CROSS_ATTN)) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_time_attention before pd_encode_context");
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  cudaEvent_t a = get_event(h), b = get_event(h);
+  const long long own0 = h->own_launches;
+  pd_status st = PD_OK;
+  for (int rep = -1; rep < reps && st == PD_OK; ++rep) {       // rep -1 is a warm-up pass
+    if (rep == 0) cudaEventRecord(a, h->stream);
+    for (int l = 0; l < h->dm.L && st == PD_OK; ++l)
+      st = which == PD_PROF_SELF_ATTN ? enqueue_self_attention(h, l) : enqueue_cross_attention(h, l);
+  }
+  cudaEventRecord(b, h->stream);
+  cudaError_t e = cudaStreamSynchronize(h->stream);
+  float ms = 0.f;
+  if (st == PD_OK && e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+  h->ev_pool.push_back(a); h->ev_pool.push_back(b);
+  h->own_launches = own0;
+  if (st != PD_OK) return st;
+  CU_TRY(h, e);
+  *avg_us = 1e3f * ms / (float)((long long)reps * h->dm.L);
   return PD_OK;
 }
 
