@@ -37,6 +37,8 @@ __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_
     st.state[b * dm.SM] = SUB_ACTIVE;
     st.row_sub[b * dm.C] = 1;
     st.page_table[(size_t)b * dm.SM * dm.PPS] = (int32_t)b;   // pages 0..batch-1 go to the first subsequences
+    st.plist[(size_t)b * dm.SM * dm.PPS] = make_int4((int)b, 1, 1, 1);   // step 1: bos of subsequence 1 at position 0 + 1
+    st.plist_n[b] = 1;
   }
   if (gid == 0) {
     st.hdr[HDR_STEP_T] = 1;
@@ -51,6 +53,24 @@ cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, co
                                cudaStream_t s) {
   reset_state_kernel<<<148, 256, 0, s>>>(dm, st, batch, ctx_len_dev, forced_len_dev, state_words, state_base, 0);
   reset_state_kernel<<<148, 256, 0, s>>>(dm, st, batch, ctx_len_dev, forced_len_dev, state_words, state_base, 1);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// bias_tab[h][dist] = rel_bias[h][bucket(dist)] * log2(e): the positional term of a score in the
+// log2 domain, indexed by the Manhattan distance itself.  Built once per handle.
+__global__ void build_bias_table_kernel(int H, int n_dist, int rel_buckets, const float *__restrict__ rel_bias,
+                                        const int32_t *__restrict__ dist_bucket, float *__restrict__ bias_tab) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= H * n_dist) return;
+  int h = i / n_dist, dd = i % n_dist;
+  bias_tab[i] = rel_bias[h * rel_buckets + dist_bucket[dd]] * 1.4426950408889634f;
+}
+
+cudaError_t launch_build_bias_table(const Dims &dm, const float *rel_bias, int rel_buckets, const int32_t *dist_bucket,
+                                    float *bias_tab, cudaStream_t s) {
+  int n = dm.H * dm.n_dist;
+  build_bias_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(dm.H, dm.n_dist, rel_buckets, rel_bias, dist_bucket, bias_tab);
   return cudaGetLastError();
 }
 

@@ -22,8 +22,8 @@ struct Region { size_t off = 0, bytes = 0; };
 struct Layout {
   // integer state (offsets in int32 words from the start of the state block)
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
-      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, state_words;
-  Region state, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
+      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, state_words;
+  Region state, plist, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
       ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, cublas_ws;
   size_t total = 0;
 };
@@ -69,6 +69,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   L.w_hdr = take(HDR_WORDS);
   L.w_stats = take(2 * PD_STAT_COUNT);            // 64-bit counters, 8-byte aligned (HDR_WORDS is even)
   L.w_trace = take(2 * (size_t)dm.T * B);         // 64-bit masks
+  L.w_plist_n = take(B);
   L.w_k = take(B); L.w_done = take(B); L.w_steps = take(B); L.w_nact = take(B); L.w_ctx = take(B); L.w_ticket = take(B);
   L.w_start = take(B * SM); L.w_len = take(B * SM); L.w_state = take(B * SM); L.w_flag = take(B * SM);
   L.w_last = take(B * SM); L.w_forced = take(B * SM);
@@ -83,6 +84,8 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   const size_t e = c.dtype == PD_DTYPE_BF16 ? 2 : 4;
   const size_t M = B * C;
   reg(L.state, L.state_words * 4);
+  reg(L.plist, B * SM * dm.PPS * sizeof(int4));
+  reg(L.bias_tab, (size_t)dm.H * dm.n_dist * 4);
   reg(L.ctx_len_in, B * 4);
   reg(L.forced_in, B * SM * 4);
   reg(L.teacher, B * SM * 4);
@@ -211,6 +214,7 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.dist_bucket = h->ptr<int32_t>(h->lay.dist_bucket);
   a.rel_bias = h->w.rel_bias;
   a.rel_buckets = h->cfg.rel_buckets;
+  a.bias_tab = h->cfg.pos_mode == PD_POS_T5_BIAS ? h->ptr<float>(h->lay.bias_tab) : nullptr;
   return a;
 }
 
@@ -353,6 +357,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   st.trace = reinterpret_cast<unsigned long long *>(sb + L.w_trace);
   st.k = sb + L.w_k; st.done = sb + L.w_done; st.steps = sb + L.w_steps; st.n_active = sb + L.w_nact;
   st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket;
+  st.plist_n = sb + L.w_plist_n; st.plist = h->ptr<int4>(L.plist);
   st.start = sb + L.w_start; st.len = sb + L.w_len; st.state = sb + L.w_state; st.flag = sb + L.w_flag;
   st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced;
   st.row_sub = sb + L.w_row; st.prev_row_sub = sb + L.w_prow; st.row_tok = sb + L.w_rtok;
@@ -372,6 +377,10 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
       cudaMemcpyAsync(h->ptr<void>(L.rope_tab), rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
       cudaMemsetAsync(h->ptr<void>(L.state), 0, L.state.bytes, h->stream) != cudaSuccess ||
       cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return bail(PD_ERR_CUDA);
+  if (cfg->pos_mode == PD_POS_T5_BIAS &&
+      (launch_build_bias_table(dm, weights->rel_bias, cfg->rel_buckets, h->ptr<int32_t>(L.dist_bucket), h->ptr<float>(L.bias_tab),
+                               h->stream) != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess))
     return bail(PD_ERR_CUDA);
   if (cfg->dtype == PD_DTYPE_BF16 && dm.C <= 32) {
     pd_status s = make_tensor_map(h);

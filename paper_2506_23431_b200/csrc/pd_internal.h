@@ -59,6 +59,8 @@ struct DecState {
   int32_t *hdr;                 // [HDR_WORDS]
   unsigned long long *stats;    // [PD_STAT_COUNT]
   int32_t *k, *done, *steps, *n_active, *ctx_len, *seq_ticket;        // [B]
+  int32_t *plist_n;             // [B] entries of the sequence's page list for the coming step
+  int4 *plist;                  // [B][SM*PPS] (page, entries in it, subsequence, position tau'+i' of its first entry)
   int32_t *start, *len, *state, *flag, *last_tok, *forced_len;        // [B*SM]
   int32_t *row_sub, *prev_row_sub, *row_tok;                          // [B*C]
   int32_t *page_table;          // [B*SM*PPS]
@@ -80,6 +82,7 @@ struct AttnArgs {
   const int32_t *dist_bucket;  // [n_dist]
   const float *rel_bias;       // [H, rel_buckets]
   int rel_buckets;
+  const float *bias_tab;       // [H, n_dist]: rel_bias[h][bucket(dist)] * log2(e), or null
 };
 
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
@@ -95,6 +98,8 @@ cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int lay
 cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
 cudaError_t launch_attn_merge(const AttnArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, cudaStream_t s);
+cudaError_t launch_build_bias_table(const Dims &dm, const float *rel_bias, int rel_buckets, const int32_t *dist_bucket,
+                                    float *bias_tab, cudaStream_t s);
 bool self_attn_tc_supported(const Dims &dm);
 cudaError_t self_attn_tc_prepare();     // once per device, outside any stream capture
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s);

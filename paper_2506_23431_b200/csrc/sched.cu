@@ -26,6 +26,7 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
     if (!st.done[b]) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
     for (int c = 0; c < C; ++c) st.row_sub[b * C + c] = 0;
     st.n_active[b] = 0;
+    st.plist_n[b] = 0;
     return;
   }
   // traffic counters of the step just executed (before any length changes)
@@ -103,6 +104,23 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
   }
   for (int c = n; c < C; ++c) st.row_sub[b * C + c] = 0;
   st.n_active[b] = n;
+  // Page list of the coming step for the self-attention kernels: every page of subsequences
+  // 1..i_max (i_max = last active one; later ones are invisible to every row), with the number
+  // of entries it will hold once the step's inputs are appended (bos + content = len + 1 per
+  // subsequence), its subsequence i' and the position tau' + i' of its first entry.
+  int np = 0;
+  if (n > 0) {
+    const int i_max = st.row_sub[b * C + n - 1];
+    int4 *pl = st.plist + (size_t)b * SM * dm.PPS;
+    for (int i = 1; i <= i_max; ++i) {
+      const int sidx = b * SM + i - 1;
+      const int entries = st.len[sidx] + 1;
+      const int pos0 = st.start[sidx] - 1 + i;
+      for (int j = 0; j * dm.P < entries; ++j)
+        pl[np++] = make_int4(st.page_table[(size_t)sidx * dm.PPS + j], min(dm.P, entries - j * dm.P), i, pos0 + j * dm.P);
+    }
+  }
+  st.plist_n[b] = np;
 }
 
 __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, int batch, const float *__restrict__ logits,

@@ -75,10 +75,12 @@ def test_fp32_sub_max_1_is_sequential_decoding():
     check(wl)
 
 
+@pytest.mark.parametrize("page_tokens", [16, 32])
 @pytest.mark.parametrize("pos_mode", [W.POS_T5_BIAS, W.POS_ROPE])
-def test_small_bf16_tma_cross_attention(pos_mode):
-    wl = W.CONFIGS["bart_base"].scaled(name="small_bf16", batch=3, ctx=300, sub_max=6, delta_t=2, max_sub_len=20,
-                                       length_dist=("uniform", 1, 20), time_max=48, pos_mode=pos_mode, **SMALL_BF16)
+def test_small_bf16_tensor_core_attention(pos_mode, page_tokens):
+    wl = W.CONFIGS["bart_base"].scaled(name="small_bf16", batch=3, ctx=300, sub_max=6, delta_t=2, max_sub_len=40,
+                                       length_dist=("uniform", 1, 40), time_max=60, pos_mode=pos_mode,
+                                       page_tokens=page_tokens, **SMALL_BF16)
     s = check(wl, ragged=True, cross_splits=2, self_splits=2)
     assert s["max_err"] < 2e-2
 
@@ -88,6 +90,7 @@ def test_small_bf16_many_short_subsequences_two_query_tiles():
     wl = W.CONFIGS["keyphrase"].scaled(name="small_kp", batch=2, ctx=130, sub_max=24, delta_t=1, max_sub_len=19,
                                        length_dist=("uniform", 3, 19), time_max=48, **SMALL_BF16)
     check(wl, ragged=True)
+    check(wl.scaled(page_tokens=32, pos_mode=W.POS_T5_BIAS), ragged=True, self_splits=3)
 
 
 def test_small_bf16_wide_rows_use_cuda_core_cross_attention():
