@@ -213,9 +213,10 @@ PD_API pd_status pd_get_stats(pd_handle *h, int64_t *stats);
  *   dtype        PD_DTYPE_FP32 or PD_DTYPE_BF16: element type of q, kv and out
  *   q, out       device [batch*rows_per_seq, n_heads*64]; rows at or beyond n_rows[b] of a
  *                sequence are not read and come back as zeros
- *   kv           device [batch, max_ctx, 2*n_heads*64], 16-byte aligned: per context position
- *                the keys of all heads, then the values of all heads; positions at or beyond
- *                ctx_len[b] are ignored (they may hold anything)
+ *   kv           device [batch, n_heads, 2, max_ctx, 64], 16-byte aligned: per sequence and head
+ *                the keys of all context positions, then the values (the layout the decoder keeps
+ *                its projected context in); positions at or beyond ctx_len[b] are ignored (they
+ *                may hold anything)
  *   n_rows       device int32 [batch], 0..rows_per_seq;  ctx_len  device int32 [batch], 1..max_ctx
  *   splits       1..32: split-K factor over the context (partials are merged by a second kernel)
  *   scratch      device, 256-byte aligned, at least pd_cross_attention_scratch_bytes(...): a

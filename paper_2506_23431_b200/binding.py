@@ -304,8 +304,9 @@ class PipelinedDecoder:
 
 def _attention_call(fn_name: str, q, kv, n_rows, ctx_len, attn_scale: float, splits: int, scratch):
     """Shared marshalling of the stand-alone cross-attention entry points.  q [batch, rows, heads*64],
-    kv [batch, ctx, 2*heads*64] CUDA tensors of one dtype (float32 or bfloat16); n_rows, ctx_len CUDA
-    int32 [batch].  Runs on torch's current stream; returns out (same shape as q)."""
+    kv [batch, heads, 2, ctx, 64] (keys, then values, per head) CUDA tensors of one dtype (float32 or
+    bfloat16); n_rows, ctx_len CUDA int32 [batch].  Runs on torch's current stream; returns out
+    (same shape as q)."""
     import torch
     if q.dtype not in (torch.float32, torch.bfloat16) or kv.dtype != q.dtype:
         raise ValueError("q and kv must both be float32 or both bfloat16")
@@ -314,13 +315,14 @@ def _attention_call(fn_name: str, q, kv, n_rows, ctx_len, attn_scale: float, spl
             raise ValueError("tensors must be contiguous CUDA tensors")
     batch, rows, hd = q.shape
     heads = hd // 64
-    if hd % 64 or kv.shape[0] != batch or kv.shape[2] != 2 * hd or n_rows.dtype != torch.int32 \
+    if hd % 64 or tuple(kv.shape[:3]) != (batch, heads, 2) or kv.dim() != 5 or kv.shape[4] != 64 \
+            or n_rows.dtype != torch.int32 \
             or ctx_len.dtype != torch.int32 or n_rows.numel() != batch or ctx_len.numel() != batch:
         raise ValueError("shape mismatch")
     out = torch.empty_like(q)
     dt = PD_DTYPE_BF16 if q.dtype == torch.bfloat16 else PD_DTYPE_FP32
     stream = torch.cuda.current_stream(q.device).cuda_stream
-    args = [dt, batch, rows, heads, int(kv.shape[1]), float(attn_scale), int(splits), C.c_void_p(q.data_ptr()),
+    args = [dt, batch, rows, heads, int(kv.shape[3]), float(attn_scale), int(splits), C.c_void_p(q.data_ptr()),
             C.c_void_p(kv.data_ptr()), C.c_void_p(n_rows.data_ptr()), C.c_void_p(ctx_len.data_ptr()),
             C.c_void_p(out.data_ptr())]
     if scratch is not None:

@@ -100,10 +100,9 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
     } else {
       int pos0 = tile * TK;
       n_valid = min(TK, ctx_len - pos0);
-      size_t base = (((size_t)a.layer * dm.B + b) * dm.ctx + pos0) * 2 * dm.d + h * kDh;
-      kp = (const T *)a.kv + base;
-      vp = kp + dm.d;
-      kstride = 2 * (size_t)dm.d;
+      kp = (const T *)a.kv + ctx_kv_offset(a.layer, dm.B, b, dm.H, h, 0, dm.ctx) + (size_t)pos0 * kDh;
+      vp = kp + (size_t)dm.ctx * kDh;
+      kstride = kDh;
     }
     __syncthreads();   // previous tile fully consumed
     for (int idx = tid; idx < n_valid * kDh; idx += NT) {

@@ -25,7 +25,7 @@ bool cross_attention_args_ok(int dtype, int batch, int rows_per_seq, int n_heads
   if (batch < 1 || batch > 65535 || rows_per_seq < 1 || rows_per_seq > kMaxRows) return false;
   if (n_heads < 1 || n_heads > 65535 || max_ctx < 1) return false;
   if (splits < 1 || splits > 32 || !(attn_scale > 0.f)) return false;
-  if ((unsigned long long)batch * max_ctx > 0x7fffffffull) return false;
+  if ((unsigned long long)batch * n_heads * 2 * max_ctx > 0x7fffffffull) return false;
   return true;
 }
 
@@ -55,7 +55,7 @@ pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_
   cudaError_t e;
   if (dtype == PD_DTYPE_BF16 && rows_per_seq <= 32) {
     CUtensorMap tmap;
-    if (encode_ctx_kv_tensor_map(&tmap, kv, (uint64_t)batch * max_ctx, dm.d, nullptr) != cudaSuccess) return PD_ERR_CUDA;
+    if (encode_ctx_kv_tensor_map(&tmap, kv, (uint64_t)batch * n_heads * 2 * max_ctx, nullptr) != cudaSuccess) return PD_ERR_CUDA;
     if (cross_attn_tma_prepare() != cudaSuccess) return PD_ERR_CUDA;
     e = launch_cross_attn_tma(a, tmap, s);
   } else {

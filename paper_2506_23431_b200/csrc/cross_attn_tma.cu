@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   if (warp == XCW) {
     // ------------------------------------------------------------------ producer (one lane)
     if (lane == 0) {
-      const int y0 = (a.layer * dm.B + b) * dm.ctx;
+      const int y0 = (int)(ctx_kv_offset(a.layer, dm.B, b, dm.H, h, 0, dm.ctx) / kDh);   // row of this head's key 0
       for (int it = 0; it < my; ++it) {
         int s = it % XSTAGES;
         uint32_t u = (uint32_t)(it / XSTAGES);
@@ -127,8 +127,8 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         mbar_expect_tx(bar_full + 8 * s, XSTAGE_BYTES);
         uint32_t dst = base + s * XSTAGE_BYTES;
         int y = y0 + (t0 + it) * XK;
-        tma_load_2d(dst, &tmap, bar_full + 8 * s, h * kDh, y);                       // K tile
-        tma_load_2d(dst + XTILE_BYTES, &tmap, bar_full + 8 * s, dm.d + h * kDh, y);  // V tile
+        tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, y);                         // K tile
+        tma_load_2d(dst + XTILE_BYTES, &tmap, bar_full + 8 * s, 0, y + dm.ctx);  // V tile
       }
     }
     return;
@@ -323,11 +323,11 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   }
 }
 
-// Tensor map of the projected context keys/values seen as a 2-D bf16 array [rows, 2*d] (row =
-// one context position of one sequence and layer; columns k | v, head-major): boxes of 128 rows
-// x 64 columns (one head's keys or values of one tile), 128-byte swizzle.  *driver_code gets the
-// CUresult when the encode itself fails.
-cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int d, int *driver_code) {
+// Tensor map of the context keys/values seen as a 2-D bf16 array [rows, 64] (row = one context
+// position of one (layer, sequence, head, K or V)): boxes of 128 rows x 64 columns (one head's
+// keys or values of one tile, 16 KB contiguous), 128-byte swizzle.  *driver_code gets the CUresult
+// when the encode itself fails.
+cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int *driver_code) {
   typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -337,8 +337,8 @@ cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess) return e;
   if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
-  cuuint64_t gdim[2] = {(cuuint64_t)2 * d, (cuuint64_t)rows};
-  cuuint64_t gstride[1] = {(cuuint64_t)2 * d * 2};
+  cuuint64_t gdim[2] = {(cuuint64_t)kDh, (cuuint64_t)rows};
+  cuuint64_t gstride[1] = {(cuuint64_t)kDh * 2};
   cuuint32_t box[2] = {(cuuint32_t)kDh, (cuuint32_t)XK};
   cuuint32_t estr[2] = {1u, 1u};
   CUresult r = ((EncodeFn)fn)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,

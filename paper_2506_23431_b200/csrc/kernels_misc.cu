@@ -208,4 +208,30 @@ cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int lay
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// The context projection writes [position][k of all heads | v of all heads]; the attention
+// kernels read head-major blocks.  One 16-byte chunk per thread and iteration.
+__global__ void ctx_kv_relayout_kernel(Dims dm, int batch, int layer, int esize, const uint4 *__restrict__ proj,
+                                       uint4 *__restrict__ kv_c) {
+  const int cpr = kDh * esize / 16;                        // 16-byte chunks of one head's row
+  const size_t per_pos = (size_t)2 * dm.H * cpr;           // chunks of one projected position
+  const size_t total = (size_t)batch * dm.ctx * per_pos;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % cpr);
+    const int h = (int)((i / cpr) % dm.H);
+    const int is_v = (int)((i / ((size_t)cpr * dm.H)) % 2);
+    const size_t bp = i / per_pos;
+    const int pos = (int)(bp % dm.ctx), b = (int)(bp / dm.ctx);
+    const size_t dst = (ctx_kv_offset(layer, dm.B, b, dm.H, h, is_v, dm.ctx) + (size_t)pos * kDh) * esize / 16 + c;
+    kv_c[dst] = proj[i];
+  }
+}
+
+cudaError_t launch_ctx_kv_relayout(const Dims &dm, int batch, int layer, int dtype, const void *proj, void *kv_c,
+                                   cudaStream_t s) {
+  const int esize = dtype == PD_DTYPE_BF16 ? 2 : 4;
+  ctx_kv_relayout_kernel<<<148 * 8, 256, 0, s>>>(dm, batch, layer, esize, (const uint4 *)proj, (uint4 *)kv_c);
+  return cudaGetLastError();
+}
+
 }  // namespace pd

@@ -24,7 +24,7 @@ struct Layout {
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
       w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, state_words;
   Region state, plist, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
-      ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, cublas_ws;
+      ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
 };
 
@@ -52,6 +52,7 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   long long worst = (long long)c.max_batch * c.sub_max * dm.PPS;
   dm.pool = c.pool_pages > 0 ? c.pool_pages : (int)worst;
   if (c.pool_pages < 0 || worst > 0x7fffffffLL) return false;
+  if ((long long)c.n_layers * c.max_batch * c.n_heads * 2 * c.max_ctx > 0x7fffffffLL) return false;   // rows of the context K/V tensor map
   dm.bos = c.bos_id; dm.eos = c.eos_id; dm.sep = c.sep_id;
   dm.pos_mode = c.pos_mode;
   dm.n_dist = c.time_max + c.sub_max + 2;
@@ -105,6 +106,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   reg(L.kv_c, (size_t)dm.L * B * dm.ctx * 2 * dm.d * e);
   reg(L.kv_pool, (size_t)dm.L * dm.pool * 2 * dm.H * dm.P * kDh * e);
   reg(L.enc_stage, B * dm.ctx * dm.d * e);
+  reg(L.proj_stage, B * dm.ctx * 2 * dm.d * e);
   reg(L.cublas_ws, kCublasWs);
   L.total = off;
 }
@@ -292,7 +294,7 @@ int t5_bucket(int dist, int num_buckets, int max_dist) {
 pd_status make_tensor_map(pd_handle *h) {
   const Dims &dm = h->dm;
   int code = 0;
-  cudaError_t e = encode_ctx_kv_tensor_map(&h->tmap_kvc, h->ptr<void>(h->lay.kv_c), (uint64_t)dm.L * dm.B * dm.ctx, dm.d, &code);
+  cudaError_t e = encode_ctx_kv_tensor_map(&h->tmap_kvc, h->ptr<void>(h->lay.kv_c), (uint64_t)dm.L * dm.B * dm.H * 2 * dm.ctx, &code);
   if (e != cudaSuccess) return fail(h, PD_ERR_CUDA, std::string("tensor map for the context keys/values: ") + cudaGetErrorString(e) +
                                                     " (driver code " + std::to_string(code) + ")");
   h->have_tmap = true;
@@ -436,8 +438,9 @@ pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ct
   h->own_launches++;   // the reset is two launches
   const size_t e = h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4;
   for (int l = 0; l < dm.L; ++l) {
-    uint8_t *dst = h->ptr<uint8_t>(L.kv_c) + (size_t)l * dm.B * dm.ctx * 2 * dm.d * e;
-    PD_TRY(gemm(h, false, batch * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5], dst, false, 0.f));
+    PD_TRY(gemm(h, false, batch * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5],
+                h->ptr<void>(L.proj_stage), false, 0.f));
+    OWN(h, PD_PROF_OTHER, launch_ctx_kv_relayout(dm, batch, l, h->cfg.dtype, h->ptr<void>(L.proj_stage), h->ptr<void>(L.kv_c), s));
   }
   h->encoded = true;
   h->steps_enqueued = 0;

@@ -29,6 +29,13 @@ __host__ __device__ __forceinline__ size_t kv_block_offset(int layer, int pool, 
   return ((((size_t)layer * pool + page) * H + h) * 2) * P * kDh;
 }
 
+// Context keys/values layout: [layer][sequence][head][K | V][max_ctx][64] - all keys of one head
+// of one sequence are contiguous (then its values), so a tile of consecutive positions is one
+// contiguous block.  Element offset of (layer, b, h, K or V, position 0):
+__host__ __device__ __forceinline__ size_t ctx_kv_offset(int layer, int B, int b, int H, int h, int is_v, int ctx) {
+  return (((((size_t)layer * B + b) * H + h) * 2 + is_v) * ctx) * kDh;
+}
+
 // header words of the state block
 enum { HDR_STEP_T = 0, HDR_ALL_DONE = 1, HDR_STATUS = 2, HDR_PAGE_BUMP = 3, HDR_BATCH = 4, HDR_N_DONE = 5,
        HDR_TICKET = 6, HDR_WORDS = 16 };
@@ -95,6 +102,7 @@ cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, 
 cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s);
 cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
                           void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s);
+cudaError_t launch_ctx_kv_relayout(const Dims &dm, int batch, int layer, int dtype, const void *proj, void *kv_c, cudaStream_t s);
 cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
 cudaError_t launch_attn_merge(const AttnArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, cudaStream_t s);
@@ -105,7 +113,7 @@ cudaError_t self_attn_tc_prepare();     // once per device, outside any stream c
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s);
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
                                 const int32_t *teacher, cudaStream_t s);
-cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int d, int *driver_code);
+cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int *driver_code);
 int cross_attn_tma_smem_bytes();
 cudaError_t cross_attn_tma_prepare();   // once per device, outside any stream capture
 

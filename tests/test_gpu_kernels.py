@@ -15,7 +15,7 @@ def cross_case(seed, batch, rows, heads, ctx, dtype, poison=True):
     g = np.random.Generator(np.random.Philox(key=np.array([seed, 77], dtype=np.uint64)))
     hd = heads * 64
     q = g.standard_normal((batch, rows, hd), dtype=np.float32)
-    kv = g.standard_normal((batch, ctx, 2 * hd), dtype=np.float32)
+    kv = g.standard_normal((batch, heads, 2, ctx, 64), dtype=np.float32)     # keys, then values, per head
     if dtype == "bf16":
         q, kv = W.bf16_round(q), W.bf16_round(kv)
     n_rows = g.integers(0, rows + 1, size=batch).astype(np.int32)
@@ -26,7 +26,7 @@ def cross_case(seed, batch, rows, heads, ctx, dtype, poison=True):
     ctx_len[0] = ctx
     if poison:                                         # positions beyond ctx_len must never matter
         for b in range(batch):
-            kv[b, ctx_len[b]:] = np.nan
+            kv[b, :, :, ctx_len[b]:] = np.nan
     return q, kv, n_rows, ctx_len
 
 
@@ -37,8 +37,8 @@ def oracle_cross(q, kv, n_rows, ctx_len, heads, scale):
         S, n = int(n_rows[b]), int(ctx_len[b])
         if S == 0:
             continue
-        K = kv[b, :n, :hd].astype(np.float64).reshape(n, heads, 64).transpose(1, 0, 2)
-        V = kv[b, :n, hd:].astype(np.float64).reshape(n, heads, 64).transpose(1, 0, 2)
+        K = kv[b, :, 0, :n].astype(np.float64)
+        V = kv[b, :, 1, :n].astype(np.float64)
         qq = q[b, :S].astype(np.float64).reshape(S, heads, 64)
         out[b, :S] = O.masked_attention(qq, K, V, np.ones((S, n), dtype=bool), scale, None).reshape(S, hd)
     return out
@@ -81,7 +81,7 @@ def test_cross_attention_rejects_bad_arguments():
     from paper_2506_23431_b200 import binding as B
     dev = torch.device("cuda", 0)
     q = torch.zeros(1, 4, 64, device=dev)
-    kv = torch.zeros(1, 8, 128, device=dev)
+    kv = torch.zeros(1, 1, 2, 8, 64, device=dev)
     n = torch.ones(1, dtype=torch.int32, device=dev)
     small = torch.empty(256, dtype=torch.uint8, device=dev)
     with pytest.raises(B.PdError) as e:

@@ -17,7 +17,7 @@ def _inputs(seed, batch, rows, heads, ctx, dtype):
     g = np.random.Generator(np.random.Philox(key=np.array([seed, 91], dtype=np.uint64)))
     hd = heads * 64
     q = g.standard_normal((batch, rows, hd), dtype=np.float32)
-    kv = g.standard_normal((batch, ctx, 2 * hd), dtype=np.float32)
+    kv = g.standard_normal((batch, heads, 2, ctx, 64), dtype=np.float32)
     n_rows = g.integers(1, rows + 1, size=batch).astype(np.int32)
     ctx_len = g.integers(ctx // 2, ctx + 1, size=batch).astype(np.int32)
     td = torch.bfloat16 if dtype == "bf16" else torch.float32
@@ -48,7 +48,7 @@ def test_static_scratch_variant_refuses_sizes_beyond_its_array():
     assert B.cross_attention_scratch_bytes(batch, rows, heads, splits) > limit
     dev = torch.device("cuda", 0)
     q = torch.zeros(batch, rows, heads * 64, dtype=torch.bfloat16, device=dev)
-    kv = torch.zeros(batch, 128, 2 * heads * 64, dtype=torch.bfloat16, device=dev)
+    kv = torch.zeros(batch, heads, 2, 128, 64, dtype=torch.bfloat16, device=dev)
     n = torch.ones(batch, dtype=torch.int32, device=dev)
     with pytest.raises(B.PdError) as e:
         B.cross_attention_static(q, kv, n, n, 0.125, splits)
