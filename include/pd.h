@@ -211,17 +211,21 @@ PD_API pd_status pd_get_stats(pd_handle *h, int64_t *stats);
  * subsequences; each attends, per head, to context positions 0 .. ctx_len[b]-1 with weights
  * softmax(attn_scale * q.k) and no positional term:  out = softmax(attn_scale * q K^T) V.
  *   dtype        PD_DTYPE_FP32 or PD_DTYPE_BF16: element type of q, kv and out
- *   q, out       device [batch*rows_per_seq, n_heads*64]; rows at or beyond n_rows[b] of a
+ *   q, out       device [batch*rows_per_seq, n_heads*64], 16-byte aligned; rows at or beyond n_rows[b] of a
  *                sequence are not read and come back as zeros
  *   kv           device [batch, n_heads, 2, max_ctx, 64], 16-byte aligned: per sequence and head
  *                the keys of all context positions, then the values (the layout the decoder keeps
  *                its projected context in); positions at or beyond ctx_len[b] are ignored (they
  *                may hold anything)
  *   n_rows       device int32 [batch], 0..rows_per_seq;  ctx_len  device int32 [batch], 1..max_ctx
- *   splits       1..32: split-K factor over the context (partials are merged by a second kernel)
+ *   splits       1..32: split-K factor over the context of the plain-ALU kernel (fp32, or more
+ *                than 32 rows per sequence; partials are merged by a second kernel).  The bf16
+ *                tensor-core kernel divides the context tiles of all sequences evenly over the
+ *                GPU by itself and merges its partials in the same launch.
  *   scratch      device, 256-byte aligned, at least pd_cross_attention_scratch_bytes(...): a
- *                256-byte header the call clears (int32 word 2 receives PD_ERR_TIMEOUT if a
- *                bounded wait inside the kernel expired), then the split-K partials
+ *                256-byte header (int32 word 2 receives PD_ERR_TIMEOUT if a bounded wait inside
+ *                the kernel expired) and per-(sequence, head) arrival counters, both cleared by
+ *                the call, then the partial results
  * rows_per_seq <= 64.  Enqueues on cuda_stream (a cudaStream_t) and returns; allocates nothing on
  * the device.  The caller owns every buffer and keeps it alive until the stream has passed the
  * call.  PD_ERR_ARG for null pointers or sizes out of range, PD_ERR_WORKSPACE for a scratch

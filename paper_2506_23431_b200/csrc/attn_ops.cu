@@ -8,12 +8,16 @@ using namespace pd;
 
 namespace pd {
 
-size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_part_o,
-                                      size_t *off_part_ml) {
+size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
+                                      size_t *off_part_o, size_t *off_part_ml) {
   const size_t rows = (size_t)batch * rows_per_seq;
   size_t off = kOpHeaderBytes;
+  if (off_tickets) *off_tickets = off;
+  off += ((size_t)batch * n_heads * sizeof(int32_t) + 255) / 256 * 256;      // cleared with the header
   if (off_part_o) *off_part_o = off;
-  off += (rows * n_heads * splits * kDh * sizeof(float) + 255) / 256 * 256;
+  const size_t split_bytes = rows * n_heads * splits * kDh * sizeof(float);
+  const size_t flat_bytes = cross_attn_tma_partial_bytes(kMaxCrossCtas, rows_per_seq);
+  off += ((split_bytes > flat_bytes ? split_bytes : flat_bytes) + 255) / 256 * 256;
   if (off_part_ml) *off_part_ml = off;
   off += (rows * n_heads * splits * 2 * sizeof(float) + 255) / 256 * 256;
   return off;
@@ -33,10 +37,10 @@ bool cross_attention_args_ok(int dtype, int batch, int rows_per_seq, int n_heads
 pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale,
                                   int splits, const void *q, const void *kv, const int32_t *n_rows,
                                   const int32_t *ctx_len, void *out, void *scratch, cudaStream_t s) {
-  size_t off_o = 0, off_ml = 0;
-  cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, &off_o, &off_ml);
+  size_t off_t = 0, off_o = 0, off_ml = 0;
+  cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, &off_t, &off_o, &off_ml);
   uint8_t *base = reinterpret_cast<uint8_t *>(scratch);
-  if (cudaMemsetAsync(base, 0, kOpHeaderBytes, s) != cudaSuccess) return PD_ERR_CUDA;
+  if (cudaMemsetAsync(base, 0, off_o, s) != cudaSuccess) return PD_ERR_CUDA;      // header and arrival counters
 
   AttnArgs a;
   memset(&a, 0, sizeof(a));
@@ -51,16 +55,16 @@ pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_
   a.q = q; a.kv = kv; a.out = out;
   a.part_o = reinterpret_cast<float *>(base + off_o);
   a.part_ml = reinterpret_cast<float *>(base + off_ml);
+  a.tickets = reinterpret_cast<int32_t *>(base + off_t);
 
   cudaError_t e;
-  if (dtype == PD_DTYPE_BF16 && rows_per_seq <= 32) {
+  if (dtype == PD_DTYPE_BF16 && cross_attn_tma_supported(dm, batch)) {
     CUtensorMap tmap;
     if (encode_ctx_kv_tensor_map(&tmap, kv, (uint64_t)batch * n_heads * 2 * max_ctx, nullptr) != cudaSuccess) return PD_ERR_CUDA;
     if (cross_attn_tma_prepare() != cudaSuccess) return PD_ERR_CUDA;
-    e = launch_cross_attn_tma(a, tmap, s);
-  } else {
-    e = launch_attn_core(a, dtype, false, s);
+    return launch_cross_attn_tma(a, tmap, cross_attn_ctas(), s) == cudaSuccess ? PD_OK : PD_ERR_CUDA;
   }
+  e = launch_attn_core(a, dtype, false, s);
   if (e != cudaSuccess) return PD_ERR_CUDA;
   if (splits > 1 && launch_attn_merge(a, dtype, s) != cudaSuccess) return PD_ERR_CUDA;
   return PD_OK;
@@ -72,7 +76,7 @@ extern "C" {
 
 size_t pd_cross_attention_scratch_bytes(int32_t batch, int32_t rows_per_seq, int32_t n_heads, int32_t splits) {
   if (!cross_attention_args_ok(PD_DTYPE_BF16, batch, rows_per_seq, n_heads, 1, 1.f, splits)) return 0;
-  return cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr);
+  return cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr);
 }
 
 pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_per_seq, int32_t n_heads, int32_t max_ctx,
@@ -80,8 +84,9 @@ pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_per_seq,
                              const int32_t *ctx_len, void *out, void *scratch, size_t scratch_bytes, void *cuda_stream) {
   if (!q || !kv || !n_rows || !ctx_len || !out || !scratch) return PD_ERR_ARG;
   if (!cross_attention_args_ok(dtype, batch, rows_per_seq, n_heads, max_ctx, attn_scale, splits)) return PD_ERR_ARG;
-  if (reinterpret_cast<uintptr_t>(kv) % 16 != 0 || reinterpret_cast<uintptr_t>(scratch) % 256 != 0) return PD_ERR_ARG;
-  if (scratch_bytes < cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr))
+  if (reinterpret_cast<uintptr_t>(kv) % 16 != 0 || reinterpret_cast<uintptr_t>(q) % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(out) % 16 != 0 || reinterpret_cast<uintptr_t>(scratch) % 256 != 0) return PD_ERR_ARG;
+  if (scratch_bytes < cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr))
     return PD_ERR_WORKSPACE;
   return cross_attention_enqueue(dtype, batch, rows_per_seq, n_heads, max_ctx, attn_scale, splits, q, kv, n_rows, ctx_len,
                                  out, scratch, reinterpret_cast<cudaStream_t>(cuda_stream));

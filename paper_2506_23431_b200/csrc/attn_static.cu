@@ -58,8 +58,9 @@ pd_status pd_cross_attention_static(int32_t dtype, int32_t batch, int32_t rows_p
   if (!q || !kv || !n_rows || !ctx_len || !out) return fail(PD_ERR_ARG, "null pointer argument");
   if (!cross_attention_args_ok(dtype, batch, rows_per_seq, n_heads, max_ctx, attn_scale, splits))
     return fail(PD_ERR_ARG, "a size or parameter is out of range");
-  if (reinterpret_cast<uintptr_t>(kv) % 16 != 0) return fail(PD_ERR_ARG, "kv must be 16-byte aligned");
-  const size_t need = cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr);
+  if (reinterpret_cast<uintptr_t>(kv) % 16 != 0 || reinterpret_cast<uintptr_t>(q) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0)
+    return fail(PD_ERR_ARG, "q, kv and out must be 16-byte aligned");
+  const size_t need = cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr);
   if (need > kStaticScratchBytes)
     return fail(PD_ERR_WORKSPACE, "these sizes need %lld bytes of scratch; the built-in scratch holds %lld "
                                   "(use fewer splits or pd_cross_attention with your own buffer)",

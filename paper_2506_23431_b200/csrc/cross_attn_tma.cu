@@ -3,13 +3,19 @@
 // visible, no positional term).  This is the one part of the step that is a dense S x L_ctx
 // contraction, so it runs on tensor cores; it stays HBM-bound (about S flop per byte).
 //
-// One CTA = one (split of the context, head, sequence).  A producer warp streams 128-key K and
-// V tiles (16 KB each) from global memory into a ring of shared-memory stages with TMA
-// (cp.async.bulk.tensor.2d, 128-byte swizzle, completion on an mbarrier); four consumer warps
-// each take 32 keys of every tile: S = Q K^T with mma.sync m16n8k16 (bf16 in, fp32 accumulate),
-// online softmax in the log2 domain with quad shuffles, O += P V.  The warps' partial
-// (m, l, O) are merged in shared memory, and the context splits by a separate merge kernel.
-// Every mbarrier wait is bounded: on expiry the kernel records PD_ERR_TIMEOUT and leaves.
+// Persistent kernel, two CTAs per SM.  The 128-key tiles of all (sequence with an active row,
+// head) pairs form one flat list that is cut into equal contiguous ranges, one per CTA, whatever
+// the number of active sequences: the GPU stays full when few sequences are left, and there
+// are no partial waves.  In every CTA a producer warp streams the K and V tiles of its range
+// (16 KB each, contiguous) through a ring of shared-memory stages with TMA (cp.async.bulk.tensor.2d,
+// 128-byte swizzle, completion on an mbarrier) without stopping at (sequence, head) boundaries;
+// four consumer warps each take 32 keys of every tile: S = Q K^T with mma.sync m16n8k16 (bf16 in,
+// fp32 accumulate), online softmax in the log2 domain with quad shuffles, O += P V.  At the end
+// of a (sequence, head) segment the warps' (m, l, O) are tree-merged through shared memory into
+// warp 0.  A segment that covers the whole context is written out; otherwise warp 0 stores the
+// partial record, takes a ticket, and the CTA that arrives last for that (sequence, head) merges
+// all records in CTA order (deterministic) and writes the output - no CTA ever waits for another.
+// Every mbarrier wait is bounded: on expiry the kernel records PD_ERR_TIMEOUT and drains.
 #include "pd_internal.h"
 
 namespace pd {
@@ -20,10 +26,19 @@ constexpr int XCW = 4;                    // consumer warps
 constexpr int XTHREADS = (XCW + 1) * 32;
 constexpr int XTILE_BYTES = XK * kDh * 2; // 16 KB
 constexpr int XSTAGE_BYTES = 2 * XTILE_BYTES;
-constexpr int XSMEM = XSTAGES * XSTAGE_BYTES + 128 /*barriers*/ + 1024 /*alignment slack*/;
+constexpr int XMIN_TILES = 4;              // fewest tiles worth a CTA of its own
+constexpr int XMAXB = 256;                // sequences per launch the tile prefix table holds
+constexpr int XREC_WORDS = 36;            // per lane and 16-row tile: 32 output values, 2 maxima, 2 sums
+constexpr int XREC_FLOATS = XREC_WORDS * 32;
+constexpr int XSCRATCH_BYTES = 2 * XREC_FLOATS * 4;   // two records for the warp tree merge
+constexpr int XSMEM = XSTAGES * XSTAGE_BYTES + XSCRATCH_BYTES + 128 /*barriers*/ + 1024 /*alignment slack*/;
 constexpr uint32_t XSPIN_LIMIT = 1u << 24;
 
 int cross_attn_tma_smem_bytes() { return XSMEM; }
+size_t cross_attn_tma_partial_bytes(int n_ctas, int rows_per_seq) {
+  return (size_t)n_ctas * 2 * ((rows_per_seq + 15) / 16) * XREC_FLOATS * sizeof(float);
+}
+bool cross_attn_tma_supported(const Dims &dm, int batch) { return dm.C <= 32 && batch <= XMAXB; }
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -82,53 +97,135 @@ __device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, 
 // Byte offset of (row, 16-byte chunk) inside a 128-byte-swizzled tile whose rows are 128 bytes.
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
+__device__ __forceinline__ float ex2f(float x) {   // 2^x; ex2(-inf) = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// One warp's (or one CTA's) state for a 16-row query tile in mma fragment layout: this lane holds
+// columns dn*8 + 2*tig, +1 of rows g (o[dn][0..1], m0, l0) and g + 8 (o[dn][2..3], m1, l1).
+struct TileAcc {
+  float o[8][4];
+  float m0, m1, l0, l1;
+  __device__ __forceinline__ void clear() {
+    m0 = m1 = -INFINITY; l0 = l1 = 0.f;
+#pragma unroll
+    for (int dn = 0; dn < 8; ++dn) o[dn][0] = o[dn][1] = o[dn][2] = o[dn][3] = 0.f;
+  }
+  // record layout [word][lane]: consecutive lanes touch consecutive words (coalesced, no bank conflicts)
+  __device__ __forceinline__ void store(float *rec, int lane) const {
+#pragma unroll
+    for (int dn = 0; dn < 8; ++dn)
+#pragma unroll
+      for (int x = 0; x < 4; ++x) rec[(dn * 4 + x) * 32 + lane] = o[dn][x];
+    rec[32 * 32 + lane] = m0; rec[33 * 32 + lane] = m1; rec[34 * 32 + lane] = l0; rec[35 * 32 + lane] = l1;
+  }
+  // acc <- acc (+) record, the log-sum-exp merge of two partial softmax states
+  template <bool GLOBAL>
+  __device__ __forceinline__ void merge(const float *rec, int lane) {
+    auto ld = [&](int w) { return GLOBAL ? __ldcg(rec + w * 32 + lane) : rec[w * 32 + lane]; };
+    const float om0 = ld(32), om1 = ld(33), ol0 = ld(34), ol1 = ld(35);
+    const float M0 = fmaxf(m0, om0), M1 = fmaxf(m1, om1);
+    const float r0 = M0 == -INFINITY ? 0.f : M0, r1 = M1 == -INFINITY ? 0.f : M1;
+    const float a0 = ex2f(m0 - r0), b0 = ex2f(om0 - r0), a1 = ex2f(m1 - r1), b1 = ex2f(om1 - r1);
+    m0 = M0; m1 = M1;
+    l0 = l0 * a0 + ol0 * b0; l1 = l1 * a1 + ol1 * b1;
+#pragma unroll
+    for (int dn = 0; dn < 8; ++dn) {
+      o[dn][0] = o[dn][0] * a0 + ld(dn * 4 + 0) * b0;
+      o[dn][1] = o[dn][1] * a0 + ld(dn * 4 + 1) * b0;
+      o[dn][2] = o[dn][2] * a1 + ld(dn * 4 + 2) * b1;
+      o[dn][3] = o[dn][3] * a1 + ld(dn * 4 + 3) * b1;
+    }
+  }
+};
+
+// The flat tile list: sequence-major, then head, then tile.  pfx[b] = tiles per head of the
+// active sequences before b; a sequence without an active row contributes none.
+struct TileCursor {
+  int b, h, tile, nt;   // current sequence, head, tile within the head's context, tiles per head of b
+  __device__ __forceinline__ void locate(const int *pfx, int batch, int H, int f) {
+    b = 0;
+    while (b + 1 < batch && (long long)H * pfx[b + 1] <= f) ++b;
+    nt = pfx[b + 1] - pfx[b];
+    const int rem = f - H * pfx[b];
+    h = rem / nt; tile = rem % nt;
+  }
+  __device__ __forceinline__ void next_segment(const int *pfx, int batch, int H) {
+    tile = 0;
+    if (++h == H) {
+      h = 0;
+      do { ++b; } while (b + 1 < batch && pfx[b + 1] == pfx[b]);
+      nt = b < batch ? pfx[b + 1] - pfx[b] : 1;
+    }
+  }
+};
+
 template <int MT>   // MT = 16-row query tiles (rows per sequence <= 16 * MT)
 __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap, AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
+  __shared__ int pfx_s[XMAXB + 1];
   const Dims &dm = a.dm;
-  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int S = a.st.n_active[b];
-  const int row0 = b * dm.C;
+  const int cta = blockIdx.x, G = gridDim.x, H = dm.H, batch = a.batch;
   __nv_bfloat16 *out = (__nv_bfloat16 *)a.out;
 
-  if (S == 0) {
-    if (split == 0)
-      for (int idx = tid; idx < dm.C * kDh; idx += XTHREADS)
-        out[(size_t)(row0 + idx / kDh) * dm.d + h * kDh + idx % kDh] = __float2bfloat16_rn(0.f);
-    return;
-  }
-
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_full = base + XSTAGES * XSTAGE_BYTES;
-  const uint32_t bar_empty = bar_full + 8 * XSTAGES;
   uint8_t *smem_al = smem_raw + (base - smem_u32(smem_raw));
+  float *scratch = reinterpret_cast<float *>(smem_al + XSTAGES * XSTAGE_BYTES);     // [2][XREC_FLOATS]
+  const uint32_t bar_full = base + XSTAGES * XSTAGE_BYTES + XSCRATCH_BYTES;
+  const uint32_t bar_empty = bar_full + 8 * XSTAGES;
 
-  const int ctx_len = a.st.ctx_len[b];
-  const int n_tiles = (ctx_len + XK - 1) / XK;
-  const int per = (n_tiles + a.splits - 1) / a.splits;
-  const int t0 = split * per;
-  const int my = max(0, min(n_tiles, t0 + per) - t0);
-
+  // ---- tiles per head of every sequence, prefix sums, this CTA's range of the flat list
+  for (int b = tid; b < batch; b += XTHREADS)
+    pfx_s[b + 1] = a.st.n_active[b] > 0 ? (a.st.ctx_len[b] + XK - 1) / XK : 0;
   if (tid == 0) {
+    pfx_s[0] = 0;
     for (int s = 0; s < XSTAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, XCW); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  if (warp == 0) {   // inclusive scan in chunks of 32
+    int carry = 0;
+    for (int c0 = 0; c0 < batch; c0 += 32) {
+      int v = c0 + lane < batch ? pfx_s[c0 + lane + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { int u = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += u; }
+      if (c0 + lane < batch) pfx_s[c0 + lane + 1] = v + carry;
+      carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+  }
+  // rows of a sequence beyond its active ones come back as zeros (all heads)
+  for (int b = cta; b < batch; b += G) {
+    const int S = a.st.n_active[b];
+    uint4 *z = reinterpret_cast<uint4 *>(out + (size_t)(b * dm.C + S) * dm.d);      // rows are d * 2 bytes, d a multiple of 64
+    for (int idx = tid; idx < (dm.C - S) * dm.d / 8; idx += XTHREADS) z[idx] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  __syncthreads();
+  const long long T = (long long)H * pfx_s[batch];
+  // CTAs that get work: every one of them at least XMIN_TILES tiles (when there are that many), so
+  // that few tiles do not turn into many one-tile CTAs whose records one CTA then merges serially
+  const long long want = (T + XMIN_TILES - 1) / XMIN_TILES;
+  const int Ge = (int)(want < G ? want : G);
+  if (cta >= Ge) return;
+  const int lo = (int)(cta * T / Ge), hi = (int)((cta + 1) * T / Ge);
 
   if (warp == XCW) {
     // ------------------------------------------------------------------ producer (one lane)
     if (lane == 0) {
-      const int y0 = (int)(ctx_kv_offset(a.layer, dm.B, b, dm.H, h, 0, dm.ctx) / kDh);   // row of this head's key 0
-      for (int it = 0; it < my; ++it) {
-        int s = it % XSTAGES;
-        uint32_t u = (uint32_t)(it / XSTAGES);
+      TileCursor cur;
+      cur.locate(pfx_s, batch, H, lo);
+      for (int it = 0; it < hi - lo; ++it) {
+        const int s = it % XSTAGES;
+        const uint32_t u = (uint32_t)(it / XSTAGES);
         if (!mbar_wait(bar_empty + 8 * s, (u & 1u) ^ 1u)) { atomicExch(&a.st.hdr[HDR_STATUS], (int)PD_ERR_TIMEOUT); break; }
         mbar_expect_tx(bar_full + 8 * s, XSTAGE_BYTES);
-        uint32_t dst = base + s * XSTAGE_BYTES;
-        int y = y0 + (t0 + it) * XK;
+        const uint32_t dst = base + s * XSTAGE_BYTES;
+        const int y = (int)(ctx_kv_offset(a.layer, dm.B, cur.b, H, cur.h, 0, dm.ctx) / kDh) + cur.tile * XK;
         tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, y);                         // K tile
         tma_load_2d(dst + XTILE_BYTES, &tmap, bar_full + 8 * s, 0, y + dm.ctx);  // V tile
+        if (++cur.tile == cur.nt) cur.next_segment(pfx_s, batch, H);
       }
     }
     return;
@@ -137,190 +234,200 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   // -------------------------------------------------------------------- consumers
   const int g = lane >> 2, tig = lane & 3;
   const __nv_bfloat16 *qbuf = (const __nv_bfloat16 *)a.q;
-  uint32_t qf[MT][4][4];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-    const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
-    const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      qf[mt][kk][0] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
-      qf[mt][kk][1] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
-      qf[mt][kk][2] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
-      qf[mt][kk][3] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
-    }
-  }
-  float o[MT][8][4];
-  float m_run[MT][2], l_run[MT][2];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    m_run[mt][0] = m_run[mt][1] = -INFINITY;
-    l_run[mt][0] = l_run[mt][1] = 0.f;
-#pragma unroll
-    for (int dn = 0; dn < 8; ++dn) o[mt][dn][0] = o[mt][dn][1] = o[mt][dn][2] = o[mt][dn][3] = 0.f;
-  }
   const int kb = warp * 32;          // this warp's keys inside every tile
   const float sl2 = dm.scale_log2e;
   bool ok = true;
-
-  for (int it = 0; it < my; ++it) {
-    const int s = it % XSTAGES;
-    const uint32_t u = (uint32_t)(it / XSTAGES);
-    if (!mbar_wait(bar_full + 8 * s, u & 1u)) {
-      ok = false;
-      mbar_wait(bar_full + 8 * s, u & 1u);   // one more bounded wait for the copies in flight
-      break;
-    }
-    const uint32_t kbase = base + s * XSTAGE_BYTES, vbase = kbase + XTILE_BYTES;
-    const int key0 = (t0 + it) * XK + kb;          // context position of this warp's first key
-    const bool ragged = key0 + 32 > ctx_len;
-    if (ragged) {
-      // Rows at or beyond ctx_len hold whatever follows in memory (or the fill value).  Their
-      // weights are exactly 0 below; zero the value rows so that 0 never multiplies a non-finite.
-      if (key0 + lane >= ctx_len) {
-        uint4 *vrow = reinterpret_cast<uint4 *>(smem_al + (vbase - base) + (kb + lane) * 128);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage's next bulk copy
-      }
-      __syncwarp();
-    }
-
-    // ---- scores: S[mt][nt] = Q (16 x 64) . K^T (64 x 8 keys)
-    float sc[MT][4][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-      for (int nt = 0; nt < 4; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      const int key = kb + nt * 8 + (lane & 7);
-#pragma unroll
-      for (int kp = 0; kp < 2; ++kp) {      // two k16 steps per ldmatrix.x4
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(kbase + swz(key, kp * 4 + (lane >> 3)), b0, b1, b2, b3);
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-          mma_bf16(sc[mt][nt], qf[mt][2 * kp][0], qf[mt][2 * kp][1], qf[mt][2 * kp][2], qf[mt][2 * kp][3], b0, b1);
-          mma_bf16(sc[mt][nt], qf[mt][2 * kp + 1][0], qf[mt][2 * kp + 1][1], qf[mt][2 * kp + 1][2],
-                   qf[mt][2 * kp + 1][3], b2, b3);
-        }
-      }
-    }
-    // ---- scale, mask the ragged end of the context, online softmax
-    uint32_t pf[MT][2][4];
+  int it = 0;
+  TileCursor cur;
+  cur.locate(pfx_s, batch, H, lo);
+  for (int f = lo; f < hi;) {
+    const int b = cur.b, h = cur.h;
+    const int seg_start = H * pfx_s[b] + h * cur.nt, seg_end = seg_start + cur.nt;
+    const int my_end = min(hi, seg_end);
+    const int S = a.st.n_active[b], ctx_len = a.st.ctx_len[b];
+    const int row0 = b * dm.C;
+    uint32_t qf[MT][4][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      float mx0 = -INFINITY, mx1 = -INFINITY;
+      int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+      const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
+      const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float v = sc[mt][nt][e] * sl2;
-          if (ragged && key0 + nt * 8 + 2 * tig + (e & 1) >= ctx_len) v = -INFINITY;
-          sc[mt][nt][e] = v;
-        }
-        mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
-        mx1 = fmaxf(mx1, fmaxf(sc[mt][nt][2], sc[mt][nt][3]));
+      for (int kk = 0; kk < 4; ++kk) {
+        qf[mt][kk][0] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
+        qf[mt][kk][1] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
+        qf[mt][kk][2] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
+        qf[mt][kk][3] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
       }
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      const float mn0 = fmaxf(m_run[mt][0], mx0), mn1 = fmaxf(m_run[mt][1], mx1);
-      const float ref0 = mn0 == -INFINITY ? 0.f : mn0, ref1 = mn1 == -INFINITY ? 0.f : mn1;
-      const float c0 = exp2f(m_run[mt][0] - ref0), c1 = exp2f(m_run[mt][1] - ref1);
-      m_run[mt][0] = mn0; m_run[mt][1] = mn1;
-      float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < 4; ++nt) {
-        float p0 = exp2f(sc[mt][nt][0] - ref0), p1 = exp2f(sc[mt][nt][1] - ref0);
-        float p2 = exp2f(sc[mt][nt][2] - ref1), p3 = exp2f(sc[mt][nt][3] - ref1);
-        s0 += p0 + p1; s1 += p2 + p3;
-        pf[mt][nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-        pf[mt][nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
-      }
-      l_run[mt][0] = l_run[mt][0] * c0 + s0;
-      l_run[mt][1] = l_run[mt][1] * c1 + s1;
-#pragma unroll
-      for (int dn = 0; dn < 8; ++dn) { o[mt][dn][0] *= c0; o[mt][dn][1] *= c0; o[mt][dn][2] *= c1; o[mt][dn][3] *= c1; }
     }
-    // ---- O += P (16 x 32 keys) . V (32 keys x 64)
+    TileAcc acc[MT];
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-      const int key = kb + ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+    for (int mt = 0; mt < MT; ++mt) acc[mt].clear();
+
+    for (int tile = f - seg_start; tile < my_end - seg_start; ++tile, ++it) {
+      const int s = it % XSTAGES;
+      const uint32_t u = (uint32_t)(it / XSTAGES);
+      if (ok && !mbar_wait(bar_full + 8 * s, u & 1u)) ok = false;
+      if (!ok) continue;             // drained mode: keep the control flow (barriers below) intact
+      const uint32_t kbase = base + s * XSTAGE_BYTES, vbase = kbase + XTILE_BYTES;
+      const int key0 = tile * XK + kb;               // context position of this warp's first key
+      const bool ragged = key0 + 32 > ctx_len;
+      if (ragged) {
+        // Rows at or beyond ctx_len hold whatever follows in memory.  Their weights are exactly 0
+        // below; zero the value rows so that 0 never multiplies a non-finite.
+        if (key0 + lane >= ctx_len) {
+          uint4 *vrow = reinterpret_cast<uint4 *>(smem_al + (vbase - base) + (kb + lane) * 128);
 #pragma unroll
-      for (int dp = 0; dp < 4; ++dp) {      // two 8-wide slices of the head per ldmatrix.x4
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(vbase + swz(key, dp * 2 + (lane >> 4)), b0, b1, b2, b3);
+          for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage's next bulk copy
+        }
+        __syncwarp();
+      }
+      // ---- scores: S[mt][nt] = Q (16 x 64) . K^T (64 x 8 keys)
+      float sc[MT][4][4];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const int key = kb + nt * 8 + (lane & 7);
+#pragma unroll
+        for (int kp = 0; kp < 2; ++kp) {      // two k16 steps per ldmatrix.x4
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(kbase + swz(key, kp * 4 + (lane >> 3)), b0, b1, b2, b3);
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            mma_bf16(sc[mt][nt], qf[mt][2 * kp][0], qf[mt][2 * kp][1], qf[mt][2 * kp][2], qf[mt][2 * kp][3], b0, b1);
+            mma_bf16(sc[mt][nt], qf[mt][2 * kp + 1][0], qf[mt][2 * kp + 1][1], qf[mt][2 * kp + 1][2],
+                     qf[mt][2 * kp + 1][3], b2, b3);
+          }
+        }
+      }
+      // ---- scale, mask the ragged end of the context, online softmax
+      uint32_t pf[MT][2][4];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float v = sc[mt][nt][e] * sl2;
+            if (ragged && key0 + nt * 8 + 2 * tig + (e & 1) >= ctx_len) v = -INFINITY;
+            sc[mt][nt][e] = v;
+          }
+          mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
+          mx1 = fmaxf(mx1, fmaxf(sc[mt][nt][2], sc[mt][nt][3]));
+        }
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        TileAcc &A = acc[mt];
+        const float mn0 = fmaxf(A.m0, mx0), mn1 = fmaxf(A.m1, mx1);
+        const float ref0 = mn0 == -INFINITY ? 0.f : mn0, ref1 = mn1 == -INFINITY ? 0.f : mn1;
+        const float c0 = ex2f(A.m0 - ref0), c1 = ex2f(A.m1 - ref1);
+        A.m0 = mn0; A.m1 = mn1;
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          float p0 = ex2f(sc[mt][nt][0] - ref0), p1 = ex2f(sc[mt][nt][1] - ref0);
+          float p2 = ex2f(sc[mt][nt][2] - ref1), p3 = ex2f(sc[mt][nt][3] - ref1);
+          s0 += p0 + p1; s1 += p2 + p3;
+          pf[mt][nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
+          pf[mt][nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+        }
+        A.l0 = A.l0 * c0 + s0;
+        A.l1 = A.l1 * c1 + s1;
+        if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {   // some row's running maximum moved
+#pragma unroll
+          for (int dn = 0; dn < 8; ++dn) { A.o[dn][0] *= c0; A.o[dn][1] *= c0; A.o[dn][2] *= c1; A.o[dn][3] *= c1; }
+        }
+      }
+      // ---- O += P (16 x 32 keys) . V (32 keys x 64)
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        const int key = kb + ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+        for (int dp = 0; dp < 4; ++dp) {      // two 8-wide slices of the head per ldmatrix.x4
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(vbase + swz(key, dp * 2 + (lane >> 4)), b0, b1, b2, b3);
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            mma_bf16(acc[mt].o[2 * dp], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b0, b1);
+            mma_bf16(acc[mt].o[2 * dp + 1], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b2, b3);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+    }
+
+    // ---- end of this CTA's part of the (sequence, head) segment: row sums across the quad, then
+    // tree-merge the four warps into warp 0, one 16-row tile at a time
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      TileAcc &A = acc[mt];
+      A.l0 += __shfl_xor_sync(0xffffffffu, A.l0, 1); A.l0 += __shfl_xor_sync(0xffffffffu, A.l0, 2);
+      A.l1 += __shfl_xor_sync(0xffffffffu, A.l1, 1); A.l1 += __shfl_xor_sync(0xffffffffu, A.l1, 2);
+      if (warp >= 2) A.store(scratch + (warp & 1) * XREC_FLOATS, lane);      // warps 2, 3 -> warps 0, 1
+      consumer_bar_sync();
+      if (warp < 2) A.template merge<false>(scratch + warp * XREC_FLOATS, lane);
+      consumer_bar_sync();
+      if (warp == 1) A.store(scratch, lane);                                  // warp 1 -> warp 0
+      consumer_bar_sync();
+      if (warp == 0) A.template merge<false>(scratch, lane);
+      consumer_bar_sync();
+    }
+    if (warp == 0) {
+      const bool whole = f == seg_start && my_end == seg_end;
+      bool write_out = whole;
+      if (!whole) {
+        // Partial segment: store the record, take a ticket; the last CTA to arrive merges them all.
+        const int which = lo >= seg_start ? 0 : 1;     // this CTA's first segment, or its last one
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) acc[mt].store(a.part_o + (size_t)((cta * 2 + which) * MT + mt) * XREC_FLOATS, lane);
+        __threadfence();
+        __syncwarp();
+        const int c_first = (int)((((long long)seg_start + 1) * Ge - 1) / T), c_last = (int)(((long long)seg_end * Ge - 1) / T);
+        int last = 0;
+        if (lane == 0) last = atomicAdd(&a.tickets[b * H + h], 1) == c_last - c_first;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          __threadfence();
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) acc[mt].clear();
+          for (int c2 = c_first; c2 <= c_last; ++c2) {          // fixed order: the result does not depend on arrival order
+            const int w2 = (int)(c2 * T / Ge) >= seg_start ? 0 : 1;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+              acc[mt].template merge<true>(a.part_o + (size_t)((c2 * 2 + w2) * MT + mt) * XREC_FLOATS, lane);
+          }
+          if (lane == 0) a.tickets[b * H + h] = 0;
+          write_out = true;
+        }
+      }
+      if (write_out) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          mma_bf16(o[mt][2 * dp], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b0, b1);
-          mma_bf16(o[mt][2 * dp + 1], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b2, b3);
+          const TileAcc &A = acc[mt];
+          const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+          const float i0 = 1.f / A.l0, i1 = 1.f / A.l1;
+          __nv_bfloat16 *o_lo = out + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
+          __nv_bfloat16 *o_hi = out + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
+#pragma unroll
+          for (int dn = 0; dn < 8; ++dn) {
+            if (r_lo < S) *reinterpret_cast<__nv_bfloat162 *>(o_lo + dn * 8) = __floats2bfloat162_rn(A.o[dn][0] * i0, A.o[dn][1] * i0);
+            if (r_hi < S) *reinterpret_cast<__nv_bfloat162 *>(o_hi + dn * 8) = __floats2bfloat162_rn(A.o[dn][2] * i1, A.o[dn][3] * i1);
+          }
         }
       }
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+    f = my_end;
+    if (f < hi) cur.next_segment(pfx_s, batch, H);
   }
   if (!ok && lane == 0) atomicExch(&a.st.hdr[HDR_STATUS], (int)PD_ERR_TIMEOUT);
-
-  // ---- row sums across the quad, then merge the four warps' partials through shared memory
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      l_run[mt][hh] += __shfl_xor_sync(0xffffffffu, l_run[mt][hh], 1);
-      l_run[mt][hh] += __shfl_xor_sync(0xffffffffu, l_run[mt][hh], 2);
-    }
-  consumer_bar_sync();   // every warp is past its last tile: the stages can be reused
-  constexpr int ROWS = 16 * MT;
-  float *mo = reinterpret_cast<float *>(smem_al);            // [XCW][ROWS][64]
-  float *mm = mo + XCW * ROWS * kDh;                          // [XCW][ROWS]
-  float *ml = mm + XCW * ROWS;                                // [XCW][ROWS]
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-#pragma unroll
-    for (int dn = 0; dn < 8; ++dn) {
-      int col = dn * 8 + 2 * tig;
-      *reinterpret_cast<float2 *>(&mo[(warp * ROWS + r_lo) * kDh + col]) = make_float2(o[mt][dn][0], o[mt][dn][1]);
-      *reinterpret_cast<float2 *>(&mo[(warp * ROWS + r_hi) * kDh + col]) = make_float2(o[mt][dn][2], o[mt][dn][3]);
-    }
-    if (tig == 0) {
-      mm[warp * ROWS + r_lo] = m_run[mt][0]; ml[warp * ROWS + r_lo] = l_run[mt][0];
-      mm[warp * ROWS + r_hi] = m_run[mt][1]; ml[warp * ROWS + r_hi] = l_run[mt][1];
-    }
-  }
-  consumer_bar_sync();
-  for (int idx = tid; idx < dm.C * kDh; idx += XCW * 32) {
-    int r = idx / kDh, col = idx % kDh;
-    size_t orow = (size_t)(row0 + r) * dm.d + h * kDh + col;
-    if (r >= S) {
-      if (split == 0) out[orow] = __float2bfloat16_rn(0.f);
-      continue;
-    }
-    float M = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < XCW; ++w) M = fmaxf(M, mm[w * ROWS + r]);
-    float L = 0.f, O = 0.f;
-    if (M != -INFINITY) {
-#pragma unroll
-      for (int w = 0; w < XCW; ++w) {
-        float wgt = exp2f(mm[w * ROWS + r] - M);
-        L += ml[w * ROWS + r] * wgt;
-        O += mo[(w * ROWS + r) * kDh + col] * wgt;
-      }
-    }
-    if (a.splits == 1) {
-      out[orow] = __float2bfloat16_rn(O / L);
-    } else {
-      size_t pi = ((size_t)(row0 + r) * dm.H + h) * a.splits + split;
-      a.part_o[pi * kDh + col] = O;
-      if (col == 0) { a.part_ml[pi * 2] = M; a.part_ml[pi * 2 + 1] = L; }
-    }
-  }
 }
 
 // Tensor map of the context keys/values seen as a 2-D bf16 array [rows, 64] (row = one context
@@ -348,17 +455,25 @@ cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_
   return cudaSuccess;
 }
 
+int cross_attn_ctas() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    sms = 148;
+  return 2 * sms < kMaxCrossCtas ? 2 * sms : kMaxCrossCtas;
+}
+
 cudaError_t cross_attn_tma_prepare() {
   cudaError_t e = cudaFuncSetAttribute(cross_attn_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(cross_attn_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
 }
 
-cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, cudaStream_t s) {
-  dim3 grid(a.splits, a.dm.H, a.batch);
+// n_ctas persistent CTAs (two per SM); a.part_o holds cross_attn_tma_partial_bytes(n_ctas, C),
+// a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed).
+cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, int n_ctas, cudaStream_t s) {
   int mt = (a.dm.C + 15) / 16;
-  if (mt == 1) cross_attn_tma_kernel<1><<<grid, XTHREADS, XSMEM, s>>>(tmap, a);
-  else if (mt == 2) cross_attn_tma_kernel<2><<<grid, XTHREADS, XSMEM, s>>>(tmap, a);
+  if (mt == 1) cross_attn_tma_kernel<1><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, a);
+  else if (mt == 2) cross_attn_tma_kernel<2><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, a);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }

@@ -22,7 +22,7 @@ struct Region { size_t off = 0, bytes = 0; };
 struct Layout {
   // integer state (offsets in int32 words from the start of the state block)
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
-      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, state_words;
+      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, state_words;
   Region state, plist, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
       ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
@@ -71,6 +71,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   L.w_stats = take(2 * PD_STAT_COUNT);            // 64-bit counters, 8-byte aligned (HDR_WORDS is even)
   L.w_trace = take(2 * (size_t)dm.T * B);         // 64-bit masks
   L.w_plist_n = take(B);
+  L.w_xtick = take(B * dm.H);
   L.w_k = take(B); L.w_done = take(B); L.w_steps = take(B); L.w_nact = take(B); L.w_ctx = take(B); L.w_ticket = take(B);
   L.w_start = take(B * SM); L.w_len = take(B * SM); L.w_state = take(B * SM); L.w_flag = take(B * SM);
   L.w_last = take(B * SM); L.w_forced = take(B * SM);
@@ -101,7 +102,10 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   reg(L.cross_out, M * dm.d * e);
   reg(L.ffn, M * dm.ff * e);
   reg(L.logits, M * (size_t)dm.V * 4);
-  reg(L.part_o, M * dm.H * max_splits * kDh * 4);
+  {
+    size_t split_bytes = M * dm.H * max_splits * kDh * 4, flat_bytes = cross_attn_tma_partial_bytes(kMaxCrossCtas, dm.C);
+    reg(L.part_o, split_bytes > flat_bytes ? split_bytes : flat_bytes);
+  }
   reg(L.part_ml, M * dm.H * max_splits * 2 * 4);
   reg(L.kv_c, (size_t)dm.L * B * dm.ctx * 2 * dm.d * e);
   reg(L.kv_pool, (size_t)dm.L * dm.pool * 2 * dm.H * dm.P * kDh * e);
@@ -131,6 +135,7 @@ struct pd_handle {
   int batch = 0;
   bool encoded = false;
   int self_splits = 1, cross_splits = 1;
+  int cross_ctas = 296;
   int steps_enqueued = 0;
   bool teacher_clear = false;
   // graph
@@ -216,6 +221,7 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.dist_bucket = h->ptr<int32_t>(h->lay.dist_bucket);
   a.rel_bias = h->w.rel_bias;
   a.rel_buckets = h->cfg.rel_buckets;
+  a.tickets = h->ptr<int32_t>(h->lay.state) + h->lay.w_xtick;
   a.bias_tab = h->cfg.pos_mode == PD_POS_T5_BIAS ? h->ptr<float>(h->lay.bias_tab) : nullptr;
   return a;
 }
@@ -235,8 +241,12 @@ pd_status enqueue_self_attention(pd_handle *h, int layer) {
 pd_status enqueue_cross_attention(pd_handle *h, int layer) {
   const int dt = h->cfg.dtype;
   AttnArgs a = attn_args(h, layer, false);
-  if (dt == PD_DTYPE_BF16 && h->have_tmap && h->dm.C <= 32) CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, h->stream));
-  else CU_TRY(h, launch_attn_core(a, dt, false, h->stream));
+  if (dt == PD_DTYPE_BF16 && h->have_tmap && cross_attn_tma_supported(h->dm, h->batch)) {
+    CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, h->cross_ctas, h->stream));   // merges its own partials
+    h->own_launches++;
+    return PD_OK;
+  }
+  CU_TRY(h, launch_attn_core(a, dt, false, h->stream));
   h->own_launches++;
   if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, h->stream)); h->own_launches++; }
   return PD_OK;
@@ -388,6 +398,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
     pd_status s = make_tensor_map(h);
     if (s != PD_OK) return bail(s);
     if (cross_attn_tma_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
+    h->cross_ctas = cross_attn_ctas();
   }
   if (cfg->dtype == PD_DTYPE_BF16 && self_attn_tc_supported(dm) && self_attn_tc_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
   *out = h;

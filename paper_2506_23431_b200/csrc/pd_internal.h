@@ -90,6 +90,7 @@ struct AttnArgs {
   const float *rel_bias;       // [H, rel_buckets]
   int rel_buckets;
   const float *bias_tab;       // [H, n_dist]: rel_bias[h][bucket(dist)] * log2(e), or null
+  int32_t *tickets;            // cross-attention: one arrival counter per (sequence, head), zero between launches
 };
 
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
@@ -105,7 +106,11 @@ cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int lay
 cudaError_t launch_ctx_kv_relayout(const Dims &dm, int batch, int layer, int dtype, const void *proj, void *kv_c, cudaStream_t s);
 cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
 cudaError_t launch_attn_merge(const AttnArgs &a, int dtype, cudaStream_t s);
-cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, cudaStream_t s);
+constexpr int kMaxCrossCtas = 320;      // persistent cross-attention CTAs (two per SM) the scratch is sized for
+cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, int n_ctas, cudaStream_t s);
+size_t cross_attn_tma_partial_bytes(int n_ctas, int rows_per_seq);
+bool cross_attn_tma_supported(const Dims &dm, int batch);
+int cross_attn_ctas();                  // 2 x SM count of the current device, capped at kMaxCrossCtas
 cudaError_t launch_build_bias_table(const Dims &dm, const float *rel_bias, int rel_buckets, const int32_t *dist_bucket,
                                     float *bias_tab, cudaStream_t s);
 bool self_attn_tc_supported(const Dims &dm);
@@ -119,8 +124,8 @@ cudaError_t cross_attn_tma_prepare();   // once per device, outside any stream c
 
 
 // ---- stand-alone cross-attention (attn_ops.cu) ---------------------------------------------
-size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_part_o,
-                                      size_t *off_part_ml);
+size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
+                                      size_t *off_part_o, size_t *off_part_ml);
 bool cross_attention_args_ok(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale, int splits);
 pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale,
                                   int splits, const void *q, const void *kv, const int32_t *n_rows, const int32_t *ctx_len,
