@@ -47,7 +47,7 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
                 print(" ".join(cmd), file=sys.stderr)
             subprocess.run(cmd, check=True)
     if force or _stale(LIB, objs):
-        cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-L/usr/local/cuda/lib64", "-lcublas", "-lcudart",
+        cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-L/usr/local/cuda/lib64", "-lcublas", "-lcublasLt", "-lcudart",
                "-Xlinker", "-rpath=/usr/local/cuda/lib64"]
         if verbose:
             print(" ".join(cmd), file=sys.stderr)

@@ -1,5 +1,6 @@
 // Host side of the C ABI: configuration checks, workspace carving, the per-step launch
 // sequence (own kernels + cuBLAS projections) and its CUDA-graph replay, result readers.
+#include <cublasLt.h>
 #include <cublas_v2.h>
 #include <math.h>
 #include <stdio.h>
@@ -127,6 +128,12 @@ struct pd_handle {
   uint8_t *ws = nullptr;
   cudaStream_t stream = nullptr;
   cublasHandle_t blas = nullptr;
+  cublasLtHandle_t lt = nullptr;
+  // feed-forward up-projection with the ReLU in the GEMM epilogue (plan cached per row count)
+  cublasLtMatmulDesc_t ff_desc = nullptr;
+  cublasLtMatrixLayout_t ff_w = nullptr, ff_a = nullptr, ff_c = nullptr;
+  cublasLtMatmulAlgo_t ff_algo;
+  int ff_rows = -1;          // rows the plan was made for; -2 = cuBLASLt path unavailable
   DecState st;
   std::vector<const void *> layer_w;
   pd_weights w;
@@ -200,6 +207,47 @@ pd_status gemm(pd_handle *h, bool w_is_nk, int M, int N, int K, const void *A, c
   if (s != CUBLAS_STATUS_SUCCESS) return fail(h, PD_ERR_CUDA, "cublasGemmEx failed with status " + std::to_string((int)s));
   h->gemm_calls++;
   return PD_OK;
+}
+
+void drop_ff_plan(pd_handle *h) {
+  if (h->ff_w) cublasLtMatrixLayoutDestroy(h->ff_w);
+  if (h->ff_a) cublasLtMatrixLayoutDestroy(h->ff_a);
+  if (h->ff_c) cublasLtMatrixLayoutDestroy(h->ff_c);
+  if (h->ff_desc) cublasLtMatmulDescDestroy(h->ff_desc);
+  h->ff_w = h->ff_a = h->ff_c = nullptr; h->ff_desc = nullptr;
+}
+
+// relu(A[M,K] * W[K,N]) -> C[M,N] (row-major, bf16 in and out, fp32 accumulate) in one cuBLASLt
+// call.  Returns false when no plan could be made (the caller then runs GEMM + ReLU kernel).
+bool make_ff_plan(pd_handle *h, int M, int N, int K) {
+  if (h->ff_rows == M) return true;
+  if (h->ff_rows == -2 || h->cfg.dtype != PD_DTYPE_BF16 || !h->lt) return false;
+  drop_ff_plan(h);
+  h->ff_rows = -2;
+  cublasLtEpilogue_t epi = CUBLASLT_EPILOGUE_RELU;
+  cublasOperation_t opn = CUBLAS_OP_N;
+  if (cublasLtMatmulDescCreate(&h->ff_desc, CUBLAS_COMPUTE_32F, CUDA_R_32F) != CUBLAS_STATUS_SUCCESS) return false;
+  if (cublasLtMatmulDescSetAttribute(h->ff_desc, CUBLASLT_MATMUL_DESC_TRANSA, &opn, sizeof(opn)) != CUBLAS_STATUS_SUCCESS ||
+      cublasLtMatmulDescSetAttribute(h->ff_desc, CUBLASLT_MATMUL_DESC_TRANSB, &opn, sizeof(opn)) != CUBLAS_STATUS_SUCCESS ||
+      cublasLtMatmulDescSetAttribute(h->ff_desc, CUBLASLT_MATMUL_DESC_EPILOGUE, &epi, sizeof(epi)) != CUBLAS_STATUS_SUCCESS)
+    return false;
+  // column-major view: C^T[N,M] = W^T[N,K] * A^T[K,M]
+  if (cublasLtMatrixLayoutCreate(&h->ff_w, CUDA_R_16BF, N, K, N) != CUBLAS_STATUS_SUCCESS ||
+      cublasLtMatrixLayoutCreate(&h->ff_a, CUDA_R_16BF, K, M, K) != CUBLAS_STATUS_SUCCESS ||
+      cublasLtMatrixLayoutCreate(&h->ff_c, CUDA_R_16BF, N, M, N) != CUBLAS_STATUS_SUCCESS)
+    return false;
+  cublasLtMatmulPreference_t pref = nullptr;
+  if (cublasLtMatmulPreferenceCreate(&pref) != CUBLAS_STATUS_SUCCESS) return false;
+  size_t ws = kCublasWs;
+  cublasLtMatmulPreferenceSetAttribute(pref, CUBLASLT_MATMUL_PREF_MAX_WORKSPACE_BYTES, &ws, sizeof(ws));
+  cublasLtMatmulHeuristicResult_t res;
+  int found = 0;
+  cublasStatus_t st = cublasLtMatmulAlgoGetHeuristic(h->lt, h->ff_desc, h->ff_w, h->ff_a, h->ff_c, h->ff_c, pref, 1, &res, &found);
+  cublasLtMatmulPreferenceDestroy(pref);
+  if (st != CUBLAS_STATUS_SUCCESS || found < 1) return false;
+  h->ff_algo = res.algo;
+  h->ff_rows = M;
+  return true;
 }
 
 #define OWN(h, kind, expr)                          \
@@ -284,8 +332,17 @@ pd_status enqueue_step(pd_handle *h) {
     }
     PD_TRY(gemm(h, false, M, dm.d, dm.d, h->ptr<void>(h->lay.cross_out), lw[6], x, true, 1.f));
     OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[7], hb, s));
-    PD_TRY(gemm(h, false, M, dm.ff, dm.d, hb, lw[8], ffn, false, 0.f));
-    OWN(h, PD_PROF_OTHER, launch_relu(dt, ffn, (size_t)M * dm.ff, s));
+    if (make_ff_plan(h, M, dm.ff, dm.d)) {
+      ProfScope ps(h, PD_PROF_GEMM);
+      const float one = 1.f, zero = 0.f;
+      if (cublasLtMatmul(h->lt, h->ff_desc, &one, lw[8], h->ff_w, hb, h->ff_a, &zero, ffn, h->ff_c, ffn, h->ff_c, &h->ff_algo,
+                         h->ptr<void>(h->lay.cublas_ws), kCublasWs, s) != CUBLAS_STATUS_SUCCESS)
+        return fail(h, PD_ERR_CUDA, "cublasLtMatmul (feed-forward up-projection with ReLU) failed");
+      h->gemm_calls++;
+    } else {
+      PD_TRY(gemm(h, false, M, dm.ff, dm.d, hb, lw[8], ffn, false, 0.f));
+      OWN(h, PD_PROF_OTHER, launch_relu(dt, ffn, (size_t)M * dm.ff, s));
+    }
     PD_TRY(gemm(h, false, M, dm.d, dm.ff, ffn, lw[9], x, true, 1.f));
   }
   OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, h->w.final_norm, hb, s));
@@ -358,6 +415,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   if (cudaSetDevice(cfg->device) != cudaSuccess) return bail(PD_ERR_CUDA);
   if (cublasCreate(&h->blas) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
   if (cublasSetStream(h->blas, h->stream) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
+  if (cublasLtCreate(&h->lt) != CUBLAS_STATUS_SUCCESS) h->lt = nullptr;     // optional: the ReLU then runs as its own kernel
   if (cublasSetWorkspace(h->blas, h->ptr<void>(h->lay.cublas_ws), kCublasWs) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
   if (cublasSetMathMode(h->blas, CUBLAS_DEFAULT_MATH) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
   if (cudaHostAlloc((void **)&h->pinned_flag, 64, cudaHostAllocDefault) != cudaSuccess) return bail(PD_ERR_CUDA);
@@ -425,6 +483,7 @@ pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ct
   h->teacher_clear = true;
   if (batch != h->batch) drop_graph(h);
   h->batch = batch;
+  make_ff_plan(h, batch * dm.C, dm.ff, dm.d);   // host-side planning, kept out of any stream capture
   // split-K factors
   auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
   const int bh = batch * dm.H;
@@ -679,6 +738,8 @@ void pd_destroy(pd_handle *h) {
   for (const ProfRec &r : h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->pinned_flag) cudaFreeHost(h->pinned_flag);
+  drop_ff_plan(h);
+  if (h->lt) cublasLtDestroy(h->lt);
   if (h->blas) cublasDestroy(h->blas);
   delete h;
 }

@@ -10,7 +10,7 @@
 
 namespace pd {
 
-constexpr int AT = 256;
+constexpr int AT = 512;
 
 __device__ __forceinline__ void better(float &bv, int &bi, float v, int i) {
   if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
@@ -138,11 +138,21 @@ __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, 
     const float *row = logits + (size_t)r * dm.V;
     float bv = -INFINITY;
     int bi = INT_MAX;
-    for (int v = tid; v < dm.V; v += AT) {
-      float x = __ldcs(row + v);
-      if (bar && (v == dm.eos || v == dm.sep)) continue;
+    // 16-byte streaming loads over the aligned body of the row, scalar loads for its ragged ends
+    const int head = min(dm.V, (int)((4u - (unsigned)(((size_t)r * dm.V) & 3u)) & 3u));
+    const int nvec = (dm.V - head) / 4;
+    auto take = [&](float x, int v) {
+      if (bar && (v == dm.eos || v == dm.sep)) return;
       better(bv, bi, x, v);
+    };
+    if (tid < head) take(__ldcs(row + tid), tid);
+    const float4 *body = reinterpret_cast<const float4 *>(row + head);
+    for (int q = tid; q < nvec; q += AT) {
+      const float4 x = __ldcs(body + q);
+      const int v = head + 4 * q;
+      take(x.x, v); take(x.y, v + 1); take(x.z, v + 2); take(x.w, v + 3);
     }
+    for (int v = head + 4 * nvec + tid; v < dm.V; v += AT) take(__ldcs(row + v), v);
     for (int o = 16; o > 0; o >>= 1) {
       float ov = __shfl_xor_sync(0xffffffffu, bv, o);
       int oi = __shfl_xor_sync(0xffffffffu, bi, o);
