@@ -97,6 +97,25 @@ class ClockSampler:
         return out
 
 
+def rank_workload(wl: W.Workload, rank: int) -> W.Workload:
+    """The batch a rank decodes: sequences are independent, so the path shards by batch with no
+    exchange step.  Every rank keeps the same weights (replicated) and gets its own encoder memory
+    and subsequence lengths (a different data seed), i.e. a different slice of a larger batch."""
+    return wl if rank == 0 else wl.scaled(seed=wl.seed + 7919 * rank)
+
+
+def reduce_over_ranks(times_ms, counts, dist=None, device="cpu"):
+    """Whole-job figures from per-rank ones: device times -> MAX over ranks, token counts -> SUM.
+    `dist` is torch.distributed (initialised) or None for a single process."""
+    import torch
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    c = torch.tensor(list(counts), dtype=torch.int64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], [int(x) for x in c.tolist()]
+
+
 def cpu_baseline(wl: W.Workload, weights, budget_steps: int):
     """The oracle as it stands, timed on the host cores for a bounded sample: batch row 0,
     the first `budget_steps` time-steps of its decode."""
@@ -192,10 +211,11 @@ def main():
     wl = W.CONFIGS[args.config]
     if args.batch > 0:
         wl = wl.scaled(batch=args.batch)
-    weights = W.make_weights(wl)
-    mem = W.make_encoder_memory(wl)
-    ctx_len = W.make_ctx_len(wl)
-    fl = W.make_forced_len(wl)
+    weights = W.make_weights(wl)                 # replicated on every rank
+    wl_data = rank_workload(wl, rank)            # this rank's sequences
+    mem = W.make_encoder_memory(wl_data)
+    ctx_len = W.make_ctx_len(wl_data)
+    fl = W.make_forced_len(wl_data)
     dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, device=local_rank, use_graph=not args.no_graph,
                            self_splits=args.self_splits, cross_splits=args.cross_splits)
     mem_dev = dec.device_memory(mem)
@@ -290,11 +310,8 @@ def main():
     kernel_ms = {k: round(v[0], 4) for k, v in prof.items()}
 
     # ---- max over ranks
-    t_loop = torch.tensor([loop_ms, e2e_ms, enc_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t_loop, op=dist.ReduceOp.MAX)
-    loop_ms, e2e_ms, enc_ms = [float(x) for x in t_loop.tolist()]
-    total_tokens = tokens_per_decode * args.steps * world
+    (loop_ms, e2e_ms, enc_ms), (total_tokens,) = reduce_over_ranks([loop_ms, e2e_ms, enc_ms],
+                                                                   [tokens_per_decode * args.steps], dist, "cuda")
     value = total_tokens / (loop_ms * 1e-3)
     e2e_value = total_tokens / (e2e_ms * 1e-3)
 
