@@ -37,7 +37,7 @@ __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_
     st.state[b * dm.SM] = SUB_ACTIVE;
     st.row_sub[b * dm.C] = 1;
     st.page_table[(size_t)b * dm.SM * dm.PPS] = (int32_t)b;   // pages 0..batch-1 go to the first subsequences
-    st.plist[(size_t)b * dm.SM * dm.PPS] = make_int4((int)b, 1, 1, 1);   // step 1: bos of subsequence 1 at position 0 + 1
+    st.plist[(size_t)b * dm.SM * dm.PPS] = make_int4((int)b, 1, 1, -1);  // step 1: bos of subsequence 1 at position 1, d0 = 0 - 1
     st.plist_n[b] = 1;
   }
   if (gid == 0) {

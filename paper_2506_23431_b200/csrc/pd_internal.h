@@ -67,7 +67,7 @@ struct DecState {
   unsigned long long *stats;    // [PD_STAT_COUNT]
   int32_t *k, *done, *steps, *n_active, *ctx_len, *seq_ticket;        // [B]
   int32_t *plist_n;             // [B] entries of the sequence's page list for the coming step
-  int4 *plist;                  // [B][SM*PPS] (page, entries in it, subsequence, position tau'+i' of its first entry)
+  int4 *plist;                  // [B][SM*PPS] (page, entries in it, subsequence i', distance base t - (tau' + i') of entry 0)
   int32_t *start, *len, *state, *flag, *last_tok, *forced_len;        // [B*SM]
   int32_t *row_sub, *prev_row_sub, *row_tok;                          // [B*C]
   int32_t *page_table;          // [B*SM*PPS]

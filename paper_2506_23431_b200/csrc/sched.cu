@@ -107,7 +107,9 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
   // Page list of the coming step for the self-attention kernels: every page of subsequences
   // 1..i_max (i_max = last active one; later ones are invisible to every row), with the number
   // of entries it will hold once the step's inputs are appended (bos + content = len + 1 per
-  // subsequence), its subsequence i' and the position tau' + i' of its first entry.
+  // subsequence), its subsequence i', and the Manhattan distance from a query of "subsequence 0"
+  // at that step to its first entry, d0 = t - (tau' + i') (the coming step is t + 1, whose queries sit
+  // at position t + i; a kernel adds the query's i and subtracts the key's offset in the page).
   int np = 0;
   if (n > 0) {
     const int i_max = st.row_sub[b * C + n - 1];
@@ -117,7 +119,7 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
       const int entries = st.len[sidx] + 1;
       const int pos0 = st.start[sidx] - 1 + i;
       for (int j = 0; j * dm.P < entries; ++j)
-        pl[np++] = make_int4(st.page_table[(size_t)sidx * dm.PPS + j], min(dm.P, entries - j * dm.P), i, pos0 + j * dm.P);
+        pl[np++] = make_int4(st.page_table[(size_t)sidx * dm.PPS + j], min(dm.P, entries - j * dm.P), i, t - (pos0 + j * dm.P));
     }
   }
   st.plist_n[b] = np;

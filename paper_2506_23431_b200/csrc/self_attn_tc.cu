@@ -87,18 +87,50 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
   constexpr int KS = P / 16;               // 16-key steps of P.V per page
   constexpr uint32_t SLOT = 2u * P * 128u; // keys + values of one page of one head
   extern __shared__ __align__(128) uint8_t s_ring_raw[];
-  __shared__ int4 plist_s[SMAXLIST];       // (page, entries, subsequence i', position tau'+i' of entry 0)
-  __shared__ int rsub_s[16 * MT];          // subsequence of row r (unused rows repeat the last active one)
+  __shared__ int4 plist_s[SMAXLIST];       // (page, entries, subsequence i', distance base of entry 0)
+  __shared__ int rsub_s[16 * MT];          // subsequence of row r
   __shared__ float bias_s[SMAXDIST];
 
   const Dims &dm = a.dm;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int S = a.st.n_active[b];
-  const int n_list = a.st.plist_n[b];
-  const int t = a.st.hdr[HDR_STEP_T];
   const int row0 = b * dm.C;
   __nv_bfloat16 *out = (__nv_bfloat16 *)a.out;
+  const int g = lane >> 2, tig = lane & 3;
+
+  // ---- ONE round of independent global loads, none waiting for another: active-row count, page
+  // list (first STHREADS entries), row -> subsequence, bias row of this head, query fragments.
+  // What turns out to be unused (rows beyond the active ones) is masked afterwards.
+  const int S = a.st.n_active[b];
+  const int n_list = a.st.plist_n[b];
+  const int list_cap = dm.SM * dm.PPS;
+  const int4 *pl = a.st.plist + (size_t)b * list_cap;
+  int4 my_entry = make_int4(0, 0, 0, 0);
+  if (tid < list_cap) my_entry = pl[tid];
+  int my_rsub = 0;
+  if (tid < dm.C) my_rsub = a.st.row_sub[row0 + tid];
+  const bool use_bias = a.bias_tab != nullptr;
+  float my_bias[SMAXDIST / STHREADS];
+#pragma unroll
+  for (int k = 0; k < SMAXDIST / STHREADS; ++k) {
+    const int dd = k * STHREADS + tid;
+    my_bias[k] = (use_bias && dd < dm.n_dist) ? a.bias_tab[h * dm.n_dist + dd] : 0.f;
+  }
+  const __nv_bfloat16 *qbuf = (const __nv_bfloat16 *)a.q;
+  uint32_t qf[MT][4][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+    const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
+    const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      qf[mt][kk][0] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
+      qf[mt][kk][1] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
+      qf[mt][kk][2] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
+      qf[mt][kk][3] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
+    }
+  }
 
   if (S == 0) {   // nothing active: keep the output rows of this head defined
     if (split == 0)
@@ -106,53 +138,42 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
         out[(size_t)(row0 + idx / kDh) * dm.d + h * kDh + idx % kDh] = __float2bfloat16_rn(0.f);
     return;
   }
+  if (tid < SMAXLIST) plist_s[tid] = my_entry;
+  for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
+  if (tid < 16 * MT) rsub_s[tid] = my_rsub;
+#pragma unroll
+  for (int k = 0; k < SMAXDIST / STHREADS; ++k) bias_s[k * STHREADS + tid] = my_bias[k];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {   // rows at or beyond S carry no query
+    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      if (r_lo >= S) qf[mt][kk][0] = qf[mt][kk][2] = 0u;
+      if (r_hi >= S) qf[mt][kk][1] = qf[mt][kk][3] = 0u;
+    }
+  }
+  __syncthreads();
 
-  // ---- this warp's share of the page list: entries g0, g0 + W, ...; its first two pages are
-  // requested straight from the list in global memory, before anything else
+  // ---- this warp's share of the page list: entries g0, g0 + W, ...; request its first two pages
   const int W = a.splits * SW, g0 = split * SW + warp;
   const int n_mine = n_list > g0 ? (n_list - g0 + W - 1) / W : 0;
   const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SLOT;
   const __nv_bfloat16 *pool = (const __nv_bfloat16 *)a.kv;
-  const int4 *pl = a.st.plist + (size_t)b * dm.SM * dm.PPS;
   auto fetch = [&](int n, int4 e) {
     s_fetch_page<P>(my_ring + (n & 1) * SLOT, pool + kv_block_offset(a.layer, dm.pool, e.x, dm.H, h, P), e.y, lane);
   };
-  if (n_mine > 0) fetch(0, pl[g0]);
+  if (n_mine > 0) fetch(0, plist_s[g0]);
   s_cp_async_commit();
-  if (n_mine > 1) fetch(1, pl[g0 + W]);
+  if (n_mine > 1) fetch(1, plist_s[g0 + W]);
   s_cp_async_commit();
-
-  // ---- one round of independent loads: page list, row -> subsequence, bias row of this head, queries
-  for (int i = tid; i < n_list; i += STHREADS) plist_s[i] = pl[i];
-  for (int r = tid; r < 16 * MT; r += STHREADS) rsub_s[r] = a.st.row_sub[row0 + min(r, S - 1)];
-  const bool use_bias = a.bias_tab != nullptr;
-  if (use_bias)
-    for (int dd = tid; dd < dm.n_dist; dd += STHREADS) bias_s[dd] = a.bias_tab[h * dm.n_dist + dd];
-  const int g = lane >> 2, tig = lane & 3;
-  const __nv_bfloat16 *qbuf = (const __nv_bfloat16 *)a.q;
-  uint32_t qf[MT][4][4];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-    const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
-    const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      qf[mt][kk][0] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
-      qf[mt][kk][1] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
-      qf[mt][kk][2] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
-      qf[mt][kk][3] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
-    }
-  }
-  __syncthreads();
 
   int rs[MT][2];                     // subsequence of rows g and g + 8 of every query tile
   int tile_last[MT];                 // subsequence of the tile's last active row (rows are sorted)
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) {
-    rs[mt][0] = rsub_s[mt * 16 + g];
-    rs[mt][1] = rsub_s[mt * 16 + g + 8];
-    tile_last[mt] = 16 * mt < S ? rsub_s[16 * mt + 15] : 0;
+    rs[mt][0] = rsub_s[min(mt * 16 + g, S - 1)];           // unused rows repeat the last active one
+    rs[mt][1] = rsub_s[min(mt * 16 + g + 8, S - 1)];
+    tile_last[mt] = 16 * mt < S ? rsub_s[min(16 * mt + 15, S - 1)] : 0;
   }
   const int sub_first = rsub_s[0];   // the smallest active subsequence: a page it sees, every row sees
   float o[MT][8][4];
@@ -172,7 +193,7 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
     const int4 e = plist_s[g0 + n * W];
     const int nv = e.y;                // entries of this page that exist
     const int ksub = e.z;              // subsequence the page belongs to
-    const int kpos0 = e.w;             // position tau' + i' of its first entry
+    const int d0 = e.w;                // distance base of its first entry: distance = d0 + i - key offset
     const uint32_t kbase = my_ring + (n & 1) * SLOT, vbase = kbase + P * 128u;
     // Dependency rule: a row of subsequence i sees this page iff i' <= i (every stored entry was
     // generated before the current step).  A query tile none of whose rows sees it is skipped;
@@ -215,8 +236,8 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
     for (int mt = 0; mt < MT; ++mt) {
       if (!act[mt]) continue;
       // distance of rows g / g+8 to the page's entry 0, minus this thread's first key column
-      const float *bp0 = bias_s + (t - 1 + rs[mt][0] - kpos0 - 2 * tig);
-      const float *bp1 = bias_s + (t - 1 + rs[mt][1] - kpos0 - 2 * tig);
+      const float *bp0 = bias_s + (d0 + rs[mt][0] - 2 * tig);
+      const float *bp1 = bias_s + (d0 + rs[mt][1] - 2 * tig);
       float mx0 = -INFINITY, mx1 = -INFINITY;
       if (plain) {
 #pragma unroll
