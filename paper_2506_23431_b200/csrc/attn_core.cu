@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
       if (n_valid <= 0) continue;
       int page = a.st.page_table[(size_t)sidx * dm.PPS + j];
       kp = (const T *)a.kv + kv_block_offset(a.layer, dm.pool, page, dm.H, h, dm.P);
-      vp = kp + (size_t)dm.P * kDh;
+      vp = kp;             // values interleaved with the keys, entry by entry
       kstride = kDh;
       k_sub = ksub;
       k_tau0 = a.st.start[sidx] - 1 + e0;  // timestamp of the tile's first entry
@@ -107,9 +107,8 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
     __syncthreads();   // previous tile fully consumed
     for (int idx = tid; idx < n_valid * kDh; idx += NT) {
       int e = idx / kDh, c = idx % kDh;
-      size_t off = SELF ? kv_entry_offset<T>(e, c) : e * kstride + c;
-      Ks[e][c] = ld_f<T>(kp + off);
-      Vs[e][c] = ld_f<T>(vp + off);
+      Ks[e][c] = ld_f<T>(kp + (SELF ? kv_entry_offset<T>(e, c, 0) : e * kstride + c));
+      Vs[e][c] = ld_f<T>(vp + (SELF ? kv_entry_offset<T>(e, c, 1) : e * kstride + c));
     }
     __syncthreads();
     // scores in the log2 domain

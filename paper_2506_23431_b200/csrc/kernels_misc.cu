@@ -187,8 +187,8 @@ __global__ void append_kernel(Dims dm, DecState st, int layer, const float *__re
     }
     q_out[(size_t)r * dm.d + col] = from_f<T>(q0);
     q_out[(size_t)r * dm.d + col + 1] = from_f<T>(q1);
-    size_t base = kv_block_offset(layer, dm.pool, page, dm.H, h, dm.P) + kv_entry_offset<T>(slot, dd);
-    size_t vofs = (size_t)dm.P * kDh;
+    size_t base = kv_block_offset(layer, dm.pool, page, dm.H, h, dm.P) + kv_entry_offset<T>(slot, dd, 0);
+    size_t vofs = kDh;   // the value row follows the key row of the same entry
     kv_pool[base] = from_f<T>(k0);
     kv_pool[base + 1] = from_f<T>(k1);
     kv_pool[base + vofs] = from_f<T>(v0);

@@ -15,15 +15,18 @@ constexpr int kMaxRows = 64;     // most subsequences active at once per sequenc
 constexpr int kLayerTensors = 10;
 constexpr size_t kOpHeaderBytes = 256;   // header (HDR_* words) at the start of a stand-alone op's scratch
 
-// KV pool layout: [layer][page][head][K | V][page_tokens][64].  The keys of one (page, head) are
-// page_tokens * 64 contiguous elements, followed by its values.  With 2-byte elements the eight
-// 16-byte chunks of an entry are stored swizzled (chunk c of entry e at chunk c ^ (e & 7)), so a
-// linear copy of a block into shared memory is already in the layout ldmatrix reads without
-// bank conflicts.  Offset of element (entry e, column c) inside a block's keys (or values):
+// KV pool layout: [layer][page][head][entry][K 64 | V 64].  One (page, head) block holds its
+// entries one after the other, each the key row followed by the value row, so the first n entries
+// of a block - all that exist in a partly filled page - are one contiguous run.  With 2-byte
+// elements the eight 16-byte chunks of a row are stored swizzled (chunk c of entry e at chunk
+// c ^ (e & 7)), so a linear copy of the run into shared memory is already in the layout ldmatrix
+// reads without bank conflicts.  Offset of element (entry e, column c) of the key (is_v = 0) or
+// value (is_v = 1) row inside a block:
 template <typename T>
-__host__ __device__ __forceinline__ size_t kv_entry_offset(int e, int c) {
-  if (sizeof(T) == 2) return (size_t)e * kDh + ((((c >> 3) ^ (e & 7)) << 3) | (c & 7));
-  return (size_t)e * kDh + c;
+__host__ __device__ __forceinline__ size_t kv_entry_offset(int e, int c, int is_v) {
+  const size_t row = ((size_t)e * 2 + is_v) * kDh;
+  if (sizeof(T) == 2) return row + ((((c >> 3) ^ (e & 7)) << 3) | (c & 7));
+  return row + c;
 }
 __host__ __device__ __forceinline__ size_t kv_block_offset(int layer, int pool, int page, int H, int h, int P) {
   return ((((size_t)layer * pool + page) * H + h) * 2) * P * kDh;

@@ -11,11 +11,12 @@
 // The scheduler leaves, once per step, a list of the sequence's pages (page, entries, subsequence,
 // first position) that every layer and head reuses.  One CTA = one (split, head, sequence); each of
 // its warps is an independent worker that takes every W-th page of the list (W = splits * warps),
-// copies exactly the entries that exist into its private two-slot ring with 16-byte cp.async
-// (these blocks are a few KB and scattered: per-lane async copies have no per-request engine
-// cost and need no barrier object) and keeps its own online-softmax state over all keys of the
-// page at once.  Pages are stored pre-swizzled (16-byte chunk c of entry e at chunk c ^ (e & 7)),
-// so a linear copy lands in the bank-conflict-free layout ldmatrix wants.  The warps' partials are
+// copies exactly the entries that exist - one contiguous run, key row and value row per entry -
+// into its private two-slot ring with 16-byte cp.async (these blocks are a few KB and scattered:
+// per-lane async copies have no per-request engine cost and need no barrier object) and keeps its
+// own online-softmax state over all keys of the page at once.  Pages are stored pre-swizzled
+// (16-byte chunk c of a row of entry e at chunk c ^ (e & 7)), so a linear copy lands in the
+// bank-conflict-free layout ldmatrix wants.  The warps' partials are
 // merged through shared memory, the splits by the merge kernel.  Nothing in the kernel waits on
 // another warp's progress except the two CTA barriers of prologue and epilogue.
 #include "pd_internal.h"
@@ -29,9 +30,9 @@ constexpr int SMAXLIST = 256;              // page-list entries of one sequence 
 constexpr int SMAXDIST = 512;
 
 __device__ __forceinline__ uint32_t s_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
-__device__ __forceinline__ void s_cp_async16(uint32_t dst, const void *src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+// 16-byte asynchronous copy global -> shared
+__device__ __forceinline__ void s_cp_async16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void s_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void s_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -59,26 +60,20 @@ __device__ __forceinline__ uint32_t s_pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
-// Byte offset of (entry, 16-byte chunk) inside a swizzled block whose entries are 128 bytes.
-__device__ __forceinline__ uint32_t s_swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+// Byte offset of 16-byte chunk `chunk` of entry `row`'s key row inside a block (256 bytes per
+// entry: swizzled key row, then swizzled value row at + 128).
+__device__ __forceinline__ uint32_t s_swz(int row, int chunk) { return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4)); }
 
-// All lanes: copy the nv existing entries of one (page, head) block - keys, then values - into a
-// ring slot.  Value rows from nv up to the next multiple of 16 are zero-filled: they get weights
-// of exactly 0 in P.V and must be finite whatever the slot held before.
+// All lanes: copy the nv existing entries of one (page, head) block - nv * 256 contiguous bytes,
+// key row then value row per entry - into a ring slot.
 template <int P>
 __device__ __forceinline__ void s_fetch_page(uint32_t slot, const __nv_bfloat16 *blk, int nv, int lane) {
-  const uint8_t *src = reinterpret_cast<const uint8_t *>(blk);
-  const int nchunks = nv * 8;                    // 16-byte chunks of the keys (and of the values)
-  const int vchunks = ((nv + 15) & ~15) * 8;     // value chunks including the zero-filled rows
+  const uint8_t *src = reinterpret_cast<const uint8_t *>(blk) + lane * 16;
+  const uint32_t dst = slot + lane * 16;
+  const int nchunks = nv * 16;                   // 16-byte chunks of the run
 #pragma unroll
-  for (int k = 0; k < P / 4; ++k) {              // P * 8 chunks over 32 lanes
-    const int c = k * 32 + lane;
-    if (c < nchunks) s_cp_async16(slot + c * 16, src + c * 16, 16u);
-    if (c < vchunks) {
-      const bool real = c < nchunks;
-      s_cp_async16(slot + P * 128 + c * 16, src + P * 128 + (real ? c * 16 : 0), real ? 16u : 0u);
-    }
-  }
+  for (int k = 0; k < P / 2; ++k)                // P * 16 chunks over 32 lanes
+    if (k * 32 + lane < nchunks) s_cp_async16(dst + k * 512, src + k * 512);
 }
 
 template <int MT, int P>   // MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens
@@ -138,6 +133,13 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
         out[(size_t)(row0 + idx / kDh) * dm.d + h * kDh + idx % kDh] = __float2bfloat16_rn(0.f);
     return;
   }
+  {
+    // The ring starts out zeroed: value rows beyond a partly filled page's entries get weights of
+    // exactly 0 in P.V and must be finite, whatever the slot held before (later: earlier pages' data).
+    uint4 *ring = reinterpret_cast<uint4 *>(s_ring_raw);
+#pragma unroll
+    for (int i = 0; i < (int)(SW * SDEPTH * SLOT / 16) / STHREADS; ++i) ring[i * STHREADS + tid] = make_uint4(0u, 0u, 0u, 0u);
+  }
   if (tid < SMAXLIST) plist_s[tid] = my_entry;
   for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
   if (tid < 16 * MT) rsub_s[tid] = my_rsub;
@@ -158,10 +160,9 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
   const int W = a.splits * SW, g0 = split * SW + warp;
   const int n_mine = n_list > g0 ? (n_list - g0 + W - 1) / W : 0;
   const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SLOT;
-  const __nv_bfloat16 *pool = (const __nv_bfloat16 *)a.kv;
-  auto fetch = [&](int n, int4 e) {
-    s_fetch_page<P>(my_ring + (n & 1) * SLOT, pool + kv_block_offset(a.layer, dm.pool, e.x, dm.H, h, P), e.y, lane);
-  };
+  const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
+  const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
+  auto fetch = [&](int n, int4 e) { s_fetch_page<P>(my_ring + (n & 1) * SLOT, pool_lh + e.x * page_stride, e.y, lane); };
   if (n_mine > 0) fetch(0, plist_s[g0]);
   s_cp_async_commit();
   if (n_mine > 1) fetch(1, plist_s[g0 + W]);
@@ -194,7 +195,7 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
     const int nv = e.y;                // entries of this page that exist
     const int ksub = e.z;              // subsequence the page belongs to
     const int d0 = e.w;                // distance base of its first entry: distance = d0 + i - key offset
-    const uint32_t kbase = my_ring + (n & 1) * SLOT, vbase = kbase + P * 128u;
+    const uint32_t kbase = my_ring + (n & 1) * SLOT, vbase = kbase + 128u;
     // Dependency rule: a row of subsequence i sees this page iff i' <= i (every stored entry was
     // generated before the current step).  A query tile none of whose rows sees it is skipped;
     // a full page that every row sees needs no masking at all.
