@@ -30,6 +30,13 @@ import numpy as np
 
 from paper_2506_23431_b200 import workload as W
 
+# DRAM traffic / algorithmic bytes of the two attention kernels, from the ncu capture summarised in
+# profiles/attention_kernels_summarisation_batch16.md (dram__bytes_read.sum + dram__bytes_write.sum
+# of one launch over the bytes the method must move).  Both kernels read every sequence's
+# keys/values once, so the ratio carries over to other batch sizes.  Set to None when a kernel
+# changes after its counters were taken.
+TRAFFIC_RATIO = {"cross_attn": 1.035, "self_attn": 1.03}
+
 METRIC = "decoded tokens/s per B200"
 UNIT = "tokens/s"
 DEFAULT_CONFIG = "summarisation"      # the largest configuration (most bytes per step); fits one GPU
@@ -95,6 +102,25 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
         return out
+
+
+def scheduled_tokens(forced_len, delta_t: int, sub_max: int, time_max: int) -> int:
+    """Tokens (terminators included) Algorithm 1 emits under forced lengths: subsequence i is admitted
+    at step (i-1)*delta_t + 1 while the sequence is still running, emits m_i content tokens and one
+    terminator, and the sequence stops as soon as every admitted subsequence has ended (so a
+    sequence whose early subsequences are short can stop before the later ones are admitted)."""
+    total = 0
+    for row in np.asarray(forced_len):
+        k, t, open_until = 0, 0, []
+        while t < time_max:
+            t += 1
+            if (t - 1) % delta_t == 0 and k < sub_max:
+                open_until.append(t + int(row[k]))       # emits at steps t .. t + m
+                k += 1
+            total += sum(1 for u in open_until if u >= t)
+            if all(u <= t for u in open_until):
+                break
+    return total
 
 
 def rank_workload(wl: W.Workload, rank: int) -> W.Workload:
@@ -265,7 +291,8 @@ def main():
     res = dec.collect()
     tokens_per_decode = int(st["tokens"])
     steps_per_decode = int(st["steps"])
-    assert tokens_per_decode == int((fl + 1).sum()), "decoded token count differs from the forced-length schedule"
+    assert tokens_per_decode == scheduled_tokens(fl, wl.delta_t, wl.sub_max, wl.time_max), \
+        "decoded token count differs from the forced-length schedule"
 
     # ---- end to end through pd_generate_host (host buffers, copies inside the timed region)
     e2e_ev = []
@@ -301,8 +328,9 @@ def main():
         if n == 0 or ms <= 0:
             return None
         ach = nbytes / (ms * 1e-3) / 1e9
+        ratio = TRAFFIC_RATIO.get(name) if wl.dtype == "bf16" else None
         return {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "traffic": None, "launches": int(n), "avg_launch_us": 1e3 * ms / n,
+                "traffic": None if ratio is None else ratio * nbytes / n, "launches": int(n), "avg_launch_us": 1e3 * ms / n,
                 "bytes_per_launch": nbytes / n, "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0}
 
     roofline = roof("cross_attn", cross_bytes)

@@ -149,7 +149,19 @@ __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, 
     };
     if (tid < head) take(__ldcs(row + tid), tid);
     const float4 *body = reinterpret_cast<const float4 *>(row + head);
-    for (int q = tid; q < nvec; q += AT) {
+    constexpr int UN = 4;   // loads in flight per thread
+    int q = tid;
+    for (; q + (UN - 1) * AT < nvec; q += UN * AT) {
+      float4 x[UN];
+#pragma unroll
+      for (int u = 0; u < UN; ++u) x[u] = __ldcs(body + q + u * AT);
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        const int v = head + 4 * (q + u * AT);
+        take(x[u].x, v); take(x[u].y, v + 1); take(x[u].z, v + 2); take(x[u].w, v + 3);
+      }
+    }
+    for (; q < nvec; q += AT) {
       const float4 x = __ldcs(body + q);
       const int v = head + 4 * q;
       take(x.x, v); take(x.y, v + 1); take(x.z, v + 2); take(x.w, v + 3);
