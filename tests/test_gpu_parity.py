@@ -100,6 +100,56 @@ def test_small_bf16_wide_rows_use_cuda_core_cross_attention():
     check(wl, free_run=False)
 
 
+def test_fp32_empty_subsequences_and_early_stop():
+    """Lengths from 0: a subsequence can end at its first emission (returned empty), and a sequence
+    whose admitted subsequences have all ended stops before the later ones are ever admitted."""
+    wl = TINY.scaled(batch=4, ctx=70, sub_max=6, delta_t=3, max_sub_len=5, length_dist=("uniform", 0, 5), time_max=40,
+                     vocab=300, norm_gain_std=0.1)
+    weights, mem, ctx_len, dec, rows = make(wl)
+    fl = W.make_forced_len(wl)
+    assert (fl == 0).any()
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, fl)
+    assert any(r["n_sub"] < wl.sub_max for r in runs.values()), "no early stop in this draw"
+    assert any(len(sub) == 0 for r in runs.values() for sub in r["subsequences"])
+    parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    parity.free_run_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    dec.close()
+
+
+def test_bf16_sub_max_64_one_key_context_and_unaligned_context():
+    """The largest subsequence count (a 64-bit active mask), a context of a single position, and a
+    context length that is neither a multiple of the tile nor of 16."""
+    wl = W.CONFIGS["keyphrase"].scaled(name="edge64", batch=3, ctx=131, sub_max=64, delta_t=1, max_sub_len=6,
+                                       length_dist=("uniform", 1, 6), time_max=80, pos_mode=W.POS_T5_BIAS, **SMALL_BF16)
+    weights, mem, _, dec, rows = make(wl)
+    ctx_len = np.array([1, 131, 77], dtype=np.int32)
+    fl = W.make_forced_len(wl)
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, fl)
+    assert max(r["n_sub"] for r in runs.values()) == 64
+    stats = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    assert stats["max_err"] < 2e-2
+    dec.close()
+
+
+def test_steps_after_the_end_are_no_ops():
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = TINY.scaled(vocab=300)
+    weights, mem, ctx_len, fl = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl), W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch)
+    dec.encode_context(dec.device_memory(mem), ctx_len, fl)
+    dec.run()
+    a = dec.collect()
+    st = dec.stats()
+    for _ in range(3):
+        dec.step()
+    assert dec.done()
+    b = dec.collect()
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+    assert dec.stats()["tokens"] == st["tokens"] and dec.stats()["steps"] == st["steps"]
+    dec.close()
+
+
 def test_batch_independence():
     """B sequences share a step clock and nothing else: decoding a row alone gives its streams."""
     from paper_2506_23431_b200.binding import PipelinedDecoder
