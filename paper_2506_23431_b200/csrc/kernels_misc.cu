@@ -103,34 +103,54 @@ cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtyp
 }
 
 // ---------------------------------------------------------------------------------------------
-// RMSNorm of the fp32 residual stream, output in the GEMM input type.
+// RMSNorm of the fp32 residual stream, output in the GEMM input type.  One CTA per row; a thread
+// keeps its part of the row in registers (one pass over memory) when the row fits RN_REGS values
+// per thread, else the row is read twice.
+constexpr int RN_THREADS = 256, RN_REGS = 8;
+
 template <typename T>
-__global__ void rmsnorm_kernel(int d, float eps, const float *__restrict__ x, const T *__restrict__ gain,
-                               T *__restrict__ out) {
-  __shared__ float red[32];
+__global__ void __launch_bounds__(RN_THREADS) rmsnorm_kernel(int d, float eps, const float *__restrict__ x,
+                                                             const T *__restrict__ gain, T *__restrict__ out) {
+  __shared__ float red[RN_THREADS / 32];
   const float *xr = x + (size_t)blockIdx.x * d;
+  T *orow = out + (size_t)blockIdx.x * d;
+  const bool in_regs = d <= RN_THREADS * RN_REGS;
+  float v[RN_REGS];
   float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) { float v = xr[c]; ss += v * v; }
+  if (in_regs) {
+#pragma unroll
+    for (int k = 0; k < RN_REGS; ++k) {
+      const int c = k * RN_THREADS + threadIdx.x;
+      v[k] = c < d ? xr[c] : 0.f;
+      ss += v[k] * v[k];
+    }
+  } else {
+    for (int c = threadIdx.x; c < d; c += RN_THREADS) { float t = xr[c]; ss += t * t; }
+  }
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if (threadIdx.x == 0) red[0] = v;
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < RN_THREADS / 32; ++w) tot += red[w];     // every thread sums the warps' parts in the same order
+  const float inv = rsqrtf(tot / (float)d + eps);
+  if (in_regs) {
+#pragma unroll
+    for (int k = 0; k < RN_REGS; ++k) {
+      const int c = k * RN_THREADS + threadIdx.x;
+      if (c < d) orow[c] = from_f<T>(v[k] * inv * to_f<T>(gain[c]));
+    }
+  } else {
+    for (int c = threadIdx.x; c < d; c += RN_THREADS) orow[c] = from_f<T>(xr[c] * inv * to_f<T>(gain[c]));
   }
-  __syncthreads();
-  float inv = rsqrtf(red[0] / (float)d + eps);
-  T *orow = out + (size_t)blockIdx.x * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) orow[c] = from_f<T>(xr[c] * inv * to_f<T>(gain[c]));
 }
 
 cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, const void *gain, void *out,
                            cudaStream_t s) {
   if (dtype == PD_DTYPE_BF16)
-    rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(dm.d, dm.eps, x, (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)out);
+    rmsnorm_kernel<__nv_bfloat16><<<rows, RN_THREADS, 0, s>>>(dm.d, dm.eps, x, (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)out);
   else
-    rmsnorm_kernel<float><<<rows, 256, 0, s>>>(dm.d, dm.eps, x, (const float *)gain, (float *)out);
+    rmsnorm_kernel<float><<<rows, RN_THREADS, 0, s>>>(dm.d, dm.eps, x, (const float *)gain, (float *)out);
   return cudaGetLastError();
 }
 
