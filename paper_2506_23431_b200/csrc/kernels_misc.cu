@@ -39,6 +39,8 @@ __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_
     st.page_table[(size_t)b * dm.SM * dm.PPS] = (int32_t)b;   // pages 0..batch-1 go to the first subsequences
     st.plist[(size_t)b * dm.SM * dm.PPS] = make_int4((int)b, 1, 1, -1);  // step 1: bos of subsequence 1 at position 1, d0 = 0 - 1
     st.plist_n[b] = 1;
+    st.row_meta[b * dm.C] = make_int4((int)b, 0, 1, 1);                  // bos goes to slot 0 of that page, position 0 + 1
+    for (int c = 1; c < dm.C; ++c) st.row_meta[b * dm.C + c] = make_int4(0, 0, 0, 0);
   }
   if (gid == 0) {
     st.hdr[HDR_STEP_T] = 1;
@@ -181,45 +183,36 @@ cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s) {
 template <typename T>
 __global__ void append_kernel(Dims dm, DecState st, int layer, const float *__restrict__ qkv, T *__restrict__ q_out,
                               T *__restrict__ kv_pool, const float2 *__restrict__ rope_tab) {
-  int r = blockIdx.x;
-  int b = r / dm.C;
-  int i = st.row_sub[r];
-  if (i <= 0) return;
-  int sidx = b * dm.SM + i - 1;
-  int p = st.len[sidx];
-  int tau = st.start[sidx] - 1 + p;
-  int pos = tau + i;
-  int page = st.page_table[(size_t)sidx * dm.PPS + p / dm.P];
-  int slot = p % dm.P;
+  const int r = blockIdx.x;
   const float *row = qkv + (size_t)r * 3 * dm.d;
-  for (int j = threadIdx.x; j < dm.d / 2; j += blockDim.x) {
-    int col = 2 * j;
-    int h = col / kDh, dd = col % kDh;
-    float q0 = row[col], q1 = row[col + 1];
-    float k0 = row[dm.d + col], k1 = row[dm.d + col + 1];
-    float v0 = row[2 * dm.d + col], v1 = row[2 * dm.d + col + 1];
-    if (dm.pos_mode == PD_POS_ROPE) {
-      float2 cs = rope_tab[(size_t)pos * (kDh / 2) + dd / 2];
-      float a = q0 * cs.x - q1 * cs.y, c2 = q0 * cs.y + q1 * cs.x;
-      q0 = a; q1 = c2;
-      a = k0 * cs.x - k1 * cs.y; c2 = k0 * cs.y + k1 * cs.x;
-      k0 = a; k1 = c2;
-    }
-    q_out[(size_t)r * dm.d + col] = from_f<T>(q0);
-    q_out[(size_t)r * dm.d + col + 1] = from_f<T>(q1);
-    size_t base = kv_block_offset(layer, dm.pool, page, dm.H, h, dm.P) + kv_entry_offset<T>(slot, dd, 0);
-    size_t vofs = kDh;   // the value row follows the key row of the same entry
-    kv_pool[base] = from_f<T>(k0);
-    kv_pool[base + 1] = from_f<T>(k1);
-    kv_pool[base + vofs] = from_f<T>(v0);
-    kv_pool[base + vofs + 1] = from_f<T>(v1);
+  // one round of independent loads: where the row goes, and this thread's four columns of q, k, v
+  const int4 meta = st.row_meta[r];                 // (page, slot, position tau + i, subsequence i or 0)
+  const int col = 4 * threadIdx.x;                  // blockDim.x = d / 4; four columns never straddle a 16-byte chunk or a head
+  float4 q = *reinterpret_cast<const float4 *>(row + col);
+  float4 k = *reinterpret_cast<const float4 *>(row + dm.d + col);
+  const float4 v = *reinterpret_cast<const float4 *>(row + 2 * dm.d + col);
+  if (meta.w <= 0) return;
+  const int h = col / kDh, dd = col % kDh;
+  if (dm.pos_mode == PD_POS_ROPE) {
+    const float2 c0 = rope_tab[(size_t)meta.z * (kDh / 2) + dd / 2], c1 = rope_tab[(size_t)meta.z * (kDh / 2) + dd / 2 + 1];
+    float a;
+    a = q.x * c0.x - q.y * c0.y; q.y = q.x * c0.y + q.y * c0.x; q.x = a;
+    a = q.z * c1.x - q.w * c1.y; q.w = q.z * c1.y + q.w * c1.x; q.z = a;
+    a = k.x * c0.x - k.y * c0.y; k.y = k.x * c0.y + k.y * c0.x; k.x = a;
+    a = k.z * c1.x - k.w * c1.y; k.w = k.z * c1.y + k.w * c1.x; k.z = a;
   }
+  T *qo = q_out + (size_t)r * dm.d + col;
+  T *ko = kv_pool + kv_block_offset(layer, dm.pool, meta.x, dm.H, h, dm.P) + kv_entry_offset<T>(meta.y, dd, 0);
+  T *vo = ko + kDh;                                 // the value row follows the key row of the same entry
+  qo[0] = from_f<T>(q.x); qo[1] = from_f<T>(q.y); qo[2] = from_f<T>(q.z); qo[3] = from_f<T>(q.w);
+  ko[0] = from_f<T>(k.x); ko[1] = from_f<T>(k.y); ko[2] = from_f<T>(k.z); ko[3] = from_f<T>(k.w);
+  vo[0] = from_f<T>(v.x); vo[1] = from_f<T>(v.y); vo[2] = from_f<T>(v.z); vo[3] = from_f<T>(v.w);
 }
 
 cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
                           void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s) {
   int rows = batch * dm.C;
-  int threads = dm.d / 2 < 256 ? dm.d / 2 : 256;
+  int threads = dm.d / 4;                           // d is a multiple of 64 and at most 4096 (checked at init)
   if (dtype == PD_DTYPE_BF16)
     append_kernel<__nv_bfloat16><<<rows, threads, 0, s>>>(dm, st, layer, qkv, (__nv_bfloat16 *)q_out,
                                                          (__nv_bfloat16 *)kv_pool, rope_tab);

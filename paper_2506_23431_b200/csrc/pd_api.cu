@@ -24,7 +24,7 @@ struct Layout {
   // integer state (offsets in int32 words from the start of the state block)
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
       w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, state_words;
-  Region state, plist, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
+  Region state, plist, row_meta, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
       ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
 };
@@ -32,7 +32,7 @@ struct Layout {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
-  if (c.n_layers < 1 || c.d_model < 64 || c.n_heads < 1 || c.d_head != kDh || c.n_heads * c.d_head != c.d_model) return false;
+  if (c.n_layers < 1 || c.d_model < 64 || c.d_model > 4096 || c.n_heads < 1 || c.d_head != kDh || c.n_heads * c.d_head != c.d_model) return false;
   if (c.d_ff < 8 || c.vocab < 4 || (c.d_model % 8) || (c.d_ff % 8)) return false;
   if (c.dtype != PD_DTYPE_FP32 && c.dtype != PD_DTYPE_BF16) return false;
   if (c.max_batch < 1 || c.max_ctx < 1 || c.sub_max < 1 || c.sub_max > 64 || c.delta_t < 1 || c.time_max < 1) return false;
@@ -88,6 +88,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   const size_t M = B * C;
   reg(L.state, L.state_words * 4);
   reg(L.plist, B * SM * dm.PPS * sizeof(int4));
+  reg(L.row_meta, B * C * sizeof(int4));
   reg(L.bias_tab, (size_t)dm.H * dm.n_dist * 4);
   reg(L.ctx_len_in, B * 4);
   reg(L.forced_in, B * SM * 4);
@@ -427,7 +428,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   st.trace = reinterpret_cast<unsigned long long *>(sb + L.w_trace);
   st.k = sb + L.w_k; st.done = sb + L.w_done; st.steps = sb + L.w_steps; st.n_active = sb + L.w_nact;
   st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket;
-  st.plist_n = sb + L.w_plist_n; st.plist = h->ptr<int4>(L.plist);
+  st.plist_n = sb + L.w_plist_n; st.plist = h->ptr<int4>(L.plist); st.row_meta = h->ptr<int4>(L.row_meta);
   st.start = sb + L.w_start; st.len = sb + L.w_len; st.state = sb + L.w_state; st.flag = sb + L.w_flag;
   st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced;
   st.row_sub = sb + L.w_row; st.prev_row_sub = sb + L.w_prow; st.row_tok = sb + L.w_rtok;

@@ -70,6 +70,7 @@ struct DecState {
   unsigned long long *stats;    // [PD_STAT_COUNT]
   int32_t *k, *done, *steps, *n_active, *ctx_len, *seq_ticket;        // [B]
   int32_t *plist_n;             // [B] entries of the sequence's page list for the coming step
+  int4 *row_meta;               // [B*C] per row: (page, slot in it, position tau + i) of the entry the coming step appends, subsequence i (0 = unused row)
   int4 *plist;                  // [B][SM*PPS] (page, entries in it, subsequence i', distance base t - (tau' + i') of entry 0)
   int32_t *start, *len, *state, *flag, *last_tok, *forced_len;        // [B*SM]
   int32_t *row_sub, *prev_row_sub, *row_tok;                          // [B*C]

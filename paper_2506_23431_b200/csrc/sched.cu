@@ -24,7 +24,7 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
   for (int c = 0; c < C; ++c) st.prev_row_sub[b * C + c] = st.row_sub[b * C + c];
   if (st.done[b] || st.hdr[HDR_STATUS] != 0) {
     if (!st.done[b]) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
-    for (int c = 0; c < C; ++c) st.row_sub[b * C + c] = 0;
+    for (int c = 0; c < C; ++c) { st.row_sub[b * C + c] = 0; st.row_meta[b * C + c] = make_int4(0, 0, 0, 0); }
     st.n_active[b] = 0;
     st.plist_n[b] = 0;
     return;
@@ -92,7 +92,6 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
       const int sidx = b * SM + i - 1;
       if (st.state[sidx] != SUB_ACTIVE) continue;
       if (n >= C) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_STATE); break; }
-      st.row_sub[b * C + n++] = i;
       const int p = st.len[sidx];                  // entry the next step will write
       if (p % dm.P == 0) {
         int pg = atomicAdd(&st.hdr[HDR_PAGE_BUMP], 1);
@@ -100,9 +99,12 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
         st.page_table[(size_t)sidx * dm.PPS + p / dm.P] = pg;
         atomicAdd(&st.stats[PD_STAT_PAGES], 1ull);
       }
+      // where the append kernels of the coming step put this row's key/value, and its position tau + i
+      st.row_meta[b * C + n] = make_int4(st.page_table[(size_t)sidx * dm.PPS + p / dm.P], p % dm.P, st.start[sidx] - 1 + p + i, i);
+      st.row_sub[b * C + n++] = i;
     }
   }
-  for (int c = n; c < C; ++c) st.row_sub[b * C + c] = 0;
+  for (int c = n; c < C; ++c) { st.row_sub[b * C + c] = 0; st.row_meta[b * C + c] = make_int4(0, 0, 0, 0); }
   st.n_active[b] = n;
   // Page list of the coming step for the self-attention kernels: every page of subsequences
   // 1..i_max (i_max = last active one; later ones are invisible to every row), with the number
