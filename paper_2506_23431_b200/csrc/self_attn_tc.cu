@@ -28,6 +28,7 @@ constexpr int STHREADS = SW * 32;
 constexpr int SDEPTH = 2;                  // ring slots per warp: the page in use and the next one
 constexpr int SMAXLIST = 256;              // page-list entries of one sequence held in shared memory
 constexpr int SMAXDIST = 512;
+constexpr int SMROW = kDh + 8;               // row stride of the merge scratch in floats (spreads the eight fragment rows over the banks)
 
 __device__ __forceinline__ uint32_t s_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 // 16-byte asynchronous copy global -> shared
@@ -328,8 +329,8 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
     }
   __syncthreads();   // every warp is past its last page: the ring can be reused
   constexpr int ROWS = 16 * MT;
-  float *mo = reinterpret_cast<float *>(s_ring_raw);          // [SW][ROWS][64]
-  float *mm = mo + SW * ROWS * kDh;                           // [SW][ROWS]
+  float *mo = reinterpret_cast<float *>(s_ring_raw);          // [SW][ROWS][SMROW]
+  float *mm = mo + SW * ROWS * SMROW;                           // [SW][ROWS]
   float *ml = mm + SW * ROWS;                                 // [SW][ROWS]
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) {
@@ -337,8 +338,8 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
 #pragma unroll
     for (int dn = 0; dn < 8; ++dn) {
       int col = dn * 8 + 2 * tig;
-      *reinterpret_cast<float2 *>(&mo[(warp * ROWS + r_lo) * kDh + col]) = make_float2(o[mt][dn][0], o[mt][dn][1]);
-      *reinterpret_cast<float2 *>(&mo[(warp * ROWS + r_hi) * kDh + col]) = make_float2(o[mt][dn][2], o[mt][dn][3]);
+      *reinterpret_cast<float2 *>(&mo[(warp * ROWS + r_lo) * SMROW + col]) = make_float2(o[mt][dn][0], o[mt][dn][1]);
+      *reinterpret_cast<float2 *>(&mo[(warp * ROWS + r_hi) * SMROW + col]) = make_float2(o[mt][dn][2], o[mt][dn][3]);
     }
     if (tig == 0) {
       mm[warp * ROWS + r_lo] = m_run[mt][0]; ml[warp * ROWS + r_lo] = l_run[mt][0];
@@ -346,38 +347,51 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
     }
   }
   __syncthreads();
-  for (int idx = tid; idx < dm.C * kDh; idx += STHREADS) {
-    int r = idx / kDh, col = idx % kDh;
-    size_t orow = (size_t)(row0 + r) * dm.d + h * kDh + col;
-    if (r >= S) {
-      if (split == 0) out[orow] = __float2bfloat16_rn(0.f);
-      continue;
-    }
+  // per row once: the common maximum, each warp's weight (turned into mm in place) and the row sum
+  if (tid < ROWS && tid < S) {
+    const int r = tid;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < SW; ++w) M = fmaxf(M, mm[w * ROWS + r]);
-    float L = 0.f, O = 0.f;
-    if (M != -INFINITY) {
+    float L = 0.f;
 #pragma unroll
-      for (int w = 0; w < SW; ++w) {
-        float wgt = s_ex2(mm[w * ROWS + r] - M);
-        L += ml[w * ROWS + r] * wgt;
-        O += mo[(w * ROWS + r) * kDh + col] * wgt;
-      }
+    for (int w = 0; w < SW; ++w) {
+      const float wgt = M == -INFINITY ? 0.f : s_ex2(mm[w * ROWS + r] - M);
+      L += ml[w * ROWS + r] * wgt;
+      mm[w * ROWS + r] = wgt;
+    }
+    ml[r] = L;                     // warp 0's slots now hold the merged row sums ...
+    ml[ROWS + r] = M;              // ... and warp 1's the merged maxima
+  }
+  __syncthreads();
+  for (int idx = tid; idx < dm.C * (kDh / 2); idx += STHREADS) {          // two columns per thread
+    const int r = idx / (kDh / 2), col = 2 * (idx % (kDh / 2));
+    const size_t orow = (size_t)(row0 + r) * dm.d + h * kDh + col;
+    if (r >= S) {
+      if (split == 0) *reinterpret_cast<__nv_bfloat162 *>(out + orow) = __floats2bfloat162_rn(0.f, 0.f);
+      continue;
+    }
+    float2 O = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < SW; ++w) {
+      const float wgt = mm[w * ROWS + r];
+      const float2 v = *reinterpret_cast<const float2 *>(&mo[(w * ROWS + r) * SMROW + col]);
+      O.x += v.x * wgt; O.y += v.y * wgt;
     }
     if (a.splits == 1) {
-      out[orow] = __float2bfloat16_rn(O / L);
+      const float inv = 1.f / ml[r];
+      *reinterpret_cast<__nv_bfloat162 *>(out + orow) = __floats2bfloat162_rn(O.x * inv, O.y * inv);
     } else {
-      size_t pi = ((size_t)(row0 + r) * dm.H + h) * a.splits + split;
-      a.part_o[pi * kDh + col] = O;
-      if (col == 0) { a.part_ml[pi * 2] = M; a.part_ml[pi * 2 + 1] = L; }
+      const size_t pi = ((size_t)(row0 + r) * dm.H + h) * a.splits + split;
+      *reinterpret_cast<float2 *>(&a.part_o[pi * kDh + col]) = O;
+      if (col == 0) { a.part_ml[pi * 2] = ml[ROWS + r]; a.part_ml[pi * 2 + 1] = ml[r]; }
     }
   }
 }
 
 static int self_attn_tc_smem(int P, int mt) {
   int ring = SW * SDEPTH * 2 * P * 128;
-  int merge = SW * 16 * mt * (kDh + 2) * 4;
+  int merge = SW * 16 * mt * (SMROW + 2) * 4;
   return ring > merge ? ring : merge;
 }
 
