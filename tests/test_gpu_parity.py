@@ -131,6 +131,21 @@ def test_bf16_sub_max_64_one_key_context_and_unaligned_context():
     dec.close()
 
 
+def test_bf16_long_page_lists():
+    """More pages per sequence than the self-attention kernel's threads (the page list is staged in
+    more than one round), long subsequences over several pages, T5 bias over long distances."""
+    wl = W.CONFIGS["summarisation"].scaled(name="long_lists", batch=2, ctx=150, sub_max=48, delta_t=4, max_sub_len=50,
+                                           length_dist=("uniform", 30, 50), time_max=245, **SMALL_BF16)
+    weights, mem, ctx_len, dec, rows = make(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    runs = parity.oracle_runs(wl, weights, {0: mem[0]}, ctx_len, fl)
+    stats = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    assert dec.stats()["pages"] > 0 and stats["max_err"] < 2e-2
+    import ctypes as C
+    assert dec.cfg.sub_max * (-(-(wl.max_sub_len + 1) // wl.page_tokens)) > 128
+    dec.close()
+
+
 def test_steps_after_the_end_are_no_ops():
     from paper_2506_23431_b200.binding import PipelinedDecoder
     wl = TINY.scaled(vocab=300)
