@@ -212,7 +212,8 @@ def main():
     ap.add_argument("--config", default=DEFAULT_CONFIG, choices=W.CONFIG_ORDER)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-time-steps", type=int, default=24)
-    ap.add_argument("--cpu-baseline-steps", type=int, default=40)
+    ap.add_argument("--cpu-baseline-steps", type=int, default=256,
+                    help="time-steps of batch row 0 the CPU oracle decodes for cpu_baseline (256 = its whole decode on every config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--sequential", action="store_true",

@@ -166,6 +166,7 @@ template <int MT>   // MT = 16-row query tiles (rows per sequence <= 16 * MT)
 __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap, AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ int pfx_s[XMAXB + 1];
+  __shared__ unsigned char nact_s[XMAXB];   // active rows of every sequence (at most 32 here)
   const Dims &dm = a.dm;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, G = gridDim.x, H = dm.H, batch = a.batch;
@@ -178,8 +179,11 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   const uint32_t bar_empty = bar_full + 8 * XSTAGES;
 
   // ---- tiles per head of every sequence, prefix sums, this CTA's range of the flat list
-  for (int b = tid; b < batch; b += XTHREADS)
-    pfx_s[b + 1] = a.st.n_active[b] > 0 ? (a.st.ctx_len[b] + XK - 1) / XK : 0;
+  for (int b = tid; b < batch; b += XTHREADS) {
+    const int S = a.st.n_active[b];
+    nact_s[b] = (unsigned char)S;
+    pfx_s[b + 1] = S > 0 ? (a.st.ctx_len[b] + XK - 1) / XK : 0;
+  }
   if (tid == 0) {
     pfx_s[0] = 0;
     for (int s = 0; s < XSTAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, XCW); }
@@ -198,7 +202,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   }
   // rows of a sequence beyond its active ones come back as zeros (all heads)
   for (int b = cta; b < batch; b += G) {
-    const int S = a.st.n_active[b];
+    const int S = nact_s[b];
     uint4 *z = reinterpret_cast<uint4 *>(out + (size_t)(b * dm.C + S) * dm.d);      // rows are d * 2 bytes, d a multiple of 64
     for (int idx = tid; idx < (dm.C - S) * dm.d / 8; idx += XTHREADS) z[idx] = make_uint4(0u, 0u, 0u, 0u);
   }
@@ -244,7 +248,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
     const int b = cur.b, h = cur.h;
     const int seg_start = H * pfx_s[b] + h * cur.nt, seg_end = seg_start + cur.nt;
     const int my_end = min(hi, seg_end);
-    const int S = a.st.n_active[b], ctx_len = a.st.ctx_len[b];
+    const int S = nact_s[b], ctx_len = a.st.ctx_len[b];
     const int row0 = b * dm.C;
     uint32_t qf[MT][4][4];
 #pragma unroll
