@@ -81,7 +81,9 @@ typedef struct {
   float rope_theta, attn_scale, norm_eps;
   int32_t page_tokens;    /* KV page size in tokens: 16 or 32                                   */
   int32_t pool_pages;     /* KV pool size in pages; 0 = worst case (never exhausts)             */
-  int32_t self_splits, cross_splits; /* split-K factors of the two attention kernels; 0 = auto  */
+  int32_t self_splits, cross_splits; /* split-K factors of the attention kernels; 0 = auto.  The
+                             bf16 tensor-core cross-attention kernel ignores cross_splits: it
+                             divides the context tiles over the GPU by itself                      */
   int32_t use_graph;      /* 1: pd_step replays a CUDA graph captured at the first step         */
   int32_t device;         /* CUDA device ordinal                                                */
 } pd_config;
@@ -104,7 +106,8 @@ typedef struct {
 PD_API size_t pd_workspace_bytes(const pd_config *cfg);
 
 /* Creates a handle: validates cfg, carves the workspace (device, 256-byte aligned, at least
- * pd_workspace_bytes(cfg)), creates the cuBLAS handle and the TMA descriptor.  `cuda_stream`
+ * pd_workspace_bytes(cfg)), creates the cuBLAS handles and the TMA descriptor of the context
+ * keys/values, builds the position tables.  `cuda_stream`
  * is a cudaStream_t (NULL = legacy default stream).  Algorithm 1's inputs delta_t, time_max,
  * sub_max are fixed here. */
 PD_API pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspace, size_t workspace_bytes,

@@ -3,8 +3,9 @@
 //     rule of Section 3.2 evaluated from (subsequence, start step, entry) metadata per page;
 //   * cross-attention over the shared context keys/values (all context rows < ctx_len visible);
 //   * the split-K merge.
-// These are the fp32 path of every configuration and the reference bf16 path; the bf16 hot
-// path for cross-attention is the TMA + tensor-core kernel in cross_attn_tma.cu.
+// These are the fp32 path of every configuration and the bf16 path when a sequence has more
+// than 32 rows; otherwise bf16 runs the tensor-core kernels in self_attn_tc.cu and
+// cross_attn_tma.cu.
 #include "pd_internal.h"
 
 namespace pd {
