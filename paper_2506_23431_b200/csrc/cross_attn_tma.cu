@@ -27,6 +27,7 @@ constexpr int XTHREADS = (XCW + 1) * 32;
 constexpr int XTILE_BYTES = XK * kDh * 2; // 16 KB
 constexpr int XSTAGE_BYTES = 2 * XTILE_BYTES;
 constexpr int XMIN_TILES = 4;              // fewest tiles worth a CTA of its own
+constexpr int XMIN_WHOLE = 64;             // fewest CTAs for which whole (sequence, head) segments per CTA still beat cutting the tile list
 constexpr int XMAXB = 256;                // sequences per launch the tile prefix table holds
 constexpr int XREC_WORDS = 36;            // per lane and 16-row tile: 32 output values, 2 maxima, 2 sums
 constexpr int XREC_FLOATS = XREC_WORDS * 32;
@@ -166,6 +167,8 @@ template <int MT>   // MT = 16-row query tiles (rows per sequence <= 16 * MT)
 __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap, AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ int pfx_s[XMAXB + 1];
+  __shared__ int aseq_s[XMAXB];             // the a-th sequence that has an active row
+  __shared__ int n_aseq_s;
   __shared__ unsigned char nact_s[XMAXB];   // active rows of every sequence (at most 32 here)
   const Dims &dm = a.dm;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -199,6 +202,15 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
       if (c0 + lane < batch) pfx_s[c0 + lane + 1] = v + carry;
       carry += __shfl_sync(0xffffffffu, v, 31);
     }
+  } else if (warp == 1) {   // the sequences that have an active row, in order
+    int n = 0;
+    for (int c0 = 0; c0 < batch; c0 += 32) {
+      const bool on = c0 + lane < batch && nact_s[c0 + lane] > 0;
+      const unsigned m = __ballot_sync(0xffffffffu, on);
+      if (on) aseq_s[n + __popc(m & ((1u << lane) - 1u))] = c0 + lane;
+      n += __popc(m);
+    }
+    if (lane == 0) n_aseq_s = n;
   }
   // rows of a sequence beyond its active ones come back as zeros (all heads)
   for (int b = cta; b < batch; b += G) {
@@ -211,9 +223,28 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   // CTAs that get work: every one of them at least XMIN_TILES tiles (when there are that many), so
   // that few tiles do not turn into many one-tile CTAs whose records one CTA then merges serially
   const long long want = (T + XMIN_TILES - 1) / XMIN_TILES;
-  const int Ge = (int)(want < G ? want : G);
-  if (cta >= Ge) return;
-  const int lo = (int)(cta * T / Ge), hi = (int)((cta + 1) * T / Ge);
+  int Ge = (int)(want < G ? want : G);
+  int lo, hi;
+  // With enough (sequence, head) segments to keep at least one CTA per SM streaming, every CTA takes
+  // whole segments (the same number each): nothing is cut, so there are no partial records, no
+  // tickets and no merge after the last tile.  Otherwise the tile list itself is cut into equal ranges.
+  const int n_seg = n_aseq_s * H;
+  const int seg_per_cta = (n_seg + G - 1) / G;
+  const bool whole_segments = n_seg > 0 && (n_seg + seg_per_cta - 1) / seg_per_cta >= XMIN_WHOLE;
+  if (whole_segments) {
+    Ge = (n_seg + seg_per_cta - 1) / seg_per_cta;
+    if (cta >= Ge) return;
+    auto seg_tile = [&](int sidx) {    // first tile of segment sidx in the flat list
+      if (sidx >= n_seg) return (int)T;
+      const int bb = aseq_s[sidx / H], hh = sidx % H;
+      return H * pfx_s[bb] + hh * (pfx_s[bb + 1] - pfx_s[bb]);
+    };
+    lo = seg_tile(cta * seg_per_cta);
+    hi = seg_tile((cta + 1) * seg_per_cta);
+  } else {
+    if (cta >= Ge) return;
+    lo = (int)(cta * T / Ge); hi = (int)((cta + 1) * T / Ge);
+  }
 
   if (warp == XCW) {
     // ------------------------------------------------------------------ producer (one lane)
