@@ -4,9 +4,10 @@
 // contraction, so it runs on tensor cores; it stays HBM-bound (about S flop per byte).
 //
 // Persistent kernel, two CTAs per SM.  The 128-key tiles of all (sequence with an active row,
-// head) pairs form one flat list that is cut into equal contiguous ranges, one per CTA, whatever
-// the number of active sequences: the GPU stays full when few sequences are left, and there
-// are no partial waves.  In every CTA a producer warp streams the K and V tiles of its range
+// head) pairs form one flat list.  With enough (sequence, head) segments every CTA takes the same
+// number of whole segments (nothing is cut: no partial records, no merge); with few segments left
+// the list is cut into equal contiguous ranges, one per CTA, so that the GPU stays full.  Either
+// way there are no partial waves.  In every CTA a producer warp streams the K and V tiles of its range
 // (16 KB each, contiguous) through a ring of shared-memory stages with TMA (cp.async.bulk.tensor.2d,
 // 128-byte swizzle, completion on an mbarrier) without stopping at (sequence, head) boundaries;
 // four consumer warps each take 32 keys of every tile: S = Q K^T with mma.sync m16n8k16 (bf16 in,
