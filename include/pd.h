@@ -238,6 +238,26 @@ PD_API pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_p
                              float attn_scale, int32_t splits, const void *q, const void *kv, const int32_t *n_rows,
                              const int32_t *ctx_len, void *out, void *scratch, size_t scratch_bytes, void *cuda_stream);
 
+/* The vocabulary projection and greedy choice alone (Eq. 4: the token with the highest
+ * probability, i.e. the largest logit, ties to the lowest id), on caller-supplied rows and
+ * without a handle: logits[r][v] = sum_k hidden[r][k] * lm_head[v][k] in bf16 with fp32
+ * accumulation on the tcgen05 tensor cores, the per-row maximum taken inside the same kernel -
+ * the [rows, vocab] logits are only written when `logits` is given.
+ *   hidden     device bf16 [rows, d_model], 16-byte aligned; d_model a multiple of 64
+ *   lm_head    device bf16 [vocab, d_model], 16-byte aligned
+ *   best_id    device int32 [rows] out;  best_val  device fp32 [rows] out, or NULL
+ *   logits     device fp32 [rows, vocab] out, or NULL
+ *   scratch    device, 256-byte aligned, at least pd_vocab_argmax_scratch_bytes(rows, vocab): a
+ *              256-byte header (int32 word 2 receives PD_ERR_TIMEOUT if a bounded wait inside the
+ *              kernel expired; cleared by the call), then per-slice partial maxima
+ * Enqueues on cuda_stream and returns; allocates nothing on the device; the caller owns every
+ * buffer.  PD_ERR_ARG for null pointers, misaligned buffers or sizes out of range,
+ * PD_ERR_WORKSPACE for a scratch that is too small, PD_ERR_CUDA if a launch fails. */
+PD_API size_t pd_vocab_argmax_scratch_bytes(int32_t rows, int32_t vocab);
+PD_API pd_status pd_vocab_argmax(int32_t rows, int32_t d_model, int32_t vocab, const void *hidden, const void *lm_head,
+                                 int32_t *best_id, float *best_val, float *logits, void *scratch, size_t scratch_bytes,
+                                 void *cuda_stream);
+
 /* pd_cross_attention without a scratch argument (an addition of this library; the paper has no
  * counterpart).  Some callers have no way to obtain device memory at the moment they need the
  * op: a plug-in that runs inside a host framework which owns the whole device heap and hands

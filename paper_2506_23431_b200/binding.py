@@ -69,6 +69,8 @@ _SIGS = {
     "pd_cross_attention_scratch_bytes": (C.c_size_t, [C.c_int32] * 4),
     "pd_cross_attention": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p, C.c_size_t,
                                                                                                   C.c_void_p]),
+    "pd_vocab_argmax_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
+    "pd_vocab_argmax": (C.c_int, [C.c_int32] * 3 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]),
     "pd_cross_attention_static_max_bytes": (C.c_size_t, []),
     "pd_cross_attention_static": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p]),
     "pd_static_last_error": (C.c_char_p, []),
@@ -358,6 +360,30 @@ def cross_attention_static(q, kv, n_rows, ctx_len, attn_scale: float, splits: in
 
 def cross_attention_static_max_bytes() -> int:
     return int(_lib.pd_cross_attention_static_max_bytes())
+
+
+def vocab_argmax(hidden, lm_head, want_logits: bool = False, scratch=None):
+    """pd_vocab_argmax on torch CUDA tensors: hidden [rows, d] and lm_head [vocab, d], both bfloat16.
+    Runs on torch's current stream; returns (best_id int32 [rows], best_val float32 [rows], logits
+    float32 [rows, vocab] or None)."""
+    import torch
+    if hidden.dtype != torch.bfloat16 or lm_head.dtype != torch.bfloat16:
+        raise ValueError("hidden and lm_head must be bfloat16")
+    hidden, lm_head = hidden.contiguous(), lm_head.contiguous()
+    rows, d = hidden.shape
+    vocab = lm_head.shape[0]
+    if scratch is None:
+        n = int(_lib.pd_vocab_argmax_scratch_bytes(rows, vocab))
+        scratch = torch.empty(max(n, 256), dtype=torch.uint8, device=hidden.device)
+    best_id = torch.empty(rows, dtype=torch.int32, device=hidden.device)
+    best_val = torch.empty(rows, dtype=torch.float32, device=hidden.device)
+    logits = torch.empty(rows, vocab, dtype=torch.float32, device=hidden.device) if want_logits else None
+    st = _lib.pd_vocab_argmax(rows, d, vocab, hidden.data_ptr(), lm_head.data_ptr(), best_id.data_ptr(), best_val.data_ptr(),
+                              logits.data_ptr() if want_logits else None, scratch.data_ptr(), scratch.numel(),
+                              torch.cuda.current_stream(hidden.device).cuda_stream)
+    if st != 0:
+        raise PdError(st, "pd_vocab_argmax")
+    return best_id, best_val, logits
 
 
 def version() -> str:

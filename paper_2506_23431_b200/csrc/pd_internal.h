@@ -127,6 +127,27 @@ int cross_attn_tma_smem_bytes();
 cudaError_t cross_attn_tma_prepare();   // once per device, outside any stream capture
 
 
+// ---- vocabulary projection + per-slice maxima on tcgen05 (vocab_tc.cu) -------------------------
+struct VocabArgs {
+  const int32_t *n_active;   // [batch] active rows per sequence (the rows of `hidden` are these, packed), or null
+  int batch;
+  int m_fixed;               // number of rows when n_active is null
+  int V, K;                  // vocabulary size, model width (a multiple of 64)
+  int rows_cap;              // row stride of the partial arrays (>= the largest row count)
+  int eos, sep;              // ids kept out of the maxima (their logits go to term_val); -1 = none
+  float *part_val;           // [tiles][rows_cap] maximum of the row over the tile's ids
+  int32_t *part_idx;         // [tiles][rows_cap] the id that holds it (lowest on ties; INT_MAX = none)
+  float *term_val;           // [rows_cap][2] logits of eos and sep
+  float *logits;             // [rows][V] fp32, or null when nobody reads them
+  int32_t *status;           // error word (PD_ERR_TIMEOUT on an expired wait)
+};
+int vocab_tc_tiles(int V);
+bool vocab_tc_supported(int K, int V);
+cudaError_t vocab_tc_prepare();          // once per device, outside any stream capture
+cudaError_t encode_vocab_maps(CUtensorMap *map_a, CUtensorMap *map_b, const void *hidden, uint64_t rows, const void *lm_head,
+                              uint64_t vocab, uint64_t K, int *driver_code);
+cudaError_t launch_vocab_tc(const CUtensorMap &map_a, const CUtensorMap &map_b, const VocabArgs &a, cudaStream_t s);
+
 // ---- stand-alone cross-attention (attn_ops.cu) ---------------------------------------------
 size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
                                       size_t *off_part_o, size_t *off_part_ml);

@@ -92,3 +92,62 @@ def test_cross_attention_rejects_bad_arguments():
     assert e.value.status == -1
     assert B.cross_attention_scratch_bytes(1, 65, 1, 1) == 0
     assert B._lib.pd_cross_attention(0, 1, 4, 1, 8, C.c_float(0.125), 1, None, None, None, None, None, None, 0, None) == -1
+
+
+VOCAB_CASES = [
+    # rows, d_model, vocab
+    (100, 64, 224),        # one row tile, one vocabulary slice, a single K block
+    (200, 256, 1000),      # two row tiles (ragged), five slices, the last one partly beyond the vocabulary
+    (600, 1024, 5000),     # five row tiles: three passes over every slice
+]
+
+
+@pytest.mark.parametrize("rows,d_model,vocab", VOCAB_CASES)
+def test_vocab_argmax_kernel_against_oracle(rows, d_model, vocab):
+    """Eq. 4's greedy choice on the tensor-core kernel: logits against the fp64 product of the same
+    bf16 inputs, ids against the oracle's select_token wherever its top-2 margin is above 1e-3."""
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    g = np.random.Generator(np.random.Philox(key=np.array([rows, vocab], dtype=np.uint64)))
+    hidden = W.bf16_round(g.standard_normal((rows, d_model), dtype=np.float32))
+    lm_head = W.bf16_round(0.05 * g.standard_normal((vocab, d_model), dtype=np.float32))
+    lm_head[7] = lm_head[3]                                   # an exact tie: the lower id must win
+    ref = hidden.astype(np.float64) @ lm_head.astype(np.float64).T
+    dev = torch.device("cuda", 0)
+    h_d = torch.from_numpy(hidden).to(dev, torch.bfloat16)
+    w_d = torch.from_numpy(lm_head).to(dev, torch.bfloat16)
+    best_id, best_val, logits = B.vocab_argmax(h_d, w_d, want_logits=True)
+    id_only, _, none = B.vocab_argmax(h_d, w_d, want_logits=False)
+    torch.cuda.synchronize()
+    assert none is None
+    got = logits.cpu().numpy().astype(np.float64)
+    tol = 1e-4 * max(1.0, np.abs(ref).max())
+    assert np.abs(got - ref).max() <= tol
+    assert np.abs(best_val.cpu().numpy() - ref.max(axis=1)).max() <= tol
+    ids = best_id.cpu().numpy()
+    assert (id_only.cpu().numpy() == ids).all(), "writing the logits or not must not change the choice"
+    assert not (ids == 7).any()
+    top2 = np.sort(ref, axis=1)[:, -2:]
+    for r in range(rows):
+        row = ref[r].copy()
+        row[7] = -np.inf                                      # the tie's higher id can never be chosen
+        if np.sort(row)[-1] - np.sort(row)[-2] > 1e-3:
+            tok, _ = O.select_token(ref[r], 0, None, 10 ** 9, -1, -1)
+            assert ids[r] == tok, f"row {r}: {ids[r]} != {tok} (margin {top2[r, 1] - top2[r, 0]:.3e})"
+
+
+def test_vocab_argmax_rejects_bad_arguments():
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    h = torch.zeros(4, 96, device=dev, dtype=torch.bfloat16)           # width not a multiple of 64
+    w = torch.zeros(10, 96, device=dev, dtype=torch.bfloat16)
+    with pytest.raises(B.PdError) as e:
+        B.vocab_argmax(h, w)
+    assert e.value.status == -1
+    h = torch.zeros(4, 64, device=dev, dtype=torch.bfloat16)
+    w = torch.zeros(10, 64, device=dev, dtype=torch.bfloat16)
+    with pytest.raises(B.PdError) as e:
+        B.vocab_argmax(h, w, scratch=torch.empty(256, dtype=torch.uint8, device=dev))
+    assert e.value.status == -3
+    assert B._lib.pd_vocab_argmax_scratch_bytes(0, 10) == 0
