@@ -262,7 +262,7 @@ def main():
     ctx_len = W.make_ctx_len(wl_data)
     fl = W.make_forced_len(wl_data)
     dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, device=local_rank, use_graph=not args.no_graph,
-                           self_splits=args.self_splits, cross_splits=args.cross_splits)
+                           self_splits=args.self_splits, cross_splits=args.cross_splits, store_logits=False)
     mem_dev = dec.device_memory(mem)
     host_mem = torch.from_numpy(mem).to(dec.tdtype).pin_memory()
     e = 2 if wl.dtype == "bf16" else 4
@@ -401,7 +401,8 @@ def main():
         # the same targets decoded by the ordinary sequential decoder (sub_max = 1) with the same library
         dec.close()
         swl, sfl = sequential_workload(wl, fl)
-        sdec = PipelinedDecoder(swl.hyper(), weights, swl.batch, device=local_rank, use_graph=not args.no_graph)
+        sdec = PipelinedDecoder(swl.hyper(), weights, swl.batch, device=local_rank, use_graph=not args.no_graph,
+                                store_logits=False)
         s_ms = []
         for k in range(args.warmup + args.steps):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

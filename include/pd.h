@@ -85,6 +85,10 @@ typedef struct {
                              bf16 tensor-core cross-attention kernel ignores cross_splits: it
                              divides the context tiles over the GPU by itself                      */
   int32_t use_graph;      /* 1: pd_step replays a CUDA graph captured at the first step         */
+  int32_t store_logits;   /* 1: every step leaves its fp32 logits behind for pd_get_logits.  0: on the
+                             bf16 path the vocabulary projection keeps the logits on chip (only the
+                             greedy choice of Eq. 4 leaves the kernel) and pd_get_logits returns
+                             PD_ERR_STATE; the fp32 path stores them either way                    */
   int32_t device;         /* CUDA device ordinal                                                */
 } pd_config;
 

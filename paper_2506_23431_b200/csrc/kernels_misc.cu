@@ -156,6 +156,51 @@ cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, 
   return cudaGetLastError();
 }
 
+// The same norm for the rows that feed the vocabulary projection: only active rows are written,
+// packed back to back in (sequence, row) order, so that the projection's work follows the rows
+// that exist.  Row (b, c) goes to crow[b] + c with crow[b] = active rows of the sequences before b;
+// the CTA of row (b, 0) publishes crow[b] for the kernels that follow.
+template <typename T>
+__global__ void __launch_bounds__(RN_THREADS) rmsnorm_packed_kernel(int d, float eps, int C, DecState st,
+                                                                    const float *__restrict__ x, const T *__restrict__ gain,
+                                                                    T *__restrict__ out) {
+  __shared__ float red[RN_THREADS / 32];
+  __shared__ int redi[RN_THREADS / 32];
+  const int b = blockIdx.x / C, c = blockIdx.x % C;
+  int before = 0;
+  for (int bb = threadIdx.x; bb < b; bb += RN_THREADS) before += st.n_active[bb];
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+  if ((threadIdx.x & 31) == 0) redi[threadIdx.x >> 5] = before;
+  __syncthreads();
+  before = 0;
+#pragma unroll
+  for (int w = 0; w < RN_THREADS / 32; ++w) before += redi[w];
+  if (c == 0 && threadIdx.x == 0) st.crow[b] = before;
+  if (c >= st.n_active[b]) return;
+  const float *xr = x + (size_t)blockIdx.x * d;
+  T *orow = out + (size_t)(before + c) * d;
+  float ss = 0.f;
+  for (int col = threadIdx.x; col < d; col += RN_THREADS) { const float t = xr[col]; ss += t * t; }
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < RN_THREADS / 32; ++w) tot += red[w];
+  const float inv = rsqrtf(tot / (float)d + eps);
+  for (int col = threadIdx.x; col < d; col += RN_THREADS) orow[col] = from_f<T>(xr[col] * inv * to_f<T>(gain[col]));
+}
+
+cudaError_t launch_rmsnorm_packed(const Dims &dm, const DecState &st, int batch, int dtype, const float *x, const void *gain,
+                                  void *out, cudaStream_t s) {
+  if (dtype == PD_DTYPE_BF16)
+    rmsnorm_packed_kernel<__nv_bfloat16><<<batch * dm.C, RN_THREADS, 0, s>>>(dm.d, dm.eps, dm.C, st, x, (const __nv_bfloat16 *)gain,
+                                                                             (__nv_bfloat16 *)out);
+  else
+    rmsnorm_packed_kernel<float><<<batch * dm.C, RN_THREADS, 0, s>>>(dm.d, dm.eps, dm.C, st, x, (const float *)gain, (float *)out);
+  return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void relu_kernel(T *buf, size_t n) {

@@ -23,9 +23,9 @@ struct Region { size_t off = 0, bytes = 0; };
 struct Layout {
   // integer state (offsets in int32 words from the start of the state block)
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
-      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, state_words;
+      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, w_crow, state_words;
   Region state, plist, row_meta, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
-      ffn, logits, part_o, part_ml, kv_c, kv_pool, enc_stage, proj_stage, cublas_ws;
+      ffn, logits, vpart_val, vpart_idx, vterm, part_o, part_ml, kv_c, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
 };
 
@@ -42,6 +42,7 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   const int ids[3] = {c.bos_id, c.eos_id, c.sep_id};
   for (int v : ids) if (v < 0 || v >= c.vocab) return false;
   if (c.self_splits < 0 || c.self_splits > 32 || c.cross_splits < 0 || c.cross_splits > 32) return false;
+  if (c.store_logits != 0 && c.store_logits != 1) return false;
   if (!(c.attn_scale > 0.f) || !(c.norm_eps >= 0.f)) return false;
   dm.L = c.n_layers; dm.d = c.d_model; dm.H = c.n_heads; dm.ff = c.d_ff; dm.V = c.vocab;
   dm.B = c.max_batch; dm.ctx = c.max_ctx; dm.SM = c.sub_max; dm.dt = c.delta_t; dm.T = c.time_max;
@@ -73,6 +74,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   L.w_trace = take(2 * (size_t)dm.T * B);         // 64-bit masks
   L.w_plist_n = take(B);
   L.w_xtick = take(B * dm.H);
+  L.w_crow = take(B);
   L.w_k = take(B); L.w_done = take(B); L.w_steps = take(B); L.w_nact = take(B); L.w_ctx = take(B); L.w_ticket = take(B);
   L.w_start = take(B * SM); L.w_len = take(B * SM); L.w_state = take(B * SM); L.w_flag = take(B * SM);
   L.w_last = take(B * SM); L.w_forced = take(B * SM);
@@ -104,6 +106,12 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   reg(L.cross_out, M * dm.d * e);
   reg(L.ffn, M * dm.ff * e);
   reg(L.logits, M * (size_t)dm.V * 4);
+  {
+    const size_t tiles = (size_t)vocab_tc_tiles(dm.V);      // per-slice candidates of the vocabulary projection
+    reg(L.vpart_val, tiles * M * 4);
+    reg(L.vpart_idx, tiles * M * 4);
+    reg(L.vterm, M * 2 * 4);
+  }
   {
     size_t split_bytes = M * dm.H * max_splits * kDh * 4, flat_bytes = cross_attn_tma_partial_bytes(kMaxCrossCtas, dm.C);
     reg(L.part_o, split_bytes > flat_bytes ? split_bytes : flat_bytes);
@@ -140,6 +148,8 @@ struct pd_handle {
   pd_weights w;
   CUtensorMap tmap_kvc;
   bool have_tmap = false;
+  CUtensorMap vmap_a, vmap_b;      // hidden rows and lm_head for the tcgen05 vocabulary projection
+  bool vocab_tc = false;
   int batch = 0;
   bool encoded = false;
   int self_splits = 1, cross_splits = 1;
@@ -346,6 +356,21 @@ pd_status enqueue_step(pd_handle *h) {
     }
     PD_TRY(gemm(h, false, M, dm.d, dm.ff, ffn, lw[9], x, true, 1.f));
   }
+  if (h->vocab_tc) {
+    // active rows only, packed; logits stay in tensor memory unless they were asked for
+    VocabArgs va;
+    va.n_active = h->st.n_active; va.batch = h->batch; va.m_fixed = 0; va.V = dm.V; va.K = dm.d; va.rows_cap = M;
+    va.eos = dm.eos; va.sep = dm.sep;
+    va.part_val = h->ptr<float>(h->lay.vpart_val); va.part_idx = h->ptr<int32_t>(h->lay.vpart_idx);
+    va.term_val = h->ptr<float>(h->lay.vterm);
+    va.logits = h->cfg.store_logits ? logits : nullptr;
+    va.status = h->st.hdr + HDR_STATUS;
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm_packed(dm, h->st, h->batch, dt, x, h->w.final_norm, hb, s));
+    OWN(h, PD_PROF_ARGMAX_SCHED, launch_vocab_tc(h->vmap_a, h->vmap_b, va, s));
+    OWN(h, PD_PROF_ARGMAX_SCHED, launch_pick_sched(dm, h->st, h->batch, vocab_tc_tiles(dm.V), va.part_val, va.part_idx, va.term_val,
+                                                   h->ptr<int32_t>(h->lay.teacher), s));
+    return PD_OK;
+  }
   OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, h->w.final_norm, hb, s));
   PD_TRY(gemm(h, true, M, dm.V, dm.d, hb, h->w.lm_head, logits, true, 0.f));
   OWN(h, PD_PROF_ARGMAX_SCHED, launch_argmax_sched(dm, h->st, h->batch, logits, h->ptr<int32_t>(h->lay.teacher), s));
@@ -427,7 +452,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   st.hdr = sb + L.w_hdr; st.stats = reinterpret_cast<unsigned long long *>(sb + L.w_stats);
   st.trace = reinterpret_cast<unsigned long long *>(sb + L.w_trace);
   st.k = sb + L.w_k; st.done = sb + L.w_done; st.steps = sb + L.w_steps; st.n_active = sb + L.w_nact;
-  st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket;
+  st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket; st.crow = sb + L.w_crow;
   st.plist_n = sb + L.w_plist_n; st.plist = h->ptr<int4>(L.plist); st.row_meta = h->ptr<int4>(L.row_meta);
   st.start = sb + L.w_start; st.len = sb + L.w_len; st.state = sb + L.w_state; st.flag = sb + L.w_flag;
   st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced;
@@ -460,6 +485,14 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
     h->cross_ctas = cross_attn_ctas();
   }
   if (cfg->dtype == PD_DTYPE_BF16 && self_attn_tc_supported(dm) && self_attn_tc_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
+  if (cfg->dtype == PD_DTYPE_BF16 && vocab_tc_supported(dm.d, dm.V) && reinterpret_cast<uintptr_t>(weights->lm_head) % 16 == 0) {
+    int code = 0;
+    if (encode_vocab_maps(&h->vmap_a, &h->vmap_b, h->ptr<void>(L.hbuf), (uint64_t)dm.B * dm.C, weights->lm_head, (uint64_t)dm.V,
+                          (uint64_t)dm.d, &code) != cudaSuccess)
+      return bail(PD_ERR_CUDA);
+    if (vocab_tc_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
+    h->vocab_tc = true;
+  }
   *out = h;
   return PD_OK;
 }
@@ -630,6 +663,23 @@ pd_status pd_get_logits(pd_handle *h, float *logits, int32_t *row_sub) {
   if (!h) return PD_ERR_ARG;
   if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_get_logits before pd_encode_context");
   const size_t rows = (size_t)h->batch * h->dm.C;
+  if (h->vocab_tc && logits) {
+    // The tensor-core projection stores the rows that were active, packed in (sequence, row) order.
+    if (!h->cfg.store_logits) return fail(h, PD_ERR_STATE, "pd_get_logits: the handle was made with store_logits = 0");
+    std::vector<int32_t> prs(rows);
+    CU_TRY(h, cudaMemcpyAsync(prs.data(), h->st.prev_row_sub, rows * 4, cudaMemcpyDeviceToHost, h->stream));
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    const size_t row_bytes = (size_t)h->dm.V * 4;
+    const uint8_t *src = h->ptr<uint8_t>(h->lay.logits);
+    size_t packed = 0;
+    for (size_t r = 0; r < rows; ++r) {
+      if (prs[r] > 0) CU_TRY(h, cudaMemcpyAsync(logits + r * h->dm.V, src + packed++ * row_bytes, row_bytes, cudaMemcpyDeviceToHost, h->stream));
+      else memset(logits + r * h->dm.V, 0, row_bytes);
+    }
+    if (row_sub) memcpy(row_sub, prs.data(), rows * 4);
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    return PD_OK;
+  }
   if (logits) CU_TRY(h, cudaMemcpyAsync(logits, h->ptr<void>(h->lay.logits), rows * h->dm.V * 4, cudaMemcpyDeviceToHost, h->stream));
   if (row_sub) CU_TRY(h, cudaMemcpyAsync(row_sub, h->st.prev_row_sub, rows * 4, cudaMemcpyDeviceToHost, h->stream));
   CU_TRY(h, cudaStreamSynchronize(h->stream));

@@ -69,6 +69,7 @@ struct DecState {
   int32_t *hdr;                 // [HDR_WORDS]
   unsigned long long *stats;    // [PD_STAT_COUNT]
   int32_t *k, *done, *steps, *n_active, *ctx_len, *seq_ticket;        // [B]
+  int32_t *crow;                // [B] first row of the sequence among the step's active rows packed back to back
   int32_t *plist_n;             // [B] entries of the sequence's page list for the coming step
   int4 *row_meta;               // [B*C] per row: (page, slot in it, position tau + i) of the entry the coming step appends, subsequence i (0 = unused row)
   int4 *plist;                  // [B][SM*PPS] (page, entries in it, subsequence i', distance base t - (tau' + i') of entry 0)
@@ -104,6 +105,8 @@ cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtyp
                          cudaStream_t s);
 cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, const void *gain, void *out,
                            cudaStream_t s);
+cudaError_t launch_rmsnorm_packed(const Dims &dm, const DecState &st, int batch, int dtype, const float *x, const void *gain,
+                                  void *out, cudaStream_t s);
 cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s);
 cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
                           void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s);
@@ -122,6 +125,8 @@ cudaError_t self_attn_tc_prepare();     // once per device, outside any stream c
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s);
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
                                 const int32_t *teacher, cudaStream_t s);
+cudaError_t launch_pick_sched(const Dims &dm, const DecState &st, int batch, int tiles, const float *part_val,
+                              const int32_t *part_idx, const float *term_val, const int32_t *teacher, cudaStream_t s);
 cudaError_t encode_ctx_kv_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, int *driver_code);
 int cross_attn_tma_smem_bytes();
 cudaError_t cross_attn_tma_prepare();   // once per device, outside any stream capture

@@ -127,6 +127,33 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
   st.plist_n[b] = np;
 }
 
+// Called by every thread of a row's CTA once the row's choice is in row_tok: the CTA that arrives
+// last for its sequence runs the sequence's scheduler, the last sequence advances the step.
+__device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, const int32_t *teacher, int *is_last) {
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    __threadfence();
+    int ticket = atomicAdd(&st.seq_ticket[b], 1);
+    *is_last = ticket == dm.C - 1;
+  }
+  __syncthreads();
+  if (!*is_last || tid != 0) return;
+  __threadfence();
+  st.seq_ticket[b] = 0;
+  schedule_sequence(dm, st, batch, b, teacher);
+  __threadfence();
+  if (atomicAdd(&st.hdr[HDR_TICKET], 1) == batch - 1) {   // last sequence of the step
+    __threadfence();
+    st.hdr[HDR_TICKET] = 0;
+    const int n_done = atomicAdd(&st.hdr[HDR_N_DONE], 0);
+    if (st.hdr[HDR_ALL_DONE] == 0) {
+      atomicAdd(&st.stats[PD_STAT_STEPS], 1ull);
+      if (n_done >= batch) st.hdr[HDR_ALL_DONE] = 1;
+      else st.hdr[HDR_STEP_T] = st.hdr[HDR_STEP_T] + 1;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, int batch, const float *__restrict__ logits,
                                                           const int32_t *__restrict__ teacher) {
   __shared__ float sv[AT / 32];
@@ -181,32 +208,60 @@ __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, 
       st.row_tok[r] = bi == INT_MAX ? 0 : bi;
     }
   }
-  if (tid == 0) {
-    __threadfence();
-    int ticket = atomicAdd(&st.seq_ticket[b], 1);
-    is_last = ticket == dm.C - 1;
-  }
-  __syncthreads();
-  if (!is_last || tid != 0) return;
-  __threadfence();
-  st.seq_ticket[b] = 0;
-  schedule_sequence(dm, st, batch, b, teacher);
-  __threadfence();
-  if (atomicAdd(&st.hdr[HDR_TICKET], 1) == batch - 1) {   // last sequence of the step
-    __threadfence();
-    st.hdr[HDR_TICKET] = 0;
-    const int n_done = atomicAdd(&st.hdr[HDR_N_DONE], 0);
-    if (st.hdr[HDR_ALL_DONE] == 0) {
-      atomicAdd(&st.stats[PD_STAT_STEPS], 1ull);
-      if (n_done >= batch) st.hdr[HDR_ALL_DONE] = 1;
-      else st.hdr[HDR_STEP_T] = st.hdr[HDR_STEP_T] + 1;
-    }
-  }
+  row_done(dm, st, batch, b, teacher, &is_last);
 }
 
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
                                 const int32_t *teacher, cudaStream_t s) {
   argmax_sched_kernel<<<batch * dm.C, AT, 0, s>>>(dm, st, batch, logits, teacher);
+  return cudaGetLastError();
+}
+
+// The same step when the vocabulary projection has already reduced every row to one candidate per
+// vocabulary slice (vocab_tc.cu): one warp-sized CTA per row finishes the greedy choice over the
+// slices' maxima - ties to the lowest id; eos and sep, kept apart by the projection, join unless the
+// forced length bars them - and hands over to the scheduler exactly as above.
+constexpr int PT = 64;
+
+__global__ void __launch_bounds__(PT) pick_sched_kernel(Dims dm, DecState st, int batch, int tiles, int rows_cap,
+                                                        const float *__restrict__ part_val, const int32_t *__restrict__ part_idx,
+                                                        const float *__restrict__ term_val, const int32_t *__restrict__ teacher) {
+  __shared__ float sv[PT / 32];
+  __shared__ int si[PT / 32];
+  __shared__ int is_last;
+  const int r = blockIdx.x, tid = threadIdx.x;
+  const int b = r / dm.C;
+  const int i = st.row_sub[r];
+  if (i > 0) {
+    const int sidx = b * dm.SM + i - 1;
+    const int fl = st.forced_len[sidx];
+    const bool bar = fl >= 0 && st.len[sidx] < fl;     // terminators cannot win before the forced length
+    const int m = st.crow[b] + r % dm.C;               // the row's place among the packed rows
+    float bv = -INFINITY;
+    int bi = INT_MAX;
+    for (int t = tid; t < tiles; t += PT) better(bv, bi, __ldcg(part_val + (size_t)t * rows_cap + m), __ldcg(part_idx + (size_t)t * rows_cap + m));
+    if (tid == 0 && !bar) {
+      better(bv, bi, __ldcg(term_val + 2 * m), dm.eos);
+      if (dm.sep != dm.eos) better(bv, bi, __ldcg(term_val + 2 * m + 1), dm.sep);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      better(bv, bi, ov, oi);
+    }
+    if ((tid & 31) == 0) { sv[tid >> 5] = bv; si[tid >> 5] = bi; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < PT / 32; ++w) better(bv, bi, sv[w], si[w]);
+      st.row_tok[r] = bi == INT_MAX ? 0 : bi;
+    }
+  }
+  row_done(dm, st, batch, b, teacher, &is_last);
+}
+
+cudaError_t launch_pick_sched(const Dims &dm, const DecState &st, int batch, int tiles, const float *part_val,
+                              const int32_t *part_idx, const float *term_val, const int32_t *teacher, cudaStream_t s) {
+  pick_sched_kernel<<<batch * dm.C, PT, 0, s>>>(dm, st, batch, tiles, batch * dm.C, part_val, part_idx, term_val, teacher);
   return cudaGetLastError();
 }
 

@@ -235,6 +235,37 @@ def test_generate_host_matches_stepwise_run():
     dec.close()
 
 
+def test_bf16_choices_do_not_depend_on_storing_the_logits():
+    """store_logits = 0 keeps the logits inside the vocabulary kernel; the streams, the recorded
+    greedy choices and the schedule must be those of a run that stores them, and pd_get_logits
+    must say that there is nothing to read."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder, PdError
+    wl = W.CONFIGS["bart_base"].scaled(name="small_nolog", batch=5, ctx=200, sub_max=7, delta_t=2, max_sub_len=30,
+                                       length_dist=("uniform", 1, 30), time_max=60, **SMALL_BF16)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    out = []
+    for store in (True, False):
+        dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, store_logits=store)
+        dec.encode_context(dec.device_memory(mem), ctx_len, fl)
+        dec.step()
+        if store:
+            lg, rs = dec.get_logits()
+            assert np.isfinite(lg[rs.reshape(-1) > 0]).all()
+        else:
+            with pytest.raises(PdError) as e:
+                dec.get_logits()
+            assert e.value.status == -2
+        dec.run()
+        res = dec.collect()
+        res["chosen"] = dec.get_chosen()
+        res["trace"] = dec.get_trace()
+        out.append(res)
+        dec.close()
+    for k in out[0]:
+        assert np.array_equal(out[0][k], out[1][k]), k
+
+
 FULL = [("bart_base", 2e-2), ("long_context", 2e-2), ("summarisation", 2e-2), ("keyphrase", 2e-2)]
 
 
