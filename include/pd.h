@@ -117,7 +117,7 @@ PD_API size_t pd_workspace_bytes(const pd_config *cfg);
 PD_API pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspace, size_t workspace_bytes,
                   void *cuda_stream, pd_handle **out);
 
-/* Algorithm 1 lines 1-3 with H^E supplied: resets all decode state, projects the encoder
+/* The initialisation of Algorithm 1 with H^E supplied: resets all decode state, projects the encoder
  * memory to per-layer cross-attention keys/values, admits subsequence 1 of every sequence.
  * enc_mem: device [batch, max_ctx, d_model] of cfg.dtype (rows at or beyond ctx_len[b] are
  * ignored).  ctx_len: host [batch], 1..max_ctx.  forced_len: host [batch, sub_max] or NULL;
@@ -127,9 +127,9 @@ PD_API pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *
 PD_API pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ctx_len, int32_t batch,
                             const int32_t *forced_len);
 
-/* One iteration of Algorithm 1's loop (lines 4-13) for every sequence of the batch: one
+/* One iteration of Algorithm 1's loop for every sequence of the batch: one
  * decoder pass (Eq. 3) for all active subsequences, greedy choice (Eq. 4), append, retire on
- * eos/sep, stop test, and the admission that line 5-7 would do at the top of the next step.
+ * eos/sep, stop test, and the admission the loop would do at the top of the next step.
  * teacher_tokens: device [batch, sub_max] int32 or NULL; an entry >= 0 replaces the chosen
  * token of that subsequence as the one appended (the library's own choice is still recorded);
  * -1 keeps the own choice.  Enqueues only; a no-op for sequences that are done. */
@@ -142,7 +142,7 @@ PD_API pd_status pd_run(pd_handle *h, int32_t poll_every, int32_t *steps_run);
 /* Synchronises the stream; *all_done = 1 when every sequence has ended or hit time_max. */
 PD_API pd_status pd_done(pd_handle *h, int32_t *all_done);
 
-/* Algorithm 1 line 14: the subsequences without bos and terminator.  Host outputs (any may be
+/* The result of Algorithm 1: the subsequences without bos and terminator.  Host outputs (any may be
  * NULL): tokens [batch, sub_max, max_sub_len] (unused tail = -1), lens [batch, sub_max],
  * n_sub [batch] (k at the end), flags [batch, sub_max] (PD_FLAG_*), steps [batch] (the step
  * at which the sequence stopped).  Synchronises; returns a pending device error if any. */

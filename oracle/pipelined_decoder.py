@@ -206,7 +206,7 @@ class PipelinedDecoderOracle:
         """[N, H*dh] -> [H, N, dh]."""
         return np.ascontiguousarray(a.reshape(a.shape[0], self.H, self.dh).transpose(1, 0, 2))
 
-    # ---- context: H^E is handed over (Algorithm 1 line 3); its per-layer keys/values are fixed
+    # ---- context: H^E is handed over (Algorithm 1, initialisation); its per-layer keys/values are fixed
     def encode_context(self, enc_mem: np.ndarray, ctx_len: int):
         mem = np.asarray(enc_mem, dtype=np.float64)[:ctx_len]
         hd = self.H * self.dh

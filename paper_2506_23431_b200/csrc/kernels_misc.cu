@@ -12,7 +12,7 @@ template <> __device__ __forceinline__ float from_f<float>(float v) { return v; 
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // ---------------------------------------------------------------------------------------------
-// Reset (Algorithm 1 lines 1-2 plus the admission of subsequence 1 at step 1): clears the
+// Reset (the initialisation of Algorithm 1 plus the admission of subsequence 1 at step 1): clears the
 // whole state block, then gives every sequence its first subsequence, first KV page and row.
 __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_t *ctx_len,
                                    const int32_t *forced_len, size_t state_words, int32_t *state_base, int phase) {

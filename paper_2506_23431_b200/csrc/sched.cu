@@ -1,8 +1,8 @@
 // Fused logits-argmax + scheduler.  One CTA per row scans the row's fp32 logits for the
 // greedy choice of Eq. 4 (ties to the lowest id); the CTA that finishes a sequence's last row
-// then runs that sequence's part of Algorithm 1 for the step: append the tokens (lines 9-11),
-// retire subsequences on eos/sep, the stop test (lines 12-13), the admission that lines 5-7
-// perform at the top of the next step, and the compaction of the active rows for it.  No CTA
+// then runs that sequence's part of Algorithm 1 for the step: append the tokens, retire
+// subsequences on eos/sep, the stop test, the admission that the loop performs at the top of
+// the next step, and the compaction of the active rows for it.  No CTA
 // ever waits for another: the hand-over is an atomic ticket after a memory fence.
 #include <limits.h>
 
@@ -16,71 +16,87 @@ __device__ __forceinline__ void better(float &bv, int &bi, float v, int i) {
   if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
 }
 
-__device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch, int b, const int32_t *teacher) {
+// One sequence's integer state for the step, staged in shared memory by the CTA that runs its
+// scheduler: the scheduler itself is one thread walking dependent loads, which on global memory
+// costs a round trip each; the CTA copies the arrays in (and the changed ones back out) with all
+// its threads instead.  Indices are local to the sequence: subsequence i at [i - 1], row c at [c].
+struct SeqStage {
+  int32_t *row_sub, *row_tok;                                        // [C]
+  int32_t *len, *forced_len, *state, *flag, *start, *last_tok, *teacher;   // [SM]
+  int32_t *page_table;                                               // [SM * PPS]
+  int4 *row_meta;                                                    // [C]
+  int4 *plist;                                                       // [SM * PPS]
+};
+__host__ __device__ inline size_t seq_stage_bytes(const Dims &dm) {
+  return ((size_t)(2 * dm.C + 7 * dm.SM + dm.SM * dm.PPS + 3) / 4 * 4) * sizeof(int32_t) + ((size_t)dm.C + (size_t)dm.SM * dm.PPS) * sizeof(int4);
+}
+
+// Algorithm 1 for one sequence and one step, after the step's tokens have been chosen: the append,
+// the retirement on eos/sep, the stop test, the admission the loop performs at the top of the next
+// step, and the compaction of the active rows for it.  Runs in one thread on the staged state.
+__device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqStage &v, int b, bool have_teacher) {
   const int t = st.hdr[HDR_STEP_T];
   const int C = dm.C, SM = dm.SM;
   int nact = st.n_active[b];
   int k = st.k[b];
-  for (int c = 0; c < C; ++c) st.prev_row_sub[b * C + c] = st.row_sub[b * C + c];
   if (st.done[b] || st.hdr[HDR_STATUS] != 0) {
     if (!st.done[b]) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
-    for (int c = 0; c < C; ++c) { st.row_sub[b * C + c] = 0; st.row_meta[b * C + c] = make_int4(0, 0, 0, 0); }
+    for (int c = 0; c < C; ++c) { v.row_sub[c] = 0; v.row_meta[c] = make_int4(0, 0, 0, 0); }
     st.n_active[b] = 0;
     st.plist_n[b] = 0;
     return;
   }
   // traffic counters of the step just executed (before any length changes)
   int i_max = 0;
-  for (int c = 0; c < nact; ++c) i_max = max(i_max, st.row_sub[b * C + c]);
+  for (int c = 0; c < nact; ++c) i_max = max(i_max, v.row_sub[c]);
   unsigned long long nvis = 0;
-  for (int i = 1; i <= i_max; ++i) nvis += (unsigned long long)(st.len[b * SM + i - 1] + 1);
+  for (int i = 1; i <= i_max; ++i) nvis += (unsigned long long)(v.len[i - 1] + 1);
   atomicAdd(&st.stats[PD_STAT_SELF_ENTRIES], nvis);
   if (nact > 0) atomicAdd(&st.stats[PD_STAT_CROSS_KEYS], (unsigned long long)st.ctx_len[b]);
   atomicAdd(&st.stats[PD_STAT_TOKENS], (unsigned long long)nact);
 
   unsigned long long mask = 0ull;
   for (int c = 0; c < nact; ++c) {
-    const int i = st.row_sub[b * C + c];
+    const int i = v.row_sub[c];
     const int sidx = b * SM + i - 1;
-    const int len = st.len[sidx];
-    const int fl = st.forced_len[sidx];
-    int own = __ldcg(&st.row_tok[b * C + c]);
+    const int len = v.len[i - 1];
+    const int fl = v.forced_len[i - 1];
+    int own = v.row_tok[c];
     if (fl >= 0) { if (len >= fl) own = dm.sep; }
     else if (len >= dm.MSL) own = dm.sep;
     st.chosen[(size_t)sidx * (dm.MSL + 1) + len] = own;
     int tok = own;
-    if (teacher != nullptr) { int tt = teacher[sidx]; if (tt >= 0) tok = tt; }
-    if (len >= dm.MSL) { tok = dm.sep; if (fl < 0) st.flag[sidx] |= PD_FLAG_CAPPED; }
+    if (have_teacher) { int tt = v.teacher[i - 1]; if (tt >= 0) tok = tt; }
+    if (len >= dm.MSL) { tok = dm.sep; if (fl < 0) v.flag[i - 1] |= PD_FLAG_CAPPED; }
     if (tok == dm.eos || tok == dm.sep) {
-      st.state[sidx] = SUB_ENDED;
-      st.flag[sidx] |= PD_FLAG_COMPLETE;
+      v.state[i - 1] = SUB_ENDED;
+      v.flag[i - 1] |= PD_FLAG_COMPLETE;
     } else {
       st.tokens[(size_t)sidx * dm.MSL + len] = tok;
-      st.len[sidx] = len + 1;
-      st.last_tok[sidx] = tok;
+      v.len[i - 1] = len + 1;
+      v.last_tok[i - 1] = tok;
     }
     mask |= 1ull << (i - 1);
   }
   st.trace[(size_t)(t - 1) * dm.B + b] = mask;
 
   int ended = 0;
-  for (int i = 1; i <= k; ++i) ended += st.state[b * SM + i - 1] == SUB_ENDED;
+  for (int i = 1; i <= k; ++i) ended += v.state[i - 1] == SUB_ENDED;
   bool done = false;
   if (ended == k) {
     done = true;                                   // every subsequence has produced its terminator
   } else if (t >= dm.T) {
     done = true;                                   // time_max reached with subsequences still open
     for (int i = 1; i <= k; ++i)
-      if (st.state[b * SM + i - 1] == SUB_ACTIVE) st.flag[b * SM + i - 1] |= PD_FLAG_TRUNCATED;
+      if (v.state[i - 1] == SUB_ACTIVE) v.flag[i - 1] |= PD_FLAG_TRUNCATED;
   } else if (t % dm.dt == 0 && k < SM) {           // step t+1 satisfies (t+1-1) mod delta_t == 0
-    const int sidx = b * SM + k;
     k += 1;
     st.k[b] = k;
-    st.start[sidx] = t + 1;
-    st.len[sidx] = 0;
-    st.state[sidx] = SUB_ACTIVE;
-    st.flag[sidx] = 0;
-    st.last_tok[sidx] = dm.bos;
+    v.start[k - 1] = t + 1;
+    v.len[k - 1] = 0;
+    v.state[k - 1] = SUB_ACTIVE;
+    v.flag[k - 1] = 0;
+    v.last_tok[k - 1] = dm.bos;
   }
   int n = 0;
   if (done) {
@@ -89,22 +105,21 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
     atomicAdd(&st.hdr[HDR_N_DONE], 1);
   } else {
     for (int i = 1; i <= k; ++i) {
-      const int sidx = b * SM + i - 1;
-      if (st.state[sidx] != SUB_ACTIVE) continue;
+      if (v.state[i - 1] != SUB_ACTIVE) continue;
       if (n >= C) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_STATE); break; }
-      const int p = st.len[sidx];                  // entry the next step will write
+      const int p = v.len[i - 1];                  // entry the next step will write
       if (p % dm.P == 0) {
         int pg = atomicAdd(&st.hdr[HDR_PAGE_BUMP], 1);
         if (pg >= dm.pool) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_POOL_EXHAUSTED); pg = 0; }
-        st.page_table[(size_t)sidx * dm.PPS + p / dm.P] = pg;
+        v.page_table[(i - 1) * dm.PPS + p / dm.P] = pg;
         atomicAdd(&st.stats[PD_STAT_PAGES], 1ull);
       }
       // where the append kernels of the coming step put this row's key/value, and its position tau + i
-      st.row_meta[b * C + n] = make_int4(st.page_table[(size_t)sidx * dm.PPS + p / dm.P], p % dm.P, st.start[sidx] - 1 + p + i, i);
-      st.row_sub[b * C + n++] = i;
+      v.row_meta[n] = make_int4(v.page_table[(i - 1) * dm.PPS + p / dm.P], p % dm.P, v.start[i - 1] - 1 + p + i, i);
+      v.row_sub[n++] = i;
     }
   }
-  for (int c = n; c < C; ++c) { st.row_sub[b * C + c] = 0; st.row_meta[b * C + c] = make_int4(0, 0, 0, 0); }
+  for (int c = n; c < C; ++c) { v.row_sub[c] = 0; v.row_meta[c] = make_int4(0, 0, 0, 0); }
   st.n_active[b] = n;
   // Page list of the coming step for the self-attention kernels: every page of subsequences
   // 1..i_max (i_max = last active one; later ones are invisible to every row), with the number
@@ -114,34 +129,72 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, int batch,
   // at position t + i; a kernel adds the query's i and subtracts the key's offset in the page).
   int np = 0;
   if (n > 0) {
-    const int i_max = st.row_sub[b * C + n - 1];
-    int4 *pl = st.plist + (size_t)b * SM * dm.PPS;
-    for (int i = 1; i <= i_max; ++i) {
-      const int sidx = b * SM + i - 1;
-      const int entries = st.len[sidx] + 1;
-      const int pos0 = st.start[sidx] - 1 + i;
+    const int i_last = v.row_sub[n - 1];
+    for (int i = 1; i <= i_last; ++i) {
+      const int entries = v.len[i - 1] + 1;
+      const int pos0 = v.start[i - 1] - 1 + i;
       for (int j = 0; j * dm.P < entries; ++j)
-        pl[np++] = make_int4(st.page_table[(size_t)sidx * dm.PPS + j], min(dm.P, entries - j * dm.P), i, t - (pos0 + j * dm.P));
+        v.plist[np++] = make_int4(v.page_table[(i - 1) * dm.PPS + j], min(dm.P, entries - j * dm.P), i, t - (pos0 + j * dm.P));
     }
   }
   st.plist_n[b] = np;
 }
 
 // Called by every thread of a row's CTA once the row's choice is in row_tok: the CTA that arrives
-// last for its sequence runs the sequence's scheduler, the last sequence advances the step.
+// last for its sequence stages the sequence's state, runs its scheduler and writes the state back;
+// the last sequence advances the step.  No CTA ever waits for another.
 __device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, const int32_t *teacher, int *is_last) {
-  const int tid = threadIdx.x;
+  extern __shared__ __align__(16) uint8_t sched_smem[];
+  const int tid = threadIdx.x, nthr = blockDim.x;
   if (tid == 0) {
     __threadfence();
     int ticket = atomicAdd(&st.seq_ticket[b], 1);
     *is_last = ticket == dm.C - 1;
   }
   __syncthreads();
-  if (!*is_last || tid != 0) return;
+  if (!*is_last) return;
   __threadfence();
-  st.seq_ticket[b] = 0;
-  schedule_sequence(dm, st, batch, b, teacher);
+  const int C = dm.C, SM = dm.SM, NPT = dm.SM * dm.PPS;
+  SeqStage v;
+  int32_t *w = reinterpret_cast<int32_t *>(sched_smem);
+  v.row_sub = w; w += C;
+  v.row_tok = w; w += C;
+  v.len = w; w += SM; v.forced_len = w; w += SM; v.state = w; w += SM; v.flag = w; w += SM;
+  v.start = w; w += SM; v.last_tok = w; w += SM; v.teacher = w; w += SM;
+  v.page_table = w; w += NPT;
+  w = reinterpret_cast<int32_t *>(sched_smem) + (size_t)(2 * C + 7 * SM + NPT + 3) / 4 * 4;     // 16-byte aligned
+  v.row_meta = reinterpret_cast<int4 *>(w);
+  v.plist = v.row_meta + C;
+  for (int c = tid; c < C; c += nthr) {
+    v.row_sub[c] = st.row_sub[b * C + c];
+    v.row_tok[c] = __ldcg(&st.row_tok[b * C + c]);            // written by other CTAs of this launch
+    st.prev_row_sub[b * C + c] = v.row_sub[c];
+  }
+  for (int i = tid; i < SM; i += nthr) {
+    const int sidx = b * SM + i;
+    v.len[i] = st.len[sidx]; v.forced_len[i] = st.forced_len[sidx]; v.state[i] = st.state[sidx]; v.flag[i] = st.flag[sidx];
+    v.start[i] = st.start[sidx]; v.last_tok[i] = st.last_tok[sidx];
+    v.teacher[i] = teacher != nullptr ? teacher[sidx] : -1;
+  }
+  for (int i = tid; i < NPT; i += nthr) v.page_table[i] = st.page_table[(size_t)b * NPT + i];
+  __syncthreads();
+  if (tid == 0) {
+    st.seq_ticket[b] = 0;
+    schedule_sequence(dm, st, v, b, teacher != nullptr);
+  }
+  __syncthreads();
+  for (int c = tid; c < C; c += nthr) { st.row_sub[b * C + c] = v.row_sub[c]; st.row_meta[b * C + c] = v.row_meta[c]; }
+  for (int i = tid; i < SM; i += nthr) {
+    const int sidx = b * SM + i;
+    st.len[sidx] = v.len[i]; st.state[sidx] = v.state[i]; st.flag[sidx] = v.flag[i]; st.start[sidx] = v.start[i];
+    st.last_tok[sidx] = v.last_tok[i];
+  }
+  for (int i = tid; i < NPT; i += nthr) st.page_table[(size_t)b * NPT + i] = v.page_table[i];
+  const int np = st.plist_n[b];                        // written by thread 0 before the barrier above
+  for (int i = tid; i < np; i += nthr) st.plist[(size_t)b * NPT + i] = v.plist[i];
   __threadfence();
+  __syncthreads();
+  if (tid != 0) return;
   if (atomicAdd(&st.hdr[HDR_TICKET], 1) == batch - 1) {   // last sequence of the step
     __threadfence();
     st.hdr[HDR_TICKET] = 0;
@@ -213,7 +266,7 @@ __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, 
 
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
                                 const int32_t *teacher, cudaStream_t s) {
-  argmax_sched_kernel<<<batch * dm.C, AT, 0, s>>>(dm, st, batch, logits, teacher);
+  argmax_sched_kernel<<<batch * dm.C, AT, seq_stage_bytes(dm), s>>>(dm, st, batch, logits, teacher);
   return cudaGetLastError();
 }
 
@@ -261,7 +314,7 @@ __global__ void __launch_bounds__(PT) pick_sched_kernel(Dims dm, DecState st, in
 
 cudaError_t launch_pick_sched(const Dims &dm, const DecState &st, int batch, int tiles, const float *part_val,
                               const int32_t *part_idx, const float *term_val, const int32_t *teacher, cudaStream_t s) {
-  pick_sched_kernel<<<batch * dm.C, PT, 0, s>>>(dm, st, batch, tiles, batch * dm.C, part_val, part_idx, term_val, teacher);
+  pick_sched_kernel<<<batch * dm.C, PT, seq_stage_bytes(dm), s>>>(dm, st, batch, tiles, batch * dm.C, part_val, part_idx, term_val, teacher);
   return cudaGetLastError();
 }
 
