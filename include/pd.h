@@ -149,9 +149,11 @@ PD_API pd_status pd_done(pd_handle *h, int32_t *all_done);
 PD_API pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags,
                      int32_t *steps);
 
-/* Whole Algorithm 1 from host buffers: copies enc_mem (host [batch, max_ctx, d_model], dtype)
- * to the device, encodes, decodes until done, copies the streams back.  Output arguments as
- * in pd_collect.  Synchronises. */
+/* Whole Algorithm 1 from host buffers: copies enc_mem (host [batch, max_ctx, d_model], dtype;
+ * pinned memory lets the copy overlap) to the device in chunks of sequences on a copy stream of
+ * the handle's own while the context projection of the chunks already there runs on the handle's
+ * stream, decodes until done, copies the streams back.  Output arguments as in pd_collect.
+ * Synchronises. */
 PD_API pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t *ctx_len, int32_t batch,
                            const int32_t *forced_len, int32_t *tokens, int32_t *lens, int32_t *n_sub,
                            int32_t *flags, int32_t *steps);

@@ -269,7 +269,7 @@ cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int lay
 // ---------------------------------------------------------------------------------------------
 // The context projection writes [position][k of all heads | v of all heads]; the attention
 // kernels read head-major blocks.  One 16-byte chunk per thread and iteration.
-__global__ void ctx_kv_relayout_kernel(Dims dm, int batch, int layer, int esize, const uint4 *__restrict__ proj,
+__global__ void ctx_kv_relayout_kernel(Dims dm, int b0, int batch, int layer, int esize, const uint4 *__restrict__ proj,
                                        uint4 *__restrict__ kv_c) {
   const int cpr = kDh * esize / 16;                        // 16-byte chunks of one head's row
   const size_t per_pos = (size_t)2 * dm.H * cpr;           // chunks of one projected position
@@ -280,15 +280,16 @@ __global__ void ctx_kv_relayout_kernel(Dims dm, int batch, int layer, int esize,
     const int is_v = (int)((i / ((size_t)cpr * dm.H)) % 2);
     const size_t bp = i / per_pos;
     const int pos = (int)(bp % dm.ctx), b = (int)(bp / dm.ctx);
-    const size_t dst = (ctx_kv_offset(layer, dm.B, b, dm.H, h, is_v, dm.ctx) + (size_t)pos * kDh) * esize / 16 + c;
+    const size_t dst = (ctx_kv_offset(layer, dm.B, b0 + b, dm.H, h, is_v, dm.ctx) + (size_t)pos * kDh) * esize / 16 + c;
     kv_c[dst] = proj[i];
   }
 }
 
-cudaError_t launch_ctx_kv_relayout(const Dims &dm, int batch, int layer, int dtype, const void *proj, void *kv_c,
+// proj holds the projections of sequences b0 .. b0 + batch - 1.
+cudaError_t launch_ctx_kv_relayout(const Dims &dm, int b0, int batch, int layer, int dtype, const void *proj, void *kv_c,
                                    cudaStream_t s) {
   const int esize = dtype == PD_DTYPE_BF16 ? 2 : 4;
-  ctx_kv_relayout_kernel<<<148 * 8, 256, 0, s>>>(dm, batch, layer, esize, (const uint4 *)proj, (uint4 *)kv_c);
+  ctx_kv_relayout_kernel<<<148 * 8, 256, 0, s>>>(dm, b0, batch, layer, esize, (const uint4 *)proj, (uint4 *)kv_c);
   return cudaGetLastError();
 }
 

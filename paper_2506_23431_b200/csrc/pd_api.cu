@@ -150,6 +150,11 @@ struct pd_handle {
   bool have_tmap = false;
   CUtensorMap vmap_a, vmap_b;      // hidden rows and lm_head for the tcgen05 vocabulary projection
   bool vocab_tc = false;
+  // pd_generate_host: host-to-device copies of the encoder memory run on a stream of their own, in
+  // chunks of sequences, so that the context projection of one chunk overlaps the copy of the next
+  static constexpr int kMaxChunks = 8;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_entry = nullptr, ev_chunk[kMaxChunks] = {};
   int batch = 0;
   bool encoded = false;
   int self_splits = 1, cross_splits = 1;
@@ -407,6 +412,9 @@ pd_status device_status(pd_handle *h) {
   return PD_OK;
 }
 
+pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, const int32_t *forced_len);
+pd_status encode_project(pd_handle *h, const void *enc_mem, int b0, int nb);
+
 }  // namespace
 
 extern "C" {
@@ -445,6 +453,10 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   if (cublasSetWorkspace(h->blas, h->ptr<void>(h->lay.cublas_ws), kCublasWs) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
   if (cublasSetMathMode(h->blas, CUBLAS_DEFAULT_MATH) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
   if (cudaHostAlloc((void **)&h->pinned_flag, 64, cudaHostAllocDefault) != cudaSuccess) return bail(PD_ERR_CUDA);
+  if (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_entry, cudaEventDisableTiming) != cudaSuccess) return bail(PD_ERR_CUDA);
+  for (int c = 0; c < pd_handle::kMaxChunks; ++c)
+    if (cudaEventCreateWithFlags(&h->ev_chunk[c], cudaEventDisableTiming) != cudaSuccess) return bail(PD_ERR_CUDA);
 
   int32_t *sb = h->ptr<int32_t>(h->lay.state);
   const Layout &L = h->lay;
@@ -500,7 +512,21 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
 pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ctx_len, int32_t batch,
                             const int32_t *forced_len) {
   if (!h) return PD_ERR_ARG;
-  if (!enc_mem || !ctx_len || batch < 1 || batch > h->dm.B) return fail(h, PD_ERR_ARG, "pd_encode_context: bad argument");
+  if (!enc_mem) return fail(h, PD_ERR_ARG, "pd_encode_context: bad argument");
+  PD_TRY(encode_prepare(h, ctx_len, batch, forced_len));
+  PD_TRY(encode_project(h, enc_mem, 0, batch));
+  h->encoded = true;
+  h->steps_enqueued = 0;
+  return PD_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+// Everything of pd_encode_context but the projections: argument checks, split factors, state reset.
+pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, const int32_t *forced_len) {
+  if (!ctx_len || batch < 1 || batch > h->dm.B) return fail(h, PD_ERR_ARG, "pd_encode_context: bad argument");
   const Dims &dm = h->dm;
   for (int b = 0; b < batch; ++b)
     if (ctx_len[b] < 1 || ctx_len[b] > dm.ctx) return fail(h, PD_ERR_ARG, "pd_encode_context: ctx_len out of range");
@@ -540,16 +566,26 @@ pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ct
                                            forced_len ? h->ptr<int32_t>(L.forced_in) : nullptr, L.state_words,
                                            h->ptr<int32_t>(L.state), s));
   h->own_launches++;   // the reset is two launches
-  const size_t e = h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4;
-  for (int l = 0; l < dm.L; ++l) {
-    PD_TRY(gemm(h, false, batch * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5],
-                h->ptr<void>(L.proj_stage), false, 0.f));
-    OWN(h, PD_PROF_OTHER, launch_ctx_kv_relayout(dm, batch, l, h->cfg.dtype, h->ptr<void>(L.proj_stage), h->ptr<void>(L.kv_c), s));
-  }
-  h->encoded = true;
-  h->steps_enqueued = 0;
   return PD_OK;
 }
+
+// Cross-attention keys/values of every layer for sequences b0 .. b0 + nb - 1, whose encoder memory
+// starts at enc_mem (device, [nb, max_ctx, d]).
+pd_status encode_project(pd_handle *h, const void *enc_mem, int b0, int nb) {
+  const Dims &dm = h->dm;
+  const Layout &L = h->lay;
+  for (int l = 0; l < dm.L; ++l) {
+    PD_TRY(gemm(h, false, nb * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5],
+                h->ptr<void>(L.proj_stage), false, 0.f));
+    OWN(h, PD_PROF_OTHER, launch_ctx_kv_relayout(dm, b0, nb, l, h->cfg.dtype, h->ptr<void>(L.proj_stage), h->ptr<void>(L.kv_c), h->stream));
+  }
+  return PD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
 
 pd_status pd_step(pd_handle *h, const int32_t *teacher_tokens) {
   if (!h) return PD_ERR_ARG;
@@ -639,9 +675,31 @@ pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t
   if (batch < 1 || batch > h->dm.B) return fail(h, PD_ERR_ARG, "pd_generate_host: bad batch");
   const size_t e = h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4;
   CU_TRY(h, cudaSetDevice(h->cfg.device));
-  CU_TRY(h, cudaMemcpyAsync(h->ptr<void>(h->lay.enc_stage), enc_mem_host, (size_t)batch * h->dm.ctx * h->dm.d * e,
-                            cudaMemcpyHostToDevice, h->stream));
-  PD_TRY(pd_encode_context(h, h->ptr<void>(h->lay.enc_stage), ctx_len, batch, forced_len));
+  // Chunks of whole sequences, at least 16 MiB each: chunk c is projected on the handle's stream
+  // while chunk c + 1 is still crossing PCIe on the copy stream.
+  const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * e;
+  int n_chunks = (int)((size_t)batch * seq_bytes / ((size_t)16 << 20));
+  if (n_chunks > pd_handle::kMaxChunks) n_chunks = pd_handle::kMaxChunks;
+  if (n_chunks > batch) n_chunks = batch;
+  if (n_chunks < 1) n_chunks = 1;
+  CU_TRY(h, cudaEventRecord(h->ev_entry, h->stream));                  // the staging buffer is free once earlier work is done
+  CU_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_entry, 0));
+  uint8_t *stage = h->ptr<uint8_t>(h->lay.enc_stage);
+  const uint8_t *src = static_cast<const uint8_t *>(enc_mem_host);
+  for (int c = 0; c < n_chunks; ++c) {
+    const int b0 = (int)((long long)batch * c / n_chunks), b1 = (int)((long long)batch * (c + 1) / n_chunks);
+    CU_TRY(h, cudaMemcpyAsync(stage + b0 * seq_bytes, src + b0 * seq_bytes, (size_t)(b1 - b0) * seq_bytes, cudaMemcpyHostToDevice,
+                              h->copy_stream));
+    CU_TRY(h, cudaEventRecord(h->ev_chunk[c], h->copy_stream));
+  }
+  PD_TRY(encode_prepare(h, ctx_len, batch, forced_len));
+  for (int c = 0; c < n_chunks; ++c) {
+    const int b0 = (int)((long long)batch * c / n_chunks), b1 = (int)((long long)batch * (c + 1) / n_chunks);
+    CU_TRY(h, cudaStreamWaitEvent(h->stream, h->ev_chunk[c], 0));
+    PD_TRY(encode_project(h, stage + b0 * seq_bytes, b0, b1 - b0));
+  }
+  h->encoded = true;
+  h->steps_enqueued = 0;
   int32_t n = 0;
   PD_TRY(pd_run(h, 8, &n));
   return pd_collect(h, tokens, lens, n_sub, flags, steps);
@@ -789,6 +847,9 @@ void pd_destroy(pd_handle *h) {
   for (const ProfRec &r : h->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->pinned_flag) cudaFreeHost(h->pinned_flag);
+  for (cudaEvent_t e : h->ev_chunk) if (e) cudaEventDestroy(e);
+  if (h->ev_entry) cudaEventDestroy(h->ev_entry);
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   drop_ff_plan(h);
   if (h->lt) cublasLtDestroy(h->lt);
   if (h->blas) cublasDestroy(h->blas);
