@@ -60,7 +60,8 @@ enum { PD_FLAG_COMPLETE = 1, PD_FLAG_TRUNCATED = 2, PD_FLAG_CAPPED = 4 };
 /* intermediate buffers readable with pd_debug_read (values of the last layer of the last step) */
 enum {
   PD_BUF_X = 0,        /* residual stream after the last layer, fp32 [rows, d_model]          */
-  PD_BUF_QKV = 1,      /* self-attention projection, fp32 [rows, 3*d_model]                   */
+  PD_BUF_QKV = 1,      /* self-attention projection [rows, 3*d_model]: fp32, except bf16 on the
+                          bf16 path without rotary positions (the projection rounds itself)   */
   PD_BUF_SELF_OUT = 2, /* self-attention output, dtype [rows, d_model]                        */
   PD_BUF_CROSS_Q = 3,  /* cross-attention queries, dtype [rows, d_model]                      */
   PD_BUF_CROSS_OUT = 4,/* cross-attention output, dtype [rows, d_model]                       */

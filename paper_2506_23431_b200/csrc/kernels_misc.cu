@@ -225,6 +225,25 @@ cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s) {
 // pair.  Writes k and v to slot p of the subsequence's page list and q to the query buffer; in
 // RoPE mode q and k are rotated by the position first.  All rows of a step are appended before
 // any attends: tokens fed by earlier subsequences at the same step are visible (tau' <= t - 1).
+// The same step when q, k, v arrive already in the storage type (no rotation to apply, so the
+// projection's own epilogue did the one rounding): eight columns (16 bytes) per thread, pure copies.
+__global__ void append_copy_bf16_kernel(Dims dm, DecState st, int layer, const __nv_bfloat16 *__restrict__ qkv,
+                                        __nv_bfloat16 *__restrict__ q_out, __nv_bfloat16 *__restrict__ kv_pool) {
+  const int r = blockIdx.x;
+  const __nv_bfloat16 *row = qkv + (size_t)r * 3 * dm.d;
+  const int4 meta = st.row_meta[r];                 // (page, slot, position tau + i, subsequence i or 0)
+  const int col = 8 * threadIdx.x;                  // blockDim.x = d / 8; one 16-byte chunk of one head
+  const uint4 q = *reinterpret_cast<const uint4 *>(row + col);
+  const uint4 k = *reinterpret_cast<const uint4 *>(row + dm.d + col);
+  const uint4 v = *reinterpret_cast<const uint4 *>(row + 2 * dm.d + col);
+  if (meta.w <= 0) return;
+  const int h = col / kDh, dd = col % kDh;
+  __nv_bfloat16 *ko = kv_pool + kv_block_offset(layer, dm.pool, meta.x, dm.H, h, dm.P) + kv_entry_offset<__nv_bfloat16>(meta.y, dd, 0);
+  *reinterpret_cast<uint4 *>(q_out + (size_t)r * dm.d + col) = q;
+  *reinterpret_cast<uint4 *>(ko) = k;
+  *reinterpret_cast<uint4 *>(ko + kDh) = v;         // the value row follows the key row of the same entry
+}
+
 template <typename T>
 __global__ void append_kernel(Dims dm, DecState st, int layer, const float *__restrict__ qkv, T *__restrict__ q_out,
                               T *__restrict__ kv_pool, const float2 *__restrict__ rope_tab) {
@@ -252,6 +271,13 @@ __global__ void append_kernel(Dims dm, DecState st, int layer, const float *__re
   qo[0] = from_f<T>(q.x); qo[1] = from_f<T>(q.y); qo[2] = from_f<T>(q.z); qo[3] = from_f<T>(q.w);
   ko[0] = from_f<T>(k.x); ko[1] = from_f<T>(k.y); ko[2] = from_f<T>(k.z); ko[3] = from_f<T>(k.w);
   vo[0] = from_f<T>(v.x); vo[1] = from_f<T>(v.y); vo[2] = from_f<T>(v.z); vo[3] = from_f<T>(v.w);
+}
+
+cudaError_t launch_append_copy_bf16(const Dims &dm, const DecState &st, int batch, int layer, const void *qkv, void *q_out,
+                                    void *kv_pool, cudaStream_t s) {
+  append_copy_bf16_kernel<<<batch * dm.C, dm.d / 8, 0, s>>>(dm, st, layer, (const __nv_bfloat16 *)qkv, (__nv_bfloat16 *)q_out,
+                                                           (__nv_bfloat16 *)kv_pool);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,

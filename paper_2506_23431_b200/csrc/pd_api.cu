@@ -332,9 +332,16 @@ pd_status enqueue_step(pd_handle *h) {
   for (int l = 0; l < dm.L; ++l) {
     const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
     OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
-    PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, true, 0.f));
-    OWN(h, PD_PROF_APPEND, launch_append(dm, h->st, h->batch, l, dt, qkv, h->ptr<void>(h->lay.qbuf),
-                                         h->ptr<void>(h->lay.kv_pool), h->ptr<float2>(h->lay.rope_tab), s));
+    if (dt == PD_DTYPE_BF16 && dm.pos_mode != PD_POS_ROPE) {
+      // nothing to rotate: the projection rounds to bf16 itself and the append only places the rows
+      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, false, 0.f));
+      OWN(h, PD_PROF_APPEND, launch_append_copy_bf16(dm, h->st, h->batch, l, qkv, h->ptr<void>(h->lay.qbuf),
+                                                     h->ptr<void>(h->lay.kv_pool), s));
+    } else {
+      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, true, 0.f));
+      OWN(h, PD_PROF_APPEND, launch_append(dm, h->st, h->batch, l, dt, qkv, h->ptr<void>(h->lay.qbuf),
+                                           h->ptr<void>(h->lay.kv_pool), h->ptr<float2>(h->lay.rope_tab), s));
+    }
     {
       ProfScope ps(h, PD_PROF_SELF_ATTN);
       PD_TRY(enqueue_self_attention(h, l));

@@ -110,6 +110,8 @@ cudaError_t launch_rmsnorm_packed(const Dims &dm, const DecState &st, int batch,
 cudaError_t launch_relu(int dtype, void *buf, size_t n, cudaStream_t s);
 cudaError_t launch_append(const Dims &dm, const DecState &st, int batch, int layer, int dtype, const float *qkv,
                           void *q_out, void *kv_pool, const float2 *rope_tab, cudaStream_t s);
+cudaError_t launch_append_copy_bf16(const Dims &dm, const DecState &st, int batch, int layer, const void *qkv, void *q_out,
+                                    void *kv_pool, cudaStream_t s);
 cudaError_t launch_ctx_kv_relayout(const Dims &dm, int b0, int batch, int layer, int dtype, const void *proj, void *kv_c,
                                    cudaStream_t s);
 cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
