@@ -371,6 +371,16 @@ def main():
 
     roofline = roof("cross_attn", cross_bytes)
     roofline_self = roof("self_attn", self_bytes)
+    # the tensor-core vocabulary projection: lm_head once per launch plus the packed hidden rows; durations from
+    # the event pair around every launch of the profiled decode (these carry a few microseconds of idle time)
+    roofline_vocab = None
+    v_ms, v_n = prof.get("vocab", (0.0, 0))
+    if v_n > 0 and v_ms > 0:
+        v_bytes = (wl.vocab * d * e) * v_n + st_p["tokens"] * d * e
+        v_ach = v_bytes / (v_ms * 1e-3) / 1e9
+        roofline_vocab = {"bound": "hbm", "kernel": "vocab_tc", "achieved": v_ach, "peak": peak, "unit": "GB/s",
+                          "frac": v_ach / peak, "traffic": None, "launches": int(v_n), "event_bracketed_us": 1e3 * v_ms / v_n,
+                          "bytes_per_launch": v_bytes / v_n, "peak_source": peak_src}
     kernel_ms = {k: round(v[0], 4) for k, v in prof.items()}
 
     # ---- max over ranks
@@ -395,7 +405,8 @@ def main():
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": int(own_launches), "cublas_gemms": int(gemm_calls),
-            "roofline": roofline, "roofline_self_attn": roofline_self, "kernel_ms_per_decode": kernel_ms}
+            "roofline": roofline, "roofline_self_attn": roofline_self, "roofline_vocab": roofline_vocab,
+            "kernel_ms_per_decode": kernel_ms}
 
     if rank == 0 and world == 1 and args.sequential:
         # the same targets decoded by the ordinary sequential decoder (sub_max = 1) with the same library

@@ -190,7 +190,7 @@ PD_API pd_status pd_reset_counters(pd_handle *h);
  * pd_profile_read sums them up (synchronises): for kind k in PD_PROF_*, ms[k] = total device
  * time, launches[k] = launches.  Arrays of PD_PROF_COUNT entries. */
 enum { PD_PROF_APPEND = 0, PD_PROF_SELF_ATTN = 1, PD_PROF_CROSS_ATTN = 2, PD_PROF_ARGMAX_SCHED = 3,
-       PD_PROF_GEMM = 4, PD_PROF_OTHER = 5, PD_PROF_COUNT = 6 };
+       PD_PROF_GEMM = 4, PD_PROF_OTHER = 5, PD_PROF_VOCAB = 6 /* tensor-core vocabulary projection */, PD_PROF_COUNT = 7 };
 PD_API pd_status pd_profile_enable(pd_handle *h, int32_t on);
 PD_API pd_status pd_profile_read(pd_handle *h, double *ms, int64_t *launches);
 

@@ -24,7 +24,7 @@ PD_DTYPE_FP32, PD_DTYPE_BF16 = 0, 1
 PD_POS_T5_BIAS, PD_POS_ROPE = 0, 1
 PD_FLAG_COMPLETE, PD_FLAG_TRUNCATED, PD_FLAG_CAPPED = 1, 2, 4
 PD_BUF_X, PD_BUF_QKV, PD_BUF_SELF_OUT, PD_BUF_CROSS_Q, PD_BUF_CROSS_OUT, PD_BUF_STATE = range(6)
-PD_PROF_NAMES = ["append", "self_attn", "cross_attn", "argmax_sched", "gemm", "other"]
+PD_PROF_NAMES = ["append", "self_attn", "cross_attn", "argmax_sched", "gemm", "other", "vocab"]
 PD_STAT_TOKENS, PD_STAT_STEPS, PD_STAT_SELF_ENTRIES, PD_STAT_CROSS_KEYS, PD_STAT_PAGES = range(5)
 PD_STAT_COUNT = 8
 LAYER_TENSORS = ["norm1", "wqkv", "wo", "norm2", "wq_c", "wkv_c", "wo_c", "norm3", "w1", "w2"]

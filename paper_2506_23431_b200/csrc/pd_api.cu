@@ -378,7 +378,7 @@ pd_status enqueue_step(pd_handle *h) {
     va.logits = h->cfg.store_logits ? logits : nullptr;
     va.status = h->st.hdr + HDR_STATUS;
     OWN(h, PD_PROF_OTHER, launch_rmsnorm_packed(dm, h->st, h->batch, dt, x, h->w.final_norm, hb, s));
-    OWN(h, PD_PROF_ARGMAX_SCHED, launch_vocab_tc(h->vmap_a, h->vmap_b, va, s));
+    OWN(h, PD_PROF_VOCAB, launch_vocab_tc(h->vmap_a, h->vmap_b, va, s));
     OWN(h, PD_PROF_ARGMAX_SCHED, launch_pick_sched(dm, h->st, h->batch, vocab_tc_tiles(dm.V), va.part_val, va.part_idx, va.term_val,
                                                    h->ptr<int32_t>(h->lay.teacher), s));
     return PD_OK;
