@@ -31,32 +31,86 @@ __host__ __device__ inline size_t seq_stage_bytes(const Dims &dm) {
   return ((size_t)(2 * dm.C + 7 * dm.SM + dm.SM * dm.PPS + 3) / 4 * 4) * sizeof(int32_t) + ((size_t)dm.C + (size_t)dm.SM * dm.PPS) * sizeof(int4);
 }
 
+// Scalars of the sequence that only its own scheduler changes, read at the top of the kernel.
+struct SeqScalars { int t, nact, k, done, status; };
+
+__device__ __forceinline__ SeqStage seq_stage_views(const Dims &dm, uint8_t *smem) {
+  const int C = dm.C, SM = dm.SM, NPT = dm.SM * dm.PPS;
+  SeqStage v;
+  int32_t *w = reinterpret_cast<int32_t *>(smem);
+  v.row_sub = w; w += C;
+  v.row_tok = w; w += C;
+  v.len = w; w += SM; v.forced_len = w; w += SM; v.state = w; w += SM; v.flag = w; w += SM;
+  v.start = w; w += SM; v.last_tok = w; w += SM; v.teacher = w; w += SM;
+  v.page_table = w; w += NPT;
+  w = reinterpret_cast<int32_t *>(smem) + (size_t)(2 * C + 7 * SM + NPT + 3) / 4 * 4;     // 16-byte aligned
+  v.row_meta = reinterpret_cast<int4 *>(w);
+  v.plist = v.row_meta + C;
+  return v;
+}
+
+// Every CTA of a sequence copies the sequence's state in at its very top, while its own row's loads
+// are in flight (nothing of it changes during the launch except row_tok, which the CTA that ends up
+// running the scheduler fetches afterwards): the copy is then off the critical path.
+__device__ __forceinline__ SeqScalars stage_in(const Dims &dm, const DecState &st, int b, const int32_t *teacher, const SeqStage &v) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int C = dm.C, SM = dm.SM, NPT = dm.SM * dm.PPS;
+  SeqScalars sc;
+  sc.t = st.hdr[HDR_STEP_T]; sc.nact = st.n_active[b]; sc.k = st.k[b]; sc.done = st.done[b]; sc.status = st.hdr[HDR_STATUS];
+  for (int c = tid; c < C; c += nthr) v.row_sub[c] = st.row_sub[b * C + c];
+  for (int i = tid; i < SM; i += nthr) {
+    const int sidx = b * SM + i;
+    v.len[i] = st.len[sidx]; v.forced_len[i] = st.forced_len[sidx]; v.state[i] = st.state[sidx]; v.flag[i] = st.flag[sidx];
+    v.start[i] = st.start[sidx]; v.last_tok[i] = st.last_tok[sidx];
+    v.teacher[i] = teacher != nullptr ? teacher[sidx] : -1;
+  }
+  for (int i = tid; i < NPT; i += nthr) v.page_table[i] = st.page_table[(size_t)b * NPT + i];
+  return sc;
+}
+
+__device__ __forceinline__ int warp_sum(int x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
 // Algorithm 1 for one sequence and one step, after the step's tokens have been chosen: the append,
 // the retirement on eos/sep, the stop test, the admission the loop performs at the top of the next
-// step, and the compaction of the active rows for it.  Runs in one thread on the staged state.
-__device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqStage &v, int b, bool have_teacher) {
-  const int t = st.hdr[HDR_STEP_T];
-  const int C = dm.C, SM = dm.SM;
-  int nact = st.n_active[b];
-  int k = st.k[b];
-  if (st.done[b] || st.hdr[HDR_STATUS] != 0) {
-    if (!st.done[b]) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
-    for (int c = 0; c < C; ++c) { v.row_sub[c] = 0; v.row_meta[c] = make_int4(0, 0, 0, 0); }
-    st.n_active[b] = 0;
-    st.plist_n[b] = 0;
+// step, and the compaction of the active rows for it.  Runs in one warp on the staged state: lanes
+// take rows, then subsequences; order-dependent results (row order, page ids, page-list offsets) come
+// from ballots and prefix sums, so they equal what a loop over increasing i would give.
+__device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqStage &v, int b, bool have_teacher, const SeqScalars &sc) {
+  const unsigned FULL = 0xffffffffu;
+  const int lane = threadIdx.x & 31;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  const int t = sc.t;
+  const int C = dm.C, SM = dm.SM, P = dm.P;
+  const int nact = sc.nact;
+  int k = sc.k;
+  if (sc.done || sc.status != 0) {
+    if (lane == 0 && !sc.done) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
+    for (int c = lane; c < C; c += 32) { v.row_sub[c] = 0; v.row_meta[c] = make_int4(0, 0, 0, 0); }
+    if (lane == 0) { st.n_active[b] = 0; st.plist_n[b] = 0; }
     return;
   }
   // traffic counters of the step just executed (before any length changes)
   int i_max = 0;
-  for (int c = 0; c < nact; ++c) i_max = max(i_max, v.row_sub[c]);
-  unsigned long long nvis = 0;
-  for (int i = 1; i <= i_max; ++i) nvis += (unsigned long long)(v.len[i - 1] + 1);
-  atomicAdd(&st.stats[PD_STAT_SELF_ENTRIES], nvis);
-  if (nact > 0) atomicAdd(&st.stats[PD_STAT_CROSS_KEYS], (unsigned long long)st.ctx_len[b]);
-  atomicAdd(&st.stats[PD_STAT_TOKENS], (unsigned long long)nact);
+  for (int c = lane; c < nact; c += 32) i_max = max(i_max, v.row_sub[c]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) i_max = max(i_max, __shfl_xor_sync(FULL, i_max, o));
+  int nvis = 0;
+  for (int i = lane + 1; i <= i_max; i += 32) nvis += v.len[i - 1] + 1;
+  nvis = warp_sum(nvis);
+  if (lane == 0) {
+    atomicAdd(&st.stats[PD_STAT_SELF_ENTRIES], (unsigned long long)nvis);
+    if (nact > 0) atomicAdd(&st.stats[PD_STAT_CROSS_KEYS], (unsigned long long)st.ctx_len[b]);
+    atomicAdd(&st.stats[PD_STAT_TOKENS], (unsigned long long)nact);
+  }
+  __syncwarp();
 
-  unsigned long long mask = 0ull;
-  for (int c = 0; c < nact; ++c) {
+  // ---- the step's tokens: one row per lane (every row belongs to a different subsequence)
+  unsigned mask_lo = 0u, mask_hi = 0u;
+  for (int c = lane; c < nact; c += 32) {
     const int i = v.row_sub[c];
     const int sidx = b * SM + i - 1;
     const int len = v.len[i - 1];
@@ -76,51 +130,79 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqS
       v.len[i - 1] = len + 1;
       v.last_tok[i - 1] = tok;
     }
-    mask |= 1ull << (i - 1);
+    if (i <= 32) mask_lo |= 1u << (i - 1); else mask_hi |= 1u << (i - 33);
   }
-  st.trace[(size_t)(t - 1) * dm.B + b] = mask;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { mask_lo |= __shfl_xor_sync(FULL, mask_lo, o); mask_hi |= __shfl_xor_sync(FULL, mask_hi, o); }
+  if (lane == 0) st.trace[(size_t)(t - 1) * dm.B + b] = ((unsigned long long)mask_hi << 32) | mask_lo;
+  __syncwarp();
 
+  // ---- stop test, time limit, admission
   int ended = 0;
-  for (int i = 1; i <= k; ++i) ended += v.state[i - 1] == SUB_ENDED;
+  for (int i = lane + 1; i <= k; i += 32) ended += v.state[i - 1] == SUB_ENDED;
+  ended = warp_sum(ended);
   bool done = false;
   if (ended == k) {
     done = true;                                   // every subsequence has produced its terminator
   } else if (t >= dm.T) {
     done = true;                                   // time_max reached with subsequences still open
-    for (int i = 1; i <= k; ++i)
+    for (int i = lane + 1; i <= k; i += 32)
       if (v.state[i - 1] == SUB_ACTIVE) v.flag[i - 1] |= PD_FLAG_TRUNCATED;
   } else if (t % dm.dt == 0 && k < SM) {           // step t+1 satisfies (t+1-1) mod delta_t == 0
+    if (lane == 0) {
+      st.k[b] = k + 1;
+      v.start[k] = t + 1;
+      v.len[k] = 0;
+      v.state[k] = SUB_ACTIVE;
+      v.flag[k] = 0;
+      v.last_tok[k] = dm.bos;
+    }
     k += 1;
-    st.k[b] = k;
-    v.start[k - 1] = t + 1;
-    v.len[k - 1] = 0;
-    v.state[k - 1] = SUB_ACTIVE;
-    v.flag[k - 1] = 0;
-    v.last_tok[k - 1] = dm.bos;
   }
+  __syncwarp();
+
+  // ---- rows of the coming step: the active subsequences in increasing i
   int n = 0;
   if (done) {
-    st.done[b] = 1;
-    st.steps[b] = t;
-    atomicAdd(&st.hdr[HDR_N_DONE], 1);
+    if (lane == 0) { st.done[b] = 1; st.steps[b] = t; atomicAdd(&st.hdr[HDR_N_DONE], 1); }
   } else {
-    for (int i = 1; i <= k; ++i) {
-      if (v.state[i - 1] != SUB_ACTIVE) continue;
-      if (n >= C) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_STATE); break; }
-      const int p = v.len[i - 1];                  // entry the next step will write
-      if (p % dm.P == 0) {
-        int pg = atomicAdd(&st.hdr[HDR_PAGE_BUMP], 1);
-        if (pg >= dm.pool) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_POOL_EXHAUSTED); pg = 0; }
-        v.page_table[(i - 1) * dm.PPS + p / dm.P] = pg;
-        atomicAdd(&st.stats[PD_STAT_PAGES], 1ull);
+    int pages = 0;
+    for (int i0 = 0; i0 < k; i0 += 32) {
+      const int i = i0 + lane + 1;
+      const bool on = i <= k && v.state[i - 1] == SUB_ACTIVE;
+      const unsigned bal = __ballot_sync(FULL, on);
+      const int my_n = n + __popc(bal & lt_mask);
+      const int p = on ? v.len[i - 1] : 0;                       // entry the next step will write
+      const bool need = on && my_n < C && p % P == 0;            // it opens a new page
+      const unsigned nb = __ballot_sync(FULL, need);
+      int pg0 = 0;
+      if (nb != 0u) {
+        if (lane == 0) pg0 = atomicAdd(&st.hdr[HDR_PAGE_BUMP], __popc(nb));
+        pg0 = __shfl_sync(FULL, pg0, 0);
+        pages += __popc(nb);
       }
-      // where the append kernels of the coming step put this row's key/value, and its position tau + i
-      v.row_meta[n] = make_int4(v.page_table[(i - 1) * dm.PPS + p / dm.P], p % dm.P, v.start[i - 1] - 1 + p + i, i);
-      v.row_sub[n++] = i;
+      if (on) {
+        if (my_n >= C) {
+          atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_STATE);
+        } else {
+          if (need) {
+            int pg = pg0 + __popc(nb & lt_mask);
+            if (pg >= dm.pool) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_POOL_EXHAUSTED); pg = 0; }
+            v.page_table[(i - 1) * dm.PPS + p / P] = pg;
+          }
+          // where the append kernels of the coming step put this row's key/value, and its position tau + i
+          v.row_meta[my_n] = make_int4(v.page_table[(i - 1) * dm.PPS + p / P], p % P, v.start[i - 1] - 1 + p + i, i);
+          v.row_sub[my_n] = i;
+        }
+      }
+      n += __popc(bal);
     }
+    if (n > C) n = C;
+    if (lane == 0 && pages > 0) atomicAdd(&st.stats[PD_STAT_PAGES], (unsigned long long)pages);
   }
-  for (int c = n; c < C; ++c) { v.row_sub[c] = 0; v.row_meta[c] = make_int4(0, 0, 0, 0); }
-  st.n_active[b] = n;
+  for (int c = n + lane; c < C; c += 32) { v.row_sub[c] = 0; v.row_meta[c] = make_int4(0, 0, 0, 0); }
+  if (lane == 0) st.n_active[b] = n;
+  __syncwarp();
   // Page list of the coming step for the self-attention kernels: every page of subsequences
   // 1..i_max (i_max = last active one; later ones are invisible to every row), with the number
   // of entries it will hold once the step's inputs are appended (bos + content = len + 1 per
@@ -130,21 +212,31 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqS
   int np = 0;
   if (n > 0) {
     const int i_last = v.row_sub[n - 1];
-    for (int i = 1; i <= i_last; ++i) {
-      const int entries = v.len[i - 1] + 1;
-      const int pos0 = v.start[i - 1] - 1 + i;
-      for (int j = 0; j * dm.P < entries; ++j)
-        v.plist[np++] = make_int4(v.page_table[(i - 1) * dm.PPS + j], min(dm.P, entries - j * dm.P), i, t - (pos0 + j * dm.P));
+    for (int i0 = 0; i0 < i_last; i0 += 32) {
+      const int i = i0 + lane + 1;
+      const bool on = i <= i_last;
+      const int entries = on ? v.len[i - 1] + 1 : 0;
+      const int cnt = (entries + P - 1) / P;
+      int incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += u; }
+      if (on) {
+        const int off = np + incl - cnt;
+        const int pos0 = v.start[i - 1] - 1 + i;
+        for (int j = 0; j < cnt; ++j)
+          v.plist[off + j] = make_int4(v.page_table[(i - 1) * dm.PPS + j], min(P, entries - j * P), i, t - (pos0 + j * P));
+      }
+      np += __shfl_sync(FULL, incl, 31);
     }
   }
-  st.plist_n[b] = np;
+  if (lane == 0) st.plist_n[b] = np;
 }
 
 // Called by every thread of a row's CTA once the row's choice is in row_tok: the CTA that arrives
-// last for its sequence stages the sequence's state, runs its scheduler and writes the state back;
-// the last sequence advances the step.  No CTA ever waits for another.
-__device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, const int32_t *teacher, int *is_last) {
-  extern __shared__ __align__(16) uint8_t sched_smem[];
+// last for its sequence fetches the rows' choices, runs the sequence's scheduler in its first warp
+// and writes the state back; the last sequence advances the step.  No CTA ever waits for another.
+__device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, const int32_t *teacher, int *is_last,
+                         const SeqStage &v, const SeqScalars &sc) {
   const int tid = threadIdx.x, nthr = blockDim.x;
   if (tid == 0) {
     __threadfence();
@@ -155,32 +247,14 @@ __device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, c
   if (!*is_last) return;
   __threadfence();
   const int C = dm.C, SM = dm.SM, NPT = dm.SM * dm.PPS;
-  SeqStage v;
-  int32_t *w = reinterpret_cast<int32_t *>(sched_smem);
-  v.row_sub = w; w += C;
-  v.row_tok = w; w += C;
-  v.len = w; w += SM; v.forced_len = w; w += SM; v.state = w; w += SM; v.flag = w; w += SM;
-  v.start = w; w += SM; v.last_tok = w; w += SM; v.teacher = w; w += SM;
-  v.page_table = w; w += NPT;
-  w = reinterpret_cast<int32_t *>(sched_smem) + (size_t)(2 * C + 7 * SM + NPT + 3) / 4 * 4;     // 16-byte aligned
-  v.row_meta = reinterpret_cast<int4 *>(w);
-  v.plist = v.row_meta + C;
   for (int c = tid; c < C; c += nthr) {
-    v.row_sub[c] = st.row_sub[b * C + c];
     v.row_tok[c] = __ldcg(&st.row_tok[b * C + c]);            // written by other CTAs of this launch
     st.prev_row_sub[b * C + c] = v.row_sub[c];
   }
-  for (int i = tid; i < SM; i += nthr) {
-    const int sidx = b * SM + i;
-    v.len[i] = st.len[sidx]; v.forced_len[i] = st.forced_len[sidx]; v.state[i] = st.state[sidx]; v.flag[i] = st.flag[sidx];
-    v.start[i] = st.start[sidx]; v.last_tok[i] = st.last_tok[sidx];
-    v.teacher[i] = teacher != nullptr ? teacher[sidx] : -1;
-  }
-  for (int i = tid; i < NPT; i += nthr) v.page_table[i] = st.page_table[(size_t)b * NPT + i];
   __syncthreads();
-  if (tid == 0) {
-    st.seq_ticket[b] = 0;
-    schedule_sequence(dm, st, v, b, teacher != nullptr);
+  if (tid < 32) {
+    if (tid == 0) st.seq_ticket[b] = 0;
+    schedule_sequence(dm, st, v, b, teacher != nullptr, sc);
   }
   __syncthreads();
   for (int c = tid; c < C; c += nthr) { st.row_sub[b * C + c] = v.row_sub[c]; st.row_meta[b * C + c] = v.row_meta[c]; }
@@ -190,7 +264,7 @@ __device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, c
     st.last_tok[sidx] = v.last_tok[i];
   }
   for (int i = tid; i < NPT; i += nthr) st.page_table[(size_t)b * NPT + i] = v.page_table[i];
-  const int np = st.plist_n[b];                        // written by thread 0 before the barrier above
+  const int np = st.plist_n[b];                        // written by lane 0 before the barrier above
   for (int i = tid; i < np; i += nthr) st.plist[(size_t)b * NPT + i] = v.plist[i];
   __threadfence();
   __syncthreads();
@@ -209,11 +283,14 @@ __device__ void row_done(const Dims &dm, const DecState &st, int batch, int b, c
 
 __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, int batch, const float *__restrict__ logits,
                                                           const int32_t *__restrict__ teacher) {
+  extern __shared__ __align__(16) uint8_t sched_smem[];
   __shared__ float sv[AT / 32];
   __shared__ int si[AT / 32];
   __shared__ int is_last;
   const int r = blockIdx.x, tid = threadIdx.x;
   const int b = r / dm.C;
+  const SeqStage stage = seq_stage_views(dm, sched_smem);
+  const SeqScalars sc = stage_in(dm, st, b, teacher, stage);
   const int i = st.row_sub[r];
   if (i > 0) {
     const int sidx = b * dm.SM + i - 1;
@@ -261,7 +338,7 @@ __global__ void __launch_bounds__(AT) argmax_sched_kernel(Dims dm, DecState st, 
       st.row_tok[r] = bi == INT_MAX ? 0 : bi;
     }
   }
-  row_done(dm, st, batch, b, teacher, &is_last);
+  row_done(dm, st, batch, b, teacher, &is_last, stage, sc);
 }
 
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,
@@ -279,20 +356,26 @@ constexpr int PT = 64;
 __global__ void __launch_bounds__(PT) pick_sched_kernel(Dims dm, DecState st, int batch, int tiles, int rows_cap,
                                                         const float *__restrict__ part_val, const int32_t *__restrict__ part_idx,
                                                         const float *__restrict__ term_val, const int32_t *__restrict__ teacher) {
+  extern __shared__ __align__(16) uint8_t sched_smem[];
   __shared__ float sv[PT / 32];
   __shared__ int si[PT / 32];
   __shared__ int is_last;
   const int r = blockIdx.x, tid = threadIdx.x;
   const int b = r / dm.C;
+  // first round of loads: the row's subsequence, the sequence's place among the packed rows, and the
+  // sequence's state for the scheduler
   const int i = st.row_sub[r];
+  const int m = st.crow[b] + r % dm.C;                 // the row's place among the packed rows (meaningful when i > 0)
+  const SeqStage stage = seq_stage_views(dm, sched_smem);
+  const SeqScalars sc = stage_in(dm, st, b, teacher, stage);
   if (i > 0) {
     const int sidx = b * dm.SM + i - 1;
-    const int fl = st.forced_len[sidx];
-    const bool bar = fl >= 0 && st.len[sidx] < fl;     // terminators cannot win before the forced length
-    const int m = st.crow[b] + r % dm.C;               // the row's place among the packed rows
+    // second round: the forced-length rule's inputs and the row's candidates
+    const int fl = st.forced_len[sidx], len = st.len[sidx];
     float bv = -INFINITY;
     int bi = INT_MAX;
     for (int t = tid; t < tiles; t += PT) better(bv, bi, __ldcg(part_val + (size_t)t * rows_cap + m), __ldcg(part_idx + (size_t)t * rows_cap + m));
+    const bool bar = fl >= 0 && len < fl;              // terminators cannot win before the forced length
     if (tid == 0 && !bar) {
       better(bv, bi, __ldcg(term_val + 2 * m), dm.eos);
       if (dm.sep != dm.eos) better(bv, bi, __ldcg(term_val + 2 * m + 1), dm.sep);
@@ -309,7 +392,7 @@ __global__ void __launch_bounds__(PT) pick_sched_kernel(Dims dm, DecState st, in
       st.row_tok[r] = bi == INT_MAX ? 0 : bi;
     }
   }
-  row_done(dm, st, batch, b, teacher, &is_last);
+  row_done(dm, st, batch, b, teacher, &is_last, stage, sc);
 }
 
 cudaError_t launch_pick_sched(const Dims &dm, const DecState &st, int batch, int tiles, const float *part_val,
