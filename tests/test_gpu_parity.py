@@ -266,6 +266,30 @@ def test_bf16_choices_do_not_depend_on_storing_the_logits():
         assert np.array_equal(out[0][k], out[1][k]), k
 
 
+def test_generate_host_in_uneven_chunks_matches_stepwise_run():
+    """38 MB of encoder memory cross PCIe as two chunks of 4 and 5 sequences, each projected while
+    the next one is still being copied: the streams must be those of the plain encode + step path."""
+    import torch
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = W.CONFIGS["bart_base"].scaled(name="chunks", batch=9, ctx=4096, sub_max=3, delta_t=2, max_sub_len=6,
+                                       length_dist=("uniform", 1, 6), time_max=16, n_layers=2, d_model=512, n_heads=8,
+                                       d_ff=512, vocab=500)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch)
+    mem_dev = dec.device_memory(mem)
+    dec.encode_context(mem_dev, ctx_len, fl)
+    dec.run()
+    a = dec.collect()
+    host = mem_dev.cpu().pin_memory()
+    assert host.numel() * host.element_size() >= 2 * (16 << 20)
+    for _ in range(2):                                  # the second call reuses the staging buffer
+        b = dec.generate_host(host, ctx_len, fl)
+        for k in a:
+            assert np.array_equal(a[k], b[k]), k
+    dec.close()
+
+
 FULL = [("bart_base", 2e-2), ("long_context", 2e-2), ("summarisation", 2e-2), ("keyphrase", 2e-2)]
 
 
