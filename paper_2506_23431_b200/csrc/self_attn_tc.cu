@@ -103,6 +103,11 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
   const int4 *pl = a.st.plist + (size_t)b * list_cap;
   int4 my_entry = make_int4(0, 0, 0, 0);
   if (tid < list_cap) my_entry = pl[tid];
+  // this warp's first two pages (entries g0 and g0 + W of the list), so that their copies can start
+  // before the CTA has assembled the list in shared memory
+  const int W = a.splits * SW, g0 = split * SW + warp;
+  const int4 first0 = g0 < list_cap ? pl[g0] : make_int4(0, 0, 0, 0);
+  const int4 first1 = g0 + W < list_cap ? pl[g0 + W] : make_int4(0, 0, 0, 0);
   int my_rsub = 0;
   if (tid < dm.C) my_rsub = a.st.row_sub[row0 + tid];
   const bool use_bias = a.bias_tab != nullptr;
@@ -134,12 +139,22 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
         out[(size_t)(row0 + idx / kDh) * dm.d + h * kDh + idx % kDh] = __float2bfloat16_rn(0.f);
     return;
   }
+  const int n_mine = n_list > g0 ? (n_list - g0 + W - 1) / W : 0;
+  const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SLOT;
+  const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
+  const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
+  auto fetch = [&](int n, int4 e) { s_fetch_page<P>(my_ring + (n & 1) * SLOT, pool_lh + e.x * page_stride, e.y, lane); };
   {
-    // The ring starts out zeroed: value rows beyond a partly filled page's entries get weights of
-    // exactly 0 in P.V and must be finite, whatever the slot held before (later: earlier pages' data).
-    uint4 *ring = reinterpret_cast<uint4 *>(s_ring_raw);
+    // The warp's ring starts out zeroed: value rows beyond a partly filled page's entries get weights
+    // of exactly 0 in P.V and must be finite, whatever the slot held before (later: earlier pages' data).
+    uint4 *ring = reinterpret_cast<uint4 *>(s_ring_raw + (size_t)warp * SDEPTH * SLOT);
 #pragma unroll
-    for (int i = 0; i < (int)(SW * SDEPTH * SLOT / 16) / STHREADS; ++i) ring[i * STHREADS + tid] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = 0; i < (int)(SDEPTH * SLOT / 16) / 32; ++i) ring[i * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();                      // the zeros are in place before any lane's copy lands on them
+    if (n_mine > 0) fetch(0, first0);
+    s_cp_async_commit();
+    if (n_mine > 1) fetch(1, first1);
+    s_cp_async_commit();
   }
   if (tid < SMAXLIST) plist_s[tid] = my_entry;
   for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
@@ -157,17 +172,7 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
   }
   __syncthreads();
 
-  // ---- this warp's share of the page list: entries g0, g0 + W, ...; request its first two pages
-  const int W = a.splits * SW, g0 = split * SW + warp;
-  const int n_mine = n_list > g0 ? (n_list - g0 + W - 1) / W : 0;
-  const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SLOT;
-  const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
-  const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
-  auto fetch = [&](int n, int4 e) { s_fetch_page<P>(my_ring + (n & 1) * SLOT, pool_lh + e.x * page_stride, e.y, lane); };
-  if (n_mine > 0) fetch(0, plist_s[g0]);
-  s_cp_async_commit();
-  if (n_mine > 1) fetch(1, plist_s[g0 + W]);
-  s_cp_async_commit();
+  // ---- this warp's share of the page list is entries g0, g0 + W, ...; its first two pages are already on their way
 
   int rs[MT][2];                     // subsequence of rows g and g + 8 of every query tile
   int tile_last[MT];                 // subsequence of the tile's last active row (rows are sorted)
