@@ -29,6 +29,7 @@ constexpr int XTILE_BYTES = XK * kDh * 2; // 16 KB
 constexpr int XSTAGE_BYTES = 2 * XTILE_BYTES;
 constexpr int XMIN_TILES = 4;              // fewest tiles worth a CTA of its own
 constexpr int XMIN_WHOLE = 64;             // fewest CTAs for which whole (sequence, head) segments per CTA still beat cutting the tile list
+constexpr int XLONG_SEG = 24;              // tiles from which a segment is worth two CTAs when there are fewer segments than SMs
 constexpr int XMAXB = 256;                // sequences per launch the tile prefix table holds
 constexpr int XREC_WORDS = 36;            // per lane and 16-row tile: 32 output values, 2 maxima, 2 sums
 constexpr int XREC_FLOATS = XREC_WORDS * 32;
@@ -228,10 +229,14 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   int lo, hi;
   // With enough (sequence, head) segments to keep at least one CTA per SM streaming, every CTA takes
   // whole segments (the same number each): nothing is cut, so there are no partial records, no
-  // tickets and no merge after the last tile.  Otherwise the tile list itself is cut into equal ranges.
+  // tickets and no merge after the last tile.  Otherwise the tile list itself is cut into equal
+  // ranges.  Fewer segments than SMs, but long ones (a lone CTA streams 32 tiles too slowly): two
+  // CTAs per segment.
   const int n_seg = n_aseq_s * H;
   const int seg_per_cta = (n_seg + G - 1) / G;
-  const bool whole_segments = n_seg > 0 && (n_seg + seg_per_cta - 1) / seg_per_cta >= XMIN_WHOLE;
+  const bool two_per_segment = n_seg > 0 && 2 * n_seg <= G && T >= (long long)XLONG_SEG * n_seg;
+  const bool whole_segments = n_seg > 0 && (n_seg + seg_per_cta - 1) / seg_per_cta >= XMIN_WHOLE && !two_per_segment;
+  if (two_per_segment && 2 * n_seg < Ge) Ge = 2 * n_seg;
   if (whole_segments) {
     Ge = (n_seg + seg_per_cta - 1) / seg_per_cta;
     if (cta >= Ge) return;
@@ -308,17 +313,10 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
       const uint32_t kbase = base + s * XSTAGE_BYTES, vbase = kbase + XTILE_BYTES;
       const int key0 = tile * XK + kb;               // context position of this warp's first key
       const bool ragged = key0 + 32 > ctx_len;
-      if (ragged) {
-        // Rows at or beyond ctx_len hold whatever follows in memory.  Their weights are exactly 0
-        // below; zero the value rows so that 0 never multiplies a non-finite.
-        if (key0 + lane >= ctx_len) {
-          uint4 *vrow = reinterpret_cast<uint4 *>(smem_al + (vbase - base) + (kb + lane) * 128);
-#pragma unroll
-          for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage's next bulk copy
-        }
-        __syncwarp();
-      }
+      // Rows at or beyond ctx_len hold whatever follows in memory.  Their weights are exactly 0 below;
+      // the value fragments of those keys are cleared in registers after ldmatrix, so that 0 never
+      // multiplies a non-finite.  (Nothing but TMA ever writes a stage: zeroing the rows in shared
+      // memory raced with the next bulk copy into the stage, proxy fence or not.)
       // ---- scores: S[mt][nt] = Q (16 x 64) . K^T (64 x 8 keys)
       float sc[MT][4][4];
 #pragma unroll
@@ -385,10 +383,18 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
         const int key = kb + ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+        // this lane's fragment halves hold keys k0, k0 + 1 (b0, b2) and k0 + 8, k0 + 9 (b1, b3)
+        uint32_t keep_a = 0xffffffffu, keep_b = 0xffffffffu;
+        if (ragged) {
+          const int k0 = key0 + ks * 16 + 2 * tig;
+          keep_a = (k0 < ctx_len ? 0x0000ffffu : 0u) | (k0 + 1 < ctx_len ? 0xffff0000u : 0u);
+          keep_b = (k0 + 8 < ctx_len ? 0x0000ffffu : 0u) | (k0 + 9 < ctx_len ? 0xffff0000u : 0u);
+        }
 #pragma unroll
         for (int dp = 0; dp < 4; ++dp) {      // two 8-wide slices of the head per ldmatrix.x4
           uint32_t b0, b1, b2, b3;
           ldsm_x4_t(vbase + swz(key, dp * 2 + (lane >> 4)), b0, b1, b2, b3);
+          if (ragged) { b0 &= keep_a; b1 &= keep_b; b2 &= keep_a; b3 &= keep_b; }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             mma_bf16(acc[mt].o[2 * dp], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b0, b1);

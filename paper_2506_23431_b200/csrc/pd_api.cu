@@ -422,6 +422,15 @@ pd_status device_status(pd_handle *h) {
 pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, const int32_t *forced_len);
 pd_status encode_project(pd_handle *h, const void *enc_mem, int b0, int nb);
 
+// Chunks of whole sequences the encoder memory is projected in: at least 16 MiB each, at most kMaxChunks.
+int encode_chunks(const pd_handle *h, int batch) {
+  const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * (h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4);
+  int n = (int)((size_t)batch * seq_bytes / ((size_t)16 << 20));
+  if (n > pd_handle::kMaxChunks) n = pd_handle::kMaxChunks;
+  if (n > batch) n = batch;
+  return n < 1 ? 1 : n;
+}
+
 }  // namespace
 
 extern "C" {
@@ -521,7 +530,14 @@ pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int32_t *ct
   if (!h) return PD_ERR_ARG;
   if (!enc_mem) return fail(h, PD_ERR_ARG, "pd_encode_context: bad argument");
   PD_TRY(encode_prepare(h, ctx_len, batch, forced_len));
-  PD_TRY(encode_project(h, enc_mem, 0, batch));
+  // the same chunks of sequences as pd_generate_host, so that both project with the same GEMM shapes
+  // and give bit-identical keys/values
+  const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * (h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4);
+  const int n_chunks = encode_chunks(h, batch);
+  for (int c = 0; c < n_chunks; ++c) {
+    const int b0 = (int)((long long)batch * c / n_chunks), b1 = (int)((long long)batch * (c + 1) / n_chunks);
+    PD_TRY(encode_project(h, static_cast<const uint8_t *>(enc_mem) + b0 * seq_bytes, b0, b1 - b0));
+  }
   h->encoded = true;
   h->steps_enqueued = 0;
   return PD_OK;
@@ -685,10 +701,7 @@ pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t
   // Chunks of whole sequences, at least 16 MiB each: chunk c is projected on the handle's stream
   // while chunk c + 1 is still crossing PCIe on the copy stream.
   const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * e;
-  int n_chunks = (int)((size_t)batch * seq_bytes / ((size_t)16 << 20));
-  if (n_chunks > pd_handle::kMaxChunks) n_chunks = pd_handle::kMaxChunks;
-  if (n_chunks > batch) n_chunks = batch;
-  if (n_chunks < 1) n_chunks = 1;
+  const int n_chunks = encode_chunks(h, batch);
   CU_TRY(h, cudaEventRecord(h->ev_entry, h->stream));                  // the staging buffer is free once earlier work is done
   CU_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_entry, 0));
   uint8_t *stage = h->ptr<uint8_t>(h->lay.enc_stage);
