@@ -151,3 +151,34 @@ def test_vocab_argmax_rejects_bad_arguments():
         B.vocab_argmax(h, w, scratch=torch.empty(256, dtype=torch.uint8, device=dev))
     assert e.value.status == -3
     assert B._lib.pd_vocab_argmax_scratch_bytes(0, 10) == 0
+
+
+def test_cross_attention_is_bit_reproducible_after_ragged_tiles():
+    """Few, long (sequence, head) segments with ragged context lengths: CTAs take half segments and
+    carry on into the next segment after a ragged last tile.  Twenty launches on the same inputs must
+    give the same bits (a write into a TMA stage once raced with the next bulk copy here), and those
+    bits must match the oracle."""
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    batch, rows, heads, ctx = 9, 3, 8, 4096
+    q, kv, n_rows, _ = cross_case(5, batch, rows, heads, ctx, "bf16", poison=False)
+    n_rows[:] = rows
+    ctx_len = np.array([3256, 3607, 2257, 4079, 3732, 2935, 2640, 3064, 3757], dtype=np.int32)
+    for b in range(batch):
+        kv[b, :, :, ctx_len[b]:] = np.nan                 # positions beyond ctx_len must never matter
+    ref = oracle_cross(q, kv, n_rows, ctx_len, heads, 0.125)
+    dev = torch.device("cuda", 0)
+    q_d, kv_d = torch.from_numpy(q).to(dev, torch.bfloat16), torch.from_numpy(kv).to(dev, torch.bfloat16)
+    nr_d, cl_d = torch.from_numpy(n_rows).to(dev), torch.from_numpy(ctx_len).to(dev)
+    first = None
+    for _ in range(20):
+        out = B.cross_attention(q_d, kv_d, nr_d, cl_d, 0.125, 1)
+        torch.cuda.synchronize()
+        bits = out.view(torch.int16).cpu().numpy()
+        if first is None:
+            first = bits
+            got = out.float().cpu().numpy().astype(np.float64)
+            assert np.isfinite(got).all()
+            assert np.abs(got - ref).max() <= 2e-3
+        else:
+            assert np.array_equal(bits, first), "two launches on the same inputs gave different bits"
