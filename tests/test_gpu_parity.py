@@ -290,6 +290,35 @@ def test_generate_host_in_uneven_chunks_matches_stepwise_run():
     dec.close()
 
 
+def test_two_identical_decodes_give_identical_logits():
+    """Run-to-run reproducibility of the whole step (ragged contexts, several CTAs per (sequence, head)
+    segment in cross-attention, split self-attention): the fp32 logits of every step must repeat bit
+    for bit."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = W.CONFIGS["bart_base"].scaled(name="repeat", batch=9, ctx=4096, sub_max=3, delta_t=2, max_sub_len=6,
+                                       length_dist=("uniform", 1, 6), time_max=16, n_layers=2, d_model=512, n_heads=8,
+                                       d_ff=512, vocab=500)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch)
+    mem_dev = dec.device_memory(mem)
+
+    def trace():
+        dec.encode_context(mem_dev, ctx_len, fl)
+        out = []
+        for _ in range(8):
+            dec.step()
+            out.append(dec.get_logits()[0].copy())
+        return out
+
+    first = trace()
+    for _ in range(3):
+        again = trace()
+        for s, (x, y) in enumerate(zip(first, again)):
+            assert np.array_equal(x.view(np.int32), y.view(np.int32)), f"logits of step {s + 1} differ between two identical runs"
+    dec.close()
+
+
 FULL = [("bart_base", 2e-2), ("long_context", 2e-2), ("summarisation", 2e-2), ("keyphrase", 2e-2)]
 
 
