@@ -422,10 +422,11 @@ pd_status device_status(pd_handle *h) {
 pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, const int32_t *forced_len);
 pd_status encode_project(pd_handle *h, const void *enc_mem, int b0, int nb);
 
-// Chunks of whole sequences the encoder memory is projected in: at least 16 MiB each, at most kMaxChunks.
+// Chunks of whole sequences the encoder memory is projected in: at least 64 MiB each (smaller GEMMs
+// cost more than the overlap with the host copy returns), at most kMaxChunks.
 int encode_chunks(const pd_handle *h, int batch) {
   const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * (h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4);
-  int n = (int)((size_t)batch * seq_bytes / ((size_t)16 << 20));
+  int n = (int)((size_t)batch * seq_bytes / ((size_t)64 << 20));
   if (n > pd_handle::kMaxChunks) n = pd_handle::kMaxChunks;
   if (n > batch) n = batch;
   return n < 1 ? 1 : n;
@@ -698,8 +699,8 @@ pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t
   if (batch < 1 || batch > h->dm.B) return fail(h, PD_ERR_ARG, "pd_generate_host: bad batch");
   const size_t e = h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4;
   CU_TRY(h, cudaSetDevice(h->cfg.device));
-  // Chunks of whole sequences, at least 16 MiB each: chunk c is projected on the handle's stream
-  // while chunk c + 1 is still crossing PCIe on the copy stream.
+  // Chunks of whole sequences: chunk c is projected on the handle's stream while chunk c + 1 is still
+  // crossing PCIe on the copy stream.
   const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * e;
   const int n_chunks = encode_chunks(h, batch);
   CU_TRY(h, cudaEventRecord(h->ev_entry, h->stream));                  // the staging buffer is free once earlier work is done
