@@ -182,3 +182,37 @@ def test_cross_attention_is_bit_reproducible_after_ragged_tiles():
             assert np.abs(got - ref).max() <= 2e-3
         else:
             assert np.array_equal(bits, first), "two launches on the same inputs gave different bits"
+
+
+RANDOM_SHAPES = [
+    # seed, batch, rows, heads, ctx: chosen to reach every way the kernel divides the tile list
+    (21, 40, 5, 8, 700),       # 320 segments: whole segments per CTA, two of them for some CTAs
+    (22, 12, 9, 8, 1500),      # 96 short segments: one CTA each
+    (23, 6, 16, 8, 3300),      # 48 long segments: two CTAs per segment, ragged ends inside the CTAs' ranges
+    (24, 2, 30, 4, 2900),      # 8 segments, two query tiles: the tile list cut into many short ranges
+    (25, 1, 1, 1, 129),        # one row, one head, one key beyond a tile edge
+    (26, 70, 3, 4, 260),       # many sequences with two or three tiles each
+]
+
+
+@pytest.mark.parametrize("seed,batch,rows,heads,ctx", RANDOM_SHAPES)
+def test_cross_attention_random_ragged_shapes(seed, batch, rows, heads, ctx):
+    """Ragged contexts and row counts (some sequences inactive) on shapes that reach every partition of the
+    tile list; NaNs beyond ctx_len; the result must match the oracle and repeat bit for bit."""
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    q, kv, n_rows, ctx_len = cross_case(seed, batch, rows, heads, ctx, "bf16")
+    ref = oracle_cross(q, kv, n_rows, ctx_len, heads, 0.125)
+    dev = torch.device("cuda", 0)
+    args = (torch.from_numpy(q).to(dev, torch.bfloat16), torch.from_numpy(kv).to(dev, torch.bfloat16),
+            torch.from_numpy(n_rows).to(dev), torch.from_numpy(ctx_len).to(dev), 0.125, 1)
+    outs = []
+    for _ in range(4):
+        out = B.cross_attention(*args)
+        torch.cuda.synchronize()
+        outs.append(out)
+    got = outs[0].float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= 1e-2
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))
