@@ -136,8 +136,11 @@ PD_API pd_status pd_encode_context(pd_handle *h, const void *enc_mem, const int3
  * -1 keeps the own choice.  Enqueues only; a no-op for sequences that are done. */
 PD_API pd_status pd_step(pd_handle *h, const int32_t *teacher_tokens);
 
-/* Runs pd_step(NULL) until every sequence is done or time_max is reached, polling the device
- * every `poll_every` steps (>= 1).  Returns the number of steps enqueued in *steps_run. */
+/* Runs pd_step(NULL) until every sequence is done or time_max is reached.  The host follows the
+ * device min(poll_every, 2) steps behind (poll_every >= 1) through header snapshots copied on a
+ * stream of the handle's own, so the decode stream is never drained to look; at most that many
+ * steps are enqueued past the end (they are no-ops).  Returns the number of steps enqueued in
+ * *steps_run.  Synchronises at the end. */
 PD_API pd_status pd_run(pd_handle *h, int32_t poll_every, int32_t *steps_run);
 
 /* Synchronises the stream; *all_done = 1 when every sequence has ended or hit time_max. */

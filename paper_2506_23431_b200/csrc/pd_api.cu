@@ -155,6 +155,10 @@ struct pd_handle {
   static constexpr int kMaxChunks = 8;
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_entry = nullptr, ev_chunk[kMaxChunks] = {};
+  // pd_run: a snapshot of the header after every step travels to pinned memory on the copy stream, so
+  // that the host can follow the decode a couple of steps behind without ever draining the stream
+  static constexpr int kRunSlots = 4;
+  cudaEvent_t ev_step[kRunSlots] = {}, ev_snap[kRunSlots] = {};
   int batch = 0;
   bool encoded = false;
   int self_splits = 1, cross_splits = 1;
@@ -469,11 +473,14 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   if (cublasLtCreate(&h->lt) != CUBLAS_STATUS_SUCCESS) h->lt = nullptr;     // optional: the ReLU then runs as its own kernel
   if (cublasSetWorkspace(h->blas, h->ptr<void>(h->lay.cublas_ws), kCublasWs) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
   if (cublasSetMathMode(h->blas, CUBLAS_DEFAULT_MATH) != CUBLAS_STATUS_SUCCESS) return bail(PD_ERR_CUDA);
-  if (cudaHostAlloc((void **)&h->pinned_flag, 64, cudaHostAllocDefault) != cudaSuccess) return bail(PD_ERR_CUDA);
+  if (cudaHostAlloc((void **)&h->pinned_flag, 64 * (1 + pd_handle::kRunSlots), cudaHostAllocDefault) != cudaSuccess) return bail(PD_ERR_CUDA);
   if (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&h->ev_entry, cudaEventDisableTiming) != cudaSuccess) return bail(PD_ERR_CUDA);
   for (int c = 0; c < pd_handle::kMaxChunks; ++c)
     if (cudaEventCreateWithFlags(&h->ev_chunk[c], cudaEventDisableTiming) != cudaSuccess) return bail(PD_ERR_CUDA);
+  for (int c = 0; c < pd_handle::kRunSlots; ++c)
+    if (cudaEventCreateWithFlags(&h->ev_step[c], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_snap[c], cudaEventDisableTiming) != cudaSuccess) return bail(PD_ERR_CUDA);
 
   int32_t *sb = h->ptr<int32_t>(h->lay.state);
   const Layout &L = h->lay;
@@ -663,17 +670,29 @@ pd_status pd_done(pd_handle *h, int32_t *all_done) {
 pd_status pd_run(pd_handle *h, int32_t poll_every, int32_t *steps_run) {
   if (!h || poll_every < 1) return PD_ERR_ARG;
   if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_run before pd_encode_context");
+  // The host stays `lag` steps ahead of the device: before it enqueues step n + 1 it waits for the
+  // header snapshot taken after step n + 1 - lag (the stream still holds lag - 1 steps of work then).
+  const int lag = poll_every < 2 ? poll_every : 2;      // two is enough to keep the stream fed; more only adds steps past the end
   int n = 0;
   int32_t done = 0;
-  while (h->steps_enqueued < h->dm.T) {
+  while (h->steps_enqueued < h->dm.T && !done) {
     PD_TRY(pd_step(h, nullptr));
+    const int slot = n % pd_handle::kRunSlots;
+    int32_t *snap = h->pinned_flag + 16 * (1 + slot);
+    CU_TRY(h, cudaEventRecord(h->ev_step[slot], h->stream));
+    CU_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_step[slot], 0));
+    CU_TRY(h, cudaMemcpyAsync(snap, h->st.hdr, 8 * sizeof(int32_t), cudaMemcpyDeviceToHost, h->copy_stream));
+    CU_TRY(h, cudaEventRecord(h->ev_snap[slot], h->copy_stream));
     ++n;
-    if (n % poll_every == 0) {
-      PD_TRY(pd_done(h, &done));
-      if (done) break;
+    if (n >= lag) {
+      const int old = (n - lag) % pd_handle::kRunSlots;
+      CU_TRY(h, cudaEventSynchronize(h->ev_snap[old]));
+      const int32_t *s_old = h->pinned_flag + 16 * (1 + old);
+      if (s_old[HDR_STATUS] != 0) return fail(h, (pd_status)s_old[HDR_STATUS], "device-side error " + std::to_string(s_old[HDR_STATUS]));
+      done = s_old[HDR_ALL_DONE];
     }
   }
-  if (!done) PD_TRY(pd_done(h, &done));
+  PD_TRY(pd_done(h, &done));
   if (steps_run) *steps_run = n;
   return PD_OK;
 }
@@ -869,6 +888,8 @@ void pd_destroy(pd_handle *h) {
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   if (h->pinned_flag) cudaFreeHost(h->pinned_flag);
   for (cudaEvent_t e : h->ev_chunk) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_step) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_snap) if (e) cudaEventDestroy(e);
   if (h->ev_entry) cudaEventDestroy(h->ev_entry);
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   drop_ff_plan(h);
