@@ -99,6 +99,9 @@ VOCAB_CASES = [
     (100, 64, 224),        # one row tile, one vocabulary slice, a single K block
     (200, 256, 1000),      # two row tiles (ragged), five slices, the last one partly beyond the vocabulary
     (600, 1024, 5000),     # five row tiles: three passes over every slice
+    (1, 64, 8),            # the smallest shapes: one row, eight ids
+    (257, 128, 225),       # one row and one id beyond a tile edge: second pass with a single row, second slice with one id
+    (513, 192, 449),       # three K blocks, three passes, three slices
 ]
 
 
