@@ -426,11 +426,12 @@ pd_status device_status(pd_handle *h) {
 pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, const int32_t *forced_len);
 pd_status encode_project(pd_handle *h, const void *enc_mem, int b0, int nb);
 
-// Chunks of whole sequences the encoder memory is projected in: at least 64 MiB each (smaller GEMMs
-// cost more than the overlap with the host copy returns), at most kMaxChunks.
+// Chunks of whole sequences the encoder memory is projected in: at least 32 MiB each (many small
+// GEMMs cost pd_encode_context more than the overlap with the host copy returns to
+// pd_generate_host), at most kMaxChunks.
 int encode_chunks(const pd_handle *h, int batch) {
   const size_t seq_bytes = (size_t)h->dm.ctx * h->dm.d * (h->cfg.dtype == PD_DTYPE_BF16 ? 2 : 4);
-  int n = (int)((size_t)batch * seq_bytes / ((size_t)64 << 20));
+  int n = (int)((size_t)batch * seq_bytes / ((size_t)32 << 20));
   if (n > pd_handle::kMaxChunks) n = pd_handle::kMaxChunks;
   if (n > batch) n = batch;
   return n < 1 ? 1 : n;

@@ -267,8 +267,8 @@ def test_bf16_choices_do_not_depend_on_storing_the_logits():
 
 
 def test_generate_host_in_uneven_chunks_matches_stepwise_run():
-    """143 MB of encoder memory cross PCIe as two chunks of 8 and 9 sequences, the first projected while
-    the second is still being copied: the streams must be those of the plain encode + step path."""
+    """143 MB of encoder memory cross PCIe as four chunks of 4, 4, 4 and 5 sequences, each projected while
+    the next is still being copied: the streams must be those of the plain encode + step path."""
     import torch
     from paper_2506_23431_b200.binding import PipelinedDecoder
     wl = W.CONFIGS["bart_base"].scaled(name="chunks", batch=17, ctx=4096, sub_max=3, delta_t=2, max_sub_len=6,
