@@ -581,6 +581,14 @@ pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, co
   const int bh = batch * dm.H;
   int ss = h->cfg.self_splits > 0 ? h->cfg.self_splits : cdiv(2 * 148, bh);
   if (ss > 8 && h->cfg.self_splits == 0) ss = 8;
+  if (h->cfg.self_splits == 0 && h->cfg.dtype == PD_DTYPE_BF16 && self_attn_tc_supported(dm)) {
+    // The tensor-core kernel works through a page in well under a microsecond per warp, while a split
+    // costs a second launch for the merge (about 6 us): split only when a sequence's page list can get
+    // so long that an unsplit warp would walk more than 16 pages, and never beyond one wave of CTAs.
+    ss = cdiv(dm.SM * dm.PPS, 4 * 16);
+    while (ss > 1 && bh * ss > 2 * 148) --ss;
+    if (ss > 8) ss = 8;
+  }
   int cs = h->cfg.cross_splits;
   if (cs == 0) {
     int tiles = cdiv(dm.ctx, 128);
