@@ -231,6 +231,8 @@ PD_API pd_status pd_get_stats(pd_handle *h, int64_t *stats);
  *                its projected context in); positions at or beyond ctx_len[b] are ignored (they
  *                may hold anything)
  *   n_rows       device int32 [batch], 0..rows_per_seq;  ctx_len  device int32 [batch], 1..max_ctx
+ *                (the kernels clamp what they read to these ranges, so a bad value gives a wrong
+ *                result for that sequence, never an access outside the tensors)
  *   splits       1..32: split-K factor over the context of the plain-ALU kernel (fp32, or more
  *                than 32 rows per sequence; partials are merged by a second kernel).  The bf16
  *                tensor-core kernel divides the context tiles of all sequences evenly over the
@@ -277,9 +279,13 @@ PD_API pd_status pd_vocab_argmax(int32_t rows, int32_t d_model, int32_t vocab, c
  * the library image (pd_cross_attention_static_max_bytes()), which every GPU that loads the
  * library carries until the process exits.  The caller still passes q, kv, n_rows, ctx_len and
  * out exactly as for pd_cross_attention; results are the same.
- *  - Sizes whose partials would not fit (pd_cross_attention_scratch_bytes(...) above the
- *    maximum) are refused with PD_ERR_WORKSPACE and a message in pd_static_last_error(); use
- *    fewer splits, a smaller batch, or pd_cross_attention with a buffer of your own.
+ *  - Sizes whose partials would not fit are refused with PD_ERR_WORKSPACE and a message in
+ *    pd_static_last_error(); use fewer splits, fewer sequences or rows per call, or
+ *    pd_cross_attention with a buffer of your own.  What is needed depends on the kernel that
+ *    runs: the bf16 tensor-core kernel (at most 32 rows per sequence) keeps per-CTA records
+ *    (2.9 MiB up to 16 rows, 5.9 MiB up to 32, whatever the batch), the plain-ALU kernel (fp32,
+ *    or 33..64 rows) batch*rows*heads*splits*264 bytes; pd_cross_attention_scratch_bytes() is
+ *    the larger of the two.
  *  - Calls no cudaMalloc, cudaFree or any other allocating routine.  The first call on a device
  *    looks up the array's device address (cudaGetSymbolAddress, with the current device, which
  *    must be the device of the stream and of the buffers); make that first call before any
@@ -288,12 +294,17 @@ PD_API pd_status pd_vocab_argmax(int32_t rows, int32_t d_model, int32_t vocab, c
  *    and overwrites the partials it reads, so stale contents of earlier calls never matter, but
  *    two calls that may overlap on the GPU (different streams, no dependency) race on it:
  *    order them on one stream or with events.
+ *  - The kernel's status word (PD_ERR_TIMEOUT when a bounded wait inside it expired) lives in
+ *    that array too, where the caller cannot read it: pd_cross_attention_static_status() copies
+ *    it to *status_out (host) after synchronising cuda_stream; it allocates nothing either.  A
+ *    non-zero status means that `out` of the last call on this device is not valid.
  * pd_static_last_error() returns the calling thread's message of the last failed
- * pd_cross_attention_static (empty after a success). */
+ * pd_cross_attention_static or pd_cross_attention_static_status (empty after a success). */
 PD_API size_t pd_cross_attention_static_max_bytes(void);
 PD_API pd_status pd_cross_attention_static(int32_t dtype, int32_t batch, int32_t rows_per_seq, int32_t n_heads,
                                     int32_t max_ctx, float attn_scale, int32_t splits, const void *q, const void *kv,
                                     const int32_t *n_rows, const int32_t *ctx_len, void *out, void *cuda_stream);
+PD_API pd_status pd_cross_attention_static_status(void *cuda_stream, int32_t *status_out);
 PD_API const char *pd_static_last_error(void);
 
 PD_API const char *pd_last_error(const pd_handle *h);

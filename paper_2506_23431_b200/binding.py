@@ -73,6 +73,7 @@ _SIGS = {
     "pd_vocab_argmax": (C.c_int, [C.c_int32] * 3 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]),
     "pd_cross_attention_static_max_bytes": (C.c_size_t, []),
     "pd_cross_attention_static": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p]),
+    "pd_cross_attention_static_status": (C.c_int, [C.c_void_p, _i32p]),
     "pd_static_last_error": (C.c_char_p, []),
     "pd_last_error": (C.c_char_p, [_H]),
     "pd_version": (C.c_char_p, []),
@@ -356,6 +357,17 @@ def cross_attention_static(q, kv, n_rows, ctx_len, attn_scale: float, splits: in
     scratch array, for callers that cannot allocate device memory.  Calls sharing a device must not
     overlap on the GPU."""
     return _attention_call("pd_cross_attention_static", q, kv, n_rows, ctx_len, attn_scale, splits, None)
+
+
+def cross_attention_static_status(device=None) -> int:
+    """Status word the last pd_cross_attention_static call on the current device left behind (0 = fine);
+    synchronises torch's current stream."""
+    import torch
+    word = C.c_int32(-99)
+    st = _lib.pd_cross_attention_static_status(C.c_void_p(torch.cuda.current_stream(device).cuda_stream), C.byref(word))
+    if st != PD_OK:
+        raise PdError(st, "pd_cross_attention_static_status", (_lib.pd_static_last_error() or b"").decode())
+    return word.value
 
 
 def cross_attention_static_max_bytes() -> int:

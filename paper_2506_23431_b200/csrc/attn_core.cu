@@ -30,7 +30,8 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
   const Dims &dm = a.dm;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x;
-  const int S = a.st.n_active[b];
+  // (the stand-alone op reads caller-written counts: clamped, so that no access leaves the tensors)
+  const int S = min(max(a.st.n_active[b], 0), min(dm.C, kMaxRows));
   const int row0 = b * dm.C;
   const int t = SELF ? a.st.hdr[HDR_STEP_T] : 0;
   const T *qbuf = (const T *)a.q;
@@ -76,7 +77,7 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
     i_max = sub_s[S - 1];                  // rows are in increasing subsequence order
     n_tiles = a.st.k[b] * dm.PPS;          // one tile per page (page_tokens <= TK)
   } else {
-    ctx_len = a.st.ctx_len[b];
+    ctx_len = min(max(a.st.ctx_len[b], 1), dm.ctx);
     n_tiles = (ctx_len + TK - 1) / TK;
   }
   for (int tile = split; tile < n_tiles; tile += a.splits) {
@@ -198,7 +199,7 @@ __global__ void attn_merge_kernel(AttnArgs a) {
   const Dims &dm = a.dm;
   int r = blockIdx.x;
   int b = r / dm.C, c = r % dm.C;
-  if (c >= a.st.n_active[b]) return;       // the attention kernel already zeroed unused rows
+  if (c >= min(a.st.n_active[b], dm.C)) return;       // the attention kernel already zeroed unused rows
   T *out = (T *)a.out;
   for (int idx = threadIdx.x; idx < dm.d; idx += blockDim.x) {
     int h = idx / kDh, dim = idx % kDh;

@@ -8,7 +8,10 @@ using namespace pd;
 
 namespace pd {
 
-size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
+// Scratch of the stand-alone op: header, arrival counters, partial results.  The flat partial records
+// of the tensor-core kernel are only reserved where that kernel can run (bf16, at most 32 rows per
+// sequence); the plain-ALU kernel needs the split-K records alone.
+size_t cross_attention_scratch_layout(int dtype, int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
                                       size_t *off_part_o, size_t *off_part_ml) {
   const size_t rows = (size_t)batch * rows_per_seq;
   size_t off = kOpHeaderBytes;
@@ -16,7 +19,8 @@ size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, 
   off += ((size_t)batch * n_heads * sizeof(int32_t) + 255) / 256 * 256;      // cleared with the header
   if (off_part_o) *off_part_o = off;
   const size_t split_bytes = rows * n_heads * splits * kDh * sizeof(float);
-  const size_t flat_bytes = cross_attn_tma_partial_bytes(kMaxCrossCtas, rows_per_seq);
+  const bool tensor_core = dtype == PD_DTYPE_BF16 && rows_per_seq <= 32;
+  const size_t flat_bytes = tensor_core ? cross_attn_tma_partial_bytes(kMaxCrossCtas, rows_per_seq) : 0;
   off += ((split_bytes > flat_bytes ? split_bytes : flat_bytes) + 255) / 256 * 256;
   if (off_part_ml) *off_part_ml = off;
   off += (rows * n_heads * splits * 2 * sizeof(float) + 255) / 256 * 256;
@@ -38,7 +42,7 @@ pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_
                                   int splits, const void *q, const void *kv, const int32_t *n_rows,
                                   const int32_t *ctx_len, void *out, void *scratch, cudaStream_t s) {
   size_t off_t = 0, off_o = 0, off_ml = 0;
-  cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, &off_t, &off_o, &off_ml);
+  cross_attention_scratch_layout(dtype, batch, rows_per_seq, n_heads, splits, &off_t, &off_o, &off_ml);
   uint8_t *base = reinterpret_cast<uint8_t *>(scratch);
   if (cudaMemsetAsync(base, 0, off_o, s) != cudaSuccess) return PD_ERR_CUDA;      // header and arrival counters
 
@@ -76,7 +80,7 @@ extern "C" {
 
 size_t pd_cross_attention_scratch_bytes(int32_t batch, int32_t rows_per_seq, int32_t n_heads, int32_t splits) {
   if (!cross_attention_args_ok(PD_DTYPE_BF16, batch, rows_per_seq, n_heads, 1, 1.f, splits)) return 0;
-  return cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr);
+  return cross_attention_scratch_layout(PD_DTYPE_BF16, batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr);   // the larger of the two types
 }
 
 pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_per_seq, int32_t n_heads, int32_t max_ctx,
@@ -86,7 +90,7 @@ pd_status pd_cross_attention(int32_t dtype, int32_t batch, int32_t rows_per_seq,
   if (!cross_attention_args_ok(dtype, batch, rows_per_seq, n_heads, max_ctx, attn_scale, splits)) return PD_ERR_ARG;
   if (reinterpret_cast<uintptr_t>(kv) % 16 != 0 || reinterpret_cast<uintptr_t>(q) % 16 != 0 ||
       reinterpret_cast<uintptr_t>(out) % 16 != 0 || reinterpret_cast<uintptr_t>(scratch) % 256 != 0) return PD_ERR_ARG;
-  if (scratch_bytes < cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr))
+  if (scratch_bytes < cross_attention_scratch_layout(dtype, batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr))
     return PD_ERR_WORKSPACE;
   return cross_attention_enqueue(dtype, batch, rows_per_seq, n_heads, max_ctx, attn_scale, splits, q, kv, n_rows, ctx_len,
                                  out, scratch, reinterpret_cast<cudaStream_t>(cuda_stream));

@@ -60,10 +60,10 @@ pd_status pd_cross_attention_static(int32_t dtype, int32_t batch, int32_t rows_p
     return fail(PD_ERR_ARG, "a size or parameter is out of range");
   if (reinterpret_cast<uintptr_t>(kv) % 16 != 0 || reinterpret_cast<uintptr_t>(q) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0)
     return fail(PD_ERR_ARG, "q, kv and out must be 16-byte aligned");
-  const size_t need = cross_attention_scratch_layout(batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr);
+  const size_t need = cross_attention_scratch_layout(dtype, batch, rows_per_seq, n_heads, splits, nullptr, nullptr, nullptr);
   if (need > kStaticScratchBytes)
     return fail(PD_ERR_WORKSPACE, "these sizes need %lld bytes of scratch; the built-in scratch holds %lld "
-                                  "(use fewer splits or pd_cross_attention with your own buffer)",
+                                  "(fewer splits, fewer sequences or rows per call, or pd_cross_attention with a buffer of your own)",
                 (long long)need, (long long)kStaticScratchBytes);
   void *scratch = nullptr;
   pd_status s = static_scratch(&scratch);
@@ -73,6 +73,21 @@ pd_status pd_cross_attention_static(int32_t dtype, int32_t batch, int32_t rows_p
   s = cross_attention_enqueue(dtype, batch, rows_per_seq, n_heads, max_ctx, attn_scale, splits, q, kv, n_rows, ctx_len, out,
                               scratch, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (s != PD_OK) return fail(s, "enqueueing the cross-attention kernels failed (pd_status %lld)", (long long)s);
+  return PD_OK;
+}
+
+pd_status pd_cross_attention_static_status(void *cuda_stream, int32_t *status_out) {
+  g_err[0] = 0;
+  if (!status_out) return fail(PD_ERR_ARG, "null pointer argument");
+  void *scratch = nullptr;
+  pd_status s = static_scratch(&scratch);
+  if (s != PD_OK) return s;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, reinterpret_cast<const int32_t *>(scratch) + HDR_STATUS, sizeof(word), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return fail(PD_ERR_CUDA, "reading the status word failed (CUDA error %lld)", (long long)e);
+  *status_out = word;
   return PD_OK;
 }
 

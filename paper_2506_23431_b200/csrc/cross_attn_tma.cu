@@ -185,9 +185,10 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
 
   // ---- tiles per head of every sequence, prefix sums, this CTA's range of the flat list
   for (int b = tid; b < batch; b += XTHREADS) {
-    const int S = a.st.n_active[b];
+    // counts the caller wrote (stand-alone op) are clamped to the tensors' extents
+    const int S = min(max(a.st.n_active[b], 0), min(dm.C, 16 * MT));
     nact_s[b] = (unsigned char)S;
-    pfx_s[b + 1] = S > 0 ? (a.st.ctx_len[b] + XK - 1) / XK : 0;
+    pfx_s[b + 1] = S > 0 ? (min(max(a.st.ctx_len[b], 1), dm.ctx) + XK - 1) / XK : 0;
   }
   if (tid == 0) {
     pfx_s[0] = 0;
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
     const int b = cur.b, h = cur.h;
     const int seg_start = H * pfx_s[b] + h * cur.nt, seg_end = seg_start + cur.nt;
     const int my_end = min(hi, seg_end);
-    const int S = nact_s[b], ctx_len = a.st.ctx_len[b];
+    const int S = nact_s[b], ctx_len = min(max(a.st.ctx_len[b], 1), dm.ctx);
     const int row0 = b * dm.C;
     uint32_t qf[MT][4][4];
 #pragma unroll

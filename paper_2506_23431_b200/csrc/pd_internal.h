@@ -157,7 +157,7 @@ cudaError_t encode_vocab_maps(CUtensorMap *map_a, CUtensorMap *map_b, const void
 cudaError_t launch_vocab_tc(const CUtensorMap &map_a, const CUtensorMap &map_b, const VocabArgs &a, cudaStream_t s);
 
 // ---- stand-alone cross-attention (attn_ops.cu) ---------------------------------------------
-size_t cross_attention_scratch_layout(int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
+size_t cross_attention_scratch_layout(int dtype, int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
                                       size_t *off_part_o, size_t *off_part_ml);
 bool cross_attention_args_ok(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale, int splits);
 pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_heads, int max_ctx, float attn_scale,

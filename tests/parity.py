@@ -34,11 +34,14 @@ def _margin(logits: np.ndarray, barred: Sequence[int]) -> float:
 
 
 def replay_compare(dec, wl: W.Workload, mem_dev, ctx_len, forced_len, runs: Dict[int, dict],
-                   tol: Optional[float] = None, max_steps: Optional[int] = None) -> dict:
+                   tol: Optional[float] = None, max_steps: Optional[int] = None, use_logits: bool = True) -> dict:
     """Teacher-forced replay: the library consumes the oracle's appended tokens on the rows the
     oracle decoded (other rows run free), so every step's logits stay comparable.  Asserts:
     active sets bit-exact, logits within tol, own greedy choice equal where the oracle's margin
     exceeds MARGIN, and at the end streams / lengths / flags / steps / trace identical.
+    With use_logits = False (a decoder that keeps its logits on chip, as the benchmark runs it)
+    the logits are not read; everything else - active sets per step, the library's own choices
+    under the margin rule, streams, lengths, flags, steps, trace - is compared all the same.
     Returns statistics (max error, compared logits, compared / skipped choices)."""
     import torch
     tol = TOL[wl.dtype] if tol is None else tol
@@ -56,7 +59,7 @@ def replay_compare(dec, wl: W.Workload, mem_dev, ctx_len, forced_len, runs: Dict
                 for i, tok in r["trace"][t - 1]["appended"].items():
                     teacher[b, i - 1] = tok
         dec.step(torch.from_numpy(teacher).to(dec.device))
-        need_logits = any(t <= r["steps"] for r in runs.values())
+        need_logits = use_logits and any(t <= r["steps"] for r in runs.values())
         logits, row_sub = dec.get_logits(want_logits=need_logits)
         if need_logits:
             logits = logits.reshape(batch, dec.rows_per_seq, wl.vocab)
@@ -67,7 +70,7 @@ def replay_compare(dec, wl: W.Workload, mem_dev, ctx_len, forced_len, runs: Dict
             step = r["trace"][t - 1]
             act = [int(i) for i in row_sub[b] if i > 0]
             assert act == step["active"], f"row {b} step {t}: active {act} vs oracle {step['active']}"
-            for c, i in enumerate(act):
+            for c, i in enumerate(act if use_logits else []):
                 ref = step["logits"][c]
                 err = float(np.abs(logits[b, c].astype(np.float64) - ref).max())
                 stats["max_err"] = max(stats["max_err"], err)

@@ -75,6 +75,33 @@ def test_cross_attention_kernel_against_oracle(dtype, batch, rows, heads, ctx, s
     assert err <= tol, f"max abs error {err:.3e} > {tol:g}"
 
 
+@pytest.mark.parametrize("dtype,rows", [("bf16", 6), ("fp32", 6), ("bf16", 36)])
+def test_cross_attention_clamps_counts_it_reads_from_the_device(dtype, rows):
+    """Row counts and context lengths are device arrays the host wrapper cannot check.  Values beyond
+    the tensors' extents are clamped where they are read: the sequence is computed with rows_per_seq rows
+    and max_ctx positions, and nothing outside its own rows of `out` changes.  (The bad values sit on
+    sequence 0 of a larger allocation, so even an unclamped kernel would stay inside allocated memory.)"""
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    batch, heads, ctx = 3, 2, 150
+    q, kv, n_rows, ctx_len = cross_case(31, batch, rows, heads, ctx, dtype, poison=False)
+    n_rows[:] = [rows, rows - 2, rows]
+    ctx_len[:] = [ctx, ctx - 17, ctx]
+    ref = oracle_cross(q, kv, n_rows, ctx_len, heads, 0.125)
+    bad_rows, bad_ctx = n_rows.copy(), ctx_len.copy()
+    bad_rows[0], bad_ctx[0] = rows + 9, ctx + 1000
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev = torch.device("cuda", 0)
+    q_d, kv_d = torch.from_numpy(q).to(dev, td), torch.from_numpy(kv).to(dev, td)
+    # the call sees the first two sequences of the three allocated
+    out = B.cross_attention(q_d[:2], kv_d[:2], torch.from_numpy(bad_rows[:2]).to(dev), torch.from_numpy(bad_ctx[:2]).to(dev), 0.125, 2)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().astype(np.float64)
+    tol = 1e-2 if dtype == "bf16" else 2e-5
+    assert np.abs(got - ref[:2]).max() <= tol
+    assert not got[1, n_rows[1]:].any()
+
+
 def test_cross_attention_rejects_bad_arguments():
     import ctypes as C
     import torch

@@ -320,14 +320,70 @@ def test_two_identical_decodes_give_identical_logits():
 
 
 FULL = [("bart_base", 2e-2), ("long_context", 2e-2), ("summarisation", 2e-2), ("keyphrase", 2e-2)]
+_ORACLE_CACHE = {}
+
+
+def full_size_case(name, ragged):
+    """Weights, encoder memory, lengths and the oracle's decode of batch rows 0 and B-1 of a full-size
+    configuration; computed once per session (the oracle needs some seconds per row)."""
+    key = (name, ragged)
+    if key not in _ORACLE_CACHE:
+        wl = W.CONFIGS[name]
+        weights, mem = W.make_weights(wl), W.make_encoder_memory(wl)
+        ctx_len, fl = W.make_ctx_len(wl, ragged=ragged), W.make_forced_len(wl)
+        rows = sorted({0, wl.batch - 1})
+        runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, fl)
+        _ORACLE_CACHE[key] = (wl, weights, mem, ctx_len, fl, runs)
+    return _ORACLE_CACHE[key]
+
+
+@pytest.mark.parametrize("store_logits", [True, False])
+@pytest.mark.parametrize("name,tol", FULL)
+def test_full_size_configs_on_sampled_rows(name, tol, store_logits):
+    """The four bf16 configurations at full size, in the launch configuration the benchmark times
+    (CUDA graph, automatic splits); the oracle decodes batch rows 0 and B-1.  store_logits = False is
+    the mode the benchmark runs: the logits never leave the vocabulary kernel, so the replay compares
+    the active sets of every step, the library's own greedy choices under the margin rule, streams,
+    lengths, flags, steps and the trace; store_logits = True adds the logits element by element."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl, weights, mem, ctx_len, fl, runs = full_size_case(name, False)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, store_logits=store_logits)
+    mem_dev = dec.device_memory(mem)
+    s = parity.replay_compare(dec, wl, mem_dev, ctx_len, fl, runs, use_logits=store_logits)
+    assert s["choices"] > 0 and s["max_err"] <= tol
+    assert (s["logits"] > 0) == store_logits
+    parity.free_run_compare(dec, wl, mem_dev, ctx_len, fl, runs)
+    dec.close()
+    print(f"{name} store_logits={store_logits}: max logit error {s['max_err']:.3e} over {s['logits']} logits, "
+          f"{s['choices']} choices compared, {s['low_margin']} below margin")
 
 
 @pytest.mark.parametrize("name,tol", FULL)
-def test_full_size_configs_on_sampled_rows(name, tol):
-    """The four bf16 configurations at full size, in the launch configuration the benchmark
-    times (CUDA graph, automatic splits); the oracle decodes batch rows 0 and B-1."""
-    wl = W.CONFIGS[name]
-    s = check(wl, rows=[0, wl.batch - 1], free_run=True)
-    assert s["max_err"] <= tol
-    print(f"{name}: max logit error {s['max_err']:.3e} over {s['logits']} logits, "
-          f"{s['choices']} choices compared, {s['low_margin']} below margin")
+def test_full_size_configs_with_ragged_contexts(name, tol):
+    """Full size again with context lengths drawn from [L/2, L] per sequence (ragged last tiles, unequal
+    (sequence, head) segments in cross-attention), logits kept on chip as in the benchmark."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl, weights, mem, ctx_len, fl, runs = full_size_case(name, True)
+    assert (ctx_len < wl.ctx).any()
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, store_logits=False)
+    s = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs, use_logits=False)
+    assert s["choices"] > 0
+    dec.close()
+
+
+@pytest.mark.parametrize("store_logits", [True, False])
+def test_bf16_sequential_decoder_shape_of_the_benchmark(store_logits):
+    """sub_max = 1 on the concatenated targets - the workload `bench.py` times as the sequential decoder -
+    on the bf16 tensor-core kernels: one long subsequence per sequence, page lists of twenty and more pages."""
+    import bench
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    base = W.CONFIGS["bart_base"]
+    swl, sfl = bench.sequential_workload(base, W.make_forced_len(base))
+    assert swl.sub_max == 1 and swl.max_sub_len >= 100
+    weights, mem, ctx_len = W.make_weights(swl), W.make_encoder_memory(swl), W.make_ctx_len(swl)
+    rows = [0, int(np.argmax(sfl[:, 0]))]            # row 0 and the longest stream
+    runs = parity.oracle_runs(swl, weights, {b: mem[b] for b in rows}, ctx_len, sfl)
+    dec = PipelinedDecoder(swl.hyper(), weights, swl.batch, store_logits=store_logits)
+    s = parity.replay_compare(dec, swl, dec.device_memory(mem), ctx_len, sfl, runs, use_logits=store_logits)
+    assert s["choices"] > 0 and s["max_err"] <= 2e-2
+    dec.close()
