@@ -270,6 +270,37 @@ PD_API pd_status pd_vocab_argmax(int32_t rows, int32_t d_model, int32_t vocab, c
                                  int32_t *best_id, float *best_val, float *logits, void *scratch, size_t scratch_bytes,
                                  void *cuda_stream);
 
+/* One linear layer of the decoder stack alone (Section 3.2, Eq. 3: the Decoder is a stacked transformer
+ * decoder; every projection in it - Q/K/V, attention output, feed-forward - is  y = x W  on the step's few
+ * hundred active rows), on caller-supplied tensors and without a handle: the tcgen05 kernel pd_step uses
+ * for the bf16 projections, with the work around the product fused into it.
+ *   rows, d_in, d_out   rows >= 1; d_in a multiple of 64; d_out a multiple of 16
+ *   a          device bf16 [rows, d_in], 16-byte aligned: the layer's input.  When it is the
+ *              un-normalised RMSNorm input times the norm's gain, pass row_sumsq
+ *   w          device bf16 [d_in, d_out] row-major (y = x W), 16-byte aligned
+ *   row_sumsq  device fp32 [rows] or NULL: sum over d_in of the squared norm inputs of every row; the
+ *              product's row m is then scaled by rsqrt(row_sumsq[m] / d_in + eps) (the norm applied after
+ *              the product instead of before it)
+ *   mode 0     out (device bf16 [rows, d_out]) = a W (scaled);  mode 1: the same through max(., 0)
+ *   mode 2     residual form: x (device fp32 [rows, d_out], in and out) += a W;  xg (device bf16
+ *              [rows, d_out]) = x * gain_next (device bf16 [d_out]), the next layer's GEMM input;
+ *              sumsq_out (device fp32 [*sumsq_parts, rows], or NULL): partial sums over column slices of
+ *              the new x squared - their sum over the parts is the next norm's row_sumsq
+ *   sumsq_parts host int32 out or NULL: number of parts the kernel writes for this shape on the current
+ *              device (pd_linear_sumsq_parts(d_in, d_out) gives it beforehand, to size sumsq_out)
+ *   scratch    device, 256-byte aligned, at least pd_linear_scratch_bytes(d_in, d_out): a 256-byte header
+ *              (int32 word 2 receives PD_ERR_TIMEOUT if a bounded wait inside the kernel expired; cleared
+ *              by the call), then the weight re-laid as [d_out, d_in] (the decoder does this once per
+ *              handle, the stand-alone call every time)
+ * Enqueues on cuda_stream and returns; allocates nothing on the device; the caller owns every buffer.
+ * PD_ERR_ARG for null pointers, misaligned buffers or unsupported sizes, PD_ERR_WORKSPACE for a scratch
+ * that is too small, PD_ERR_CUDA if a launch fails. */
+PD_API size_t pd_linear_scratch_bytes(int32_t d_in, int32_t d_out);
+PD_API int32_t pd_linear_sumsq_parts(int32_t d_in, int32_t d_out);
+PD_API pd_status pd_linear(int32_t rows, int32_t d_in, int32_t d_out, int32_t mode, const void *a, const void *w,
+                           const float *row_sumsq, float eps, void *out, float *x, const void *gain_next, void *xg,
+                           float *sumsq_out, int32_t *sumsq_parts, void *scratch, size_t scratch_bytes, void *cuda_stream);
+
 /* pd_cross_attention without a scratch argument (an addition of this library; the paper has no
  * counterpart).  Some callers have no way to obtain device memory at the moment they need the
  * op: a plug-in that runs inside a host framework which owns the whole device heap and hands

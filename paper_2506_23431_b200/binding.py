@@ -71,6 +71,10 @@ _SIGS = {
                                                                                                   C.c_void_p]),
     "pd_vocab_argmax_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
     "pd_vocab_argmax": (C.c_int, [C.c_int32] * 3 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]),
+    "pd_linear_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
+    "pd_linear_sumsq_parts": (C.c_int32, [C.c_int32, C.c_int32]),
+    "pd_linear": (C.c_int, [C.c_int32] * 4 + [C.c_void_p] * 3 + [C.c_float] + [C.c_void_p] * 5 + [_i32p, C.c_void_p, C.c_size_t,
+                                                                                                C.c_void_p]),
     "pd_cross_attention_static_max_bytes": (C.c_size_t, []),
     "pd_cross_attention_static": (C.c_int, [C.c_int32] * 5 + [C.c_float, C.c_int32] + [C.c_void_p] * 5 + [C.c_void_p]),
     "pd_cross_attention_static_status": (C.c_int, [C.c_void_p, _i32p]),
@@ -396,6 +400,41 @@ def vocab_argmax(hidden, lm_head, want_logits: bool = False, scratch=None):
     if st != 0:
         raise PdError(st, "pd_vocab_argmax")
     return best_id, best_val, logits
+
+
+def linear(a, w, mode: int = 0, row_sumsq=None, eps: float = 1e-6, x=None, gain_next=None):
+    """pd_linear on torch CUDA tensors: a bf16 [rows, d_in], w bf16 [d_in, d_out].  mode 0 / 1: returns out
+    bf16 [rows, d_out] (1 = through ReLU).  mode 2 (residual): x fp32 [rows, d_out] is updated in place;
+    returns (xg bf16 [rows, d_out], sumsq fp32 [parts, rows]).  Runs on torch's current stream."""
+    import torch
+    if a.dtype != torch.bfloat16 or w.dtype != torch.bfloat16:
+        raise ValueError("a and w must be bfloat16")
+    a, w = a.contiguous(), w.contiguous()
+    rows, d_in = a.shape
+    d_out = w.shape[1]
+    dev = a.device
+    n = int(_lib.pd_linear_scratch_bytes(d_in, d_out))
+    scratch = torch.empty(max(n, 256), dtype=torch.uint8, device=dev)
+    out = xg = ssq = None
+    parts = C.c_int32(0)
+    if mode == 2:
+        xg = torch.empty(rows, d_out, dtype=torch.bfloat16, device=dev)
+        ssq = torch.full((max(1, int(_lib.pd_linear_sumsq_parts(d_in, d_out))), rows), float("nan"), dtype=torch.float32, device=dev)
+    else:
+        out = torch.empty(rows, d_out, dtype=torch.bfloat16, device=dev)
+    ptr = lambda t: None if t is None else C.c_void_p(t.data_ptr())
+    st = _lib.pd_linear(rows, d_in, d_out, mode, ptr(a), ptr(w), ptr(row_sumsq), C.c_float(eps), ptr(out), ptr(x), ptr(gain_next),
+                        ptr(xg), ptr(ssq), C.byref(parts), ptr(scratch), scratch.numel(),
+                        C.c_void_p(torch.cuda.current_stream(dev).cuda_stream))
+    if st != 0:
+        raise PdError(st, "pd_linear")
+    torch.cuda.current_stream(dev).synchronize()
+    status = int(scratch[:16].view(torch.int32)[2].item())
+    if status != 0:
+        raise PdError(status, "pd_linear (device status)")
+    if mode == 2:
+        return xg, ssq[: parts.value]
+    return out
 
 
 def version() -> str:

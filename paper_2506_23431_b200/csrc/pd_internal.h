@@ -156,6 +156,42 @@ cudaError_t encode_vocab_maps(CUtensorMap *map_a, CUtensorMap *map_b, const void
                               uint64_t vocab, uint64_t K, int *driver_code);
 cudaError_t launch_vocab_tc(const CUtensorMap &map_a, const CUtensorMap &map_b, const VocabArgs &a, cudaStream_t s);
 
+// ---- skinny-M linear layers on tcgen05 (linear_tc.cu) --------------------------------------------
+enum { LIN_EPI_STORE = 0,   // out = bf16(acc * row_scale)
+       LIN_EPI_RELU = 1,    // out = bf16(max(acc * row_scale, 0))
+       LIN_EPI_RESID = 2,   // x += acc (fp32 residual stream); xg = bf16(x * gain_next); partial sums of x^2 per row
+       LIN_EPI_QKV = 3 };   // q | k | v columns: scale, rotary positions (optional), q to its buffer, k and v to the row's cache slot
+struct LinearArgs {
+  int K, N;                  // the weight is [N][K] (K contiguous)
+  int BN, ksplit;            // columns per CTA; CTAs (one cluster) along K
+  const int32_t *rows_dev;   // device word holding the number of packed rows, or null
+  int rows_fixed;            // number of rows when rows_dev is null
+  int rows_cap;              // rows the row-indexed buffers are allocated for
+  int rows_per_cta;          // rows per CTA along grid.z (a multiple of 32; CTAs beyond the row count leave at once)
+  int epi;                   // LIN_EPI_*
+  // row scale of the RMSNorm in front of the layer (null: none): rsqrt(sum_p ssq_in[p][m] * inv_width + eps)
+  const float *ssq_in; int parts_in; float inv_width, eps;
+  __nv_bfloat16 *out;        // STORE / RELU: [rows][N]
+  float *x;                  // RESID: fp32 [rows][N], read and written
+  __nv_bfloat16 *xg;         // RESID: bf16 [rows][N] = x * gain_next (input of the next layer's GEMM)
+  const __nv_bfloat16 *gain_next;  // RESID: [N]
+  float *ssq_out;            // RESID: [(N / BN) * ksplit][rows_cap] partial sums of squares of the new x, or null
+  // QKV
+  __nv_bfloat16 *q_out, *kv_pool;
+  const int4 *prow_meta;     // per packed row: (page, slot, position tau + i, subsequence)
+  const float2 *rope_tab;
+  int layer, pool, H, P, d, rope;
+  int32_t *status;           // error word (PD_ERR_TIMEOUT on an expired wait)
+};
+int linear_tc_smem_bytes();
+bool linear_tc_plan(int N, int K, int sms, int *BN_out, int *ksplit_out);
+cudaError_t linear_tc_prepare();         // once per device, outside any stream capture
+struct LinearActMaps { CUtensorMap full, part; };   // boxes of 128 rows and of 32 rows over the same activations
+cudaError_t encode_linear_act_maps(LinearActMaps *out, const void *act, uint64_t rows, uint64_t K, int *driver_code);
+cudaError_t encode_linear_weight_map(CUtensorMap *out, const void *w_nk, uint64_t N, uint64_t K, int BN, int *driver_code);
+cudaError_t launch_linear_tc(const LinearActMaps &map_a, const CUtensorMap &map_w, const LinearArgs &a, bool pdl, cudaStream_t s);
+cudaError_t launch_transpose_bf16(int K, int N, const void *w, void *wt, cudaStream_t s);
+
 // ---- stand-alone cross-attention (attn_ops.cu) ---------------------------------------------
 size_t cross_attention_scratch_layout(int dtype, int batch, int rows_per_seq, int n_heads, int splits, size_t *off_tickets,
                                       size_t *off_part_o, size_t *off_part_ml);

@@ -246,3 +246,71 @@ def test_cross_attention_random_ragged_shapes(seed, batch, rows, heads, ctx):
     assert np.abs(got - ref).max() <= 1e-2
     for o in outs[1:]:
         assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))
+
+
+LINEAR_SHAPES = [
+    # rows, d_in, d_out: the decoder's projection shapes (square, Q/K/V, feed-forward up and down) at both
+    # model widths, and row counts on both sides of the 128-row tiles and of the accumulators one pass holds
+    (134, 1024, 1024), (1, 1024, 3072), (300, 1024, 4096), (129, 4096, 1024),
+    (576, 768, 768), (97, 768, 2304), (260, 768, 3072), (64, 3072, 768),
+    (700, 256, 512), (5, 64, 16),
+]
+
+
+@pytest.mark.parametrize("rows,d_in,d_out", LINEAR_SHAPES)
+def test_linear_kernel_against_oracle_product(rows, d_in, d_out):
+    """The tcgen05 projection kernel against the fp64 product of the same bf16 inputs, in its three
+    epilogues: plain (with the RMSNorm scale applied after the product), ReLU, and the residual form
+    that also leaves the next norm's inputs.  Tolerance: bf16 output rounding (2^-9 relative) plus fp32
+    accumulation over d_in terms."""
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    g = np.random.Generator(np.random.Philox(key=np.array([rows, d_in + d_out], dtype=np.uint64)))
+    a = W.bf16_round(g.standard_normal((rows, d_in), dtype=np.float32))
+    w = W.bf16_round(0.05 * g.standard_normal((d_in, d_out), dtype=np.float32))
+    gain = W.bf16_round(1.0 + 0.1 * g.standard_normal(d_out, dtype=np.float32))
+    x0 = g.standard_normal((rows, d_out), dtype=np.float32)
+    ssq_in = (g.random(rows, dtype=np.float32) + 0.5) * d_in
+    eps = 1e-6
+    ref = a.astype(np.float64) @ w.astype(np.float64)
+    inv = 1.0 / np.sqrt(ssq_in.astype(np.float64) / d_in + eps)
+    dev = torch.device("cuda", 0)
+    a_d, w_d = torch.from_numpy(a).to(dev, torch.bfloat16), torch.from_numpy(w).to(dev, torch.bfloat16)
+    scale = max(1.0, np.abs(ref).max())
+
+    out = B.linear(a_d, w_d, mode=0).float().cpu().numpy().astype(np.float64)
+    assert np.abs(out - ref).max() <= 2.0 ** -8 * scale
+
+    out = B.linear(a_d, w_d, mode=1, row_sumsq=torch.from_numpy(ssq_in).to(dev), eps=eps).float().cpu().numpy().astype(np.float64)
+    want = np.maximum(ref * inv[:, None], 0.0)
+    assert np.abs(out - want).max() <= 2.0 ** -8 * max(1.0, np.abs(want).max())
+
+    x_d = torch.from_numpy(x0).to(dev)
+    outs = []
+    for _ in range(2):                                  # twice: the result must repeat bit for bit
+        x_d.copy_(torch.from_numpy(x0).to(dev))
+        xg, ssq = B.linear(a_d, w_d, mode=2, x=x_d, gain_next=torch.from_numpy(gain).to(dev, torch.bfloat16))
+        outs.append((x_d.clone(), xg.clone(), ssq.clone()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1].view(torch.int16), outs[1][1].view(torch.int16))
+    x_new = outs[0][0].cpu().numpy().astype(np.float64)
+    want_x = x0.astype(np.float64) + ref
+    assert np.abs(x_new - want_x).max() <= 1e-4 * max(1.0, np.abs(want_x).max())
+    xg = outs[0][1].float().cpu().numpy().astype(np.float64)
+    want_g = want_x * gain.astype(np.float64)[None, :]
+    assert np.abs(xg - want_g).max() <= 2.0 ** -8 * max(1.0, np.abs(want_g).max())
+    ssq = outs[0][2].cpu().numpy().astype(np.float64)
+    assert np.isfinite(ssq).all()
+    want_s = (want_x ** 2).sum(axis=1)
+    assert np.abs(ssq.sum(axis=0) - want_s).max() <= 1e-4 * want_s.max()
+
+
+def test_linear_rejects_bad_arguments():
+    import torch
+    from paper_2506_23431_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    a = torch.zeros(4, 96, device=dev, dtype=torch.bfloat16)            # d_in not a multiple of 64
+    w = torch.zeros(96, 64, device=dev, dtype=torch.bfloat16)
+    with pytest.raises(B.PdError) as e:
+        B.linear(a, w)
+    assert e.value.status == -1
+    assert B._lib.pd_linear_scratch_bytes(64, 8) == 0
