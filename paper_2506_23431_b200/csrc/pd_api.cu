@@ -291,15 +291,26 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.rel_buckets = h->cfg.rel_buckets;
   a.tickets = h->ptr<int32_t>(h->lay.state) + h->lay.w_xtick;
   a.bias_tab = h->cfg.pos_mode == PD_POS_T5_BIAS ? h->ptr<float>(h->lay.bias_tab) : nullptr;
+  a.qkv = h->ptr<void>(h->lay.qkv);
+  a.qkv_f32 = h->cfg.pos_mode == PD_POS_ROPE ? 1 : 0;      // the projection rounds to bf16 itself when nothing is rotated
+  a.rope_tab = h->cfg.pos_mode == PD_POS_ROPE ? h->ptr<float2>(h->lay.rope_tab) : nullptr;
   return a;
 }
 
-// Pipelined self-attention of one layer (attention kernel + split-K merge when split).
+bool self_tc(const pd_handle *h) { return h->cfg.dtype == PD_DTYPE_BF16 && self_attn_tc_supported(h->dm); }
+
+// Pipelined self-attention of one layer.  The tensor-core kernel appends the step's keys/values itself and
+// merges its splits in the same launch; the plain-ALU kernel follows the append kernel and, when split,
+// is followed by the merge kernel.
 pd_status enqueue_self_attention(pd_handle *h, int layer) {
   const int dt = h->cfg.dtype;
   AttnArgs a = attn_args(h, layer, true);
-  if (dt == PD_DTYPE_BF16 && self_attn_tc_supported(h->dm)) CU_TRY(h, launch_self_attn_tc(a, h->stream));
-  else CU_TRY(h, launch_attn_core(a, dt, true, h->stream));
+  if (self_tc(h)) {
+    CU_TRY(h, launch_self_attn_tc(a, h->stream));
+    h->own_launches++;
+    return PD_OK;
+  }
+  CU_TRY(h, launch_attn_core(a, dt, true, h->stream));
   h->own_launches++;
   if (a.splits > 1) { CU_TRY(h, launch_attn_merge(a, dt, h->stream)); h->own_launches++; }
   return PD_OK;
@@ -336,7 +347,11 @@ pd_status enqueue_step(pd_handle *h) {
   for (int l = 0; l < dm.L; ++l) {
     const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
     OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
-    if (dt == PD_DTYPE_BF16 && dm.pos_mode != PD_POS_ROPE) {
+    if (self_tc(h)) {
+      // the attention kernel takes queries, keys and values straight from the projection's output and
+      // appends the new cache entries itself (bf16 from the projection when nothing is rotated)
+      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, dm.pos_mode == PD_POS_ROPE, 0.f));
+    } else if (dt == PD_DTYPE_BF16 && dm.pos_mode != PD_POS_ROPE) {
       // nothing to rotate: the projection rounds to bf16 itself and the append only places the rows
       PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, false, 0.f));
       OWN(h, PD_PROF_APPEND, launch_append_copy_bf16(dm, h->st, h->batch, l, qkv, h->ptr<void>(h->lay.qbuf),
@@ -581,14 +596,7 @@ pd_status encode_prepare(pd_handle *h, const int32_t *ctx_len, int32_t batch, co
   const int bh = batch * dm.H;
   int ss = h->cfg.self_splits > 0 ? h->cfg.self_splits : cdiv(2 * 148, bh);
   if (ss > 8 && h->cfg.self_splits == 0) ss = 8;
-  if (h->cfg.self_splits == 0 && h->cfg.dtype == PD_DTYPE_BF16 && self_attn_tc_supported(dm)) {
-    // The tensor-core kernel works through a page in well under a microsecond per warp, while a split
-    // costs a second launch for the merge (about 6 us): split only when a sequence's page list can get
-    // so long that an unsplit warp would walk more than 16 pages, and never beyond one wave of CTAs.
-    ss = cdiv(dm.SM * dm.PPS, 4 * 16);
-    while (ss > 1 && bh * ss > 2 * 148) --ss;
-    if (ss > 8) ss = 8;
-  }
+  if (h->cfg.self_splits == 0 && self_tc(h)) ss = self_attn_tc_splits(dm, bh, h->cross_ctas / 2);   // the kernel uses as many of them as the lists need
   int cs = h->cfg.cross_splits;
   if (cs == 0) {
     int tiles = cdiv(dm.ctx, 128);

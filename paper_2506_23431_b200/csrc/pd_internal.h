@@ -95,7 +95,12 @@ struct AttnArgs {
   const float *rel_bias;       // [H, rel_buckets]
   int rel_buckets;
   const float *bias_tab;       // [H, n_dist]: rel_bias[h][bucket(dist)] * log2(e), or null
-  int32_t *tickets;            // cross-attention: one arrival counter per (sequence, head), zero between launches
+  int32_t *tickets;            // one arrival counter per (sequence, head), zero between launches
+  // tensor-core self-attention (the step's KV-append happens inside it): the projection's output
+  // [rows][3 d] (bf16, or fp32 when qkv_f32), and the (cos, sin) table in rotary mode (else null)
+  const void *qkv;
+  int qkv_f32;
+  const float2 *rope_tab;
 };
 
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
@@ -124,6 +129,7 @@ int cross_attn_ctas();                  // 2 x SM count of the current device, c
 cudaError_t launch_build_bias_table(const Dims &dm, const float *rel_bias, int rel_buckets, const int32_t *dist_bucket,
                                     float *bias_tab, cudaStream_t s);
 bool self_attn_tc_supported(const Dims &dm);
+int self_attn_tc_splits(const Dims &dm, int pairs, int sms);
 cudaError_t self_attn_tc_prepare();     // once per device, outside any stream capture
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s);
 cudaError_t launch_argmax_sched(const Dims &dm, const DecState &st, int batch, const float *logits,

@@ -1,7 +1,9 @@
 // Pipelined self-attention for bf16 storage (sm_100a): decode attention of all active
 // subsequences of a sequence over the paged per-subsequence KV cache, with the dependency rule
 // of Section 3.2 (a query of subsequence i sees subsequences i' <= i as generated so far)
-// evaluated per page from (subsequence, first position) metadata - no mask is ever stored.
+// evaluated per page from (subsequence, first position) metadata - no mask is ever stored -
+// and the step's KV-append with its positional write (Eq. 2: the entry's position is tau + i)
+// done by the same launch.
 //
 // All S active rows of a sequence share its cache, so one key/value block serves up to S
 // queries: with S around 8-16 the scores are far too many flops for the plain ALUs to keep
@@ -10,25 +12,38 @@
 //
 // The scheduler leaves, once per step, a list of the sequence's pages (page, entries, subsequence,
 // first position) that every layer and head reuses.  One CTA = one (split, head, sequence); each of
-// its warps is an independent worker that takes every W-th page of the list (W = splits * warps),
-// copies exactly the entries that exist - one contiguous run, key row and value row per entry -
-// into its private two-slot ring with 16-byte cp.async (these blocks are a few KB and scattered:
-// per-lane async copies have no per-request engine cost and need no barrier object) and keeps its
-// own online-softmax state over all keys of the page at once.  Pages are stored pre-swizzled
-// (16-byte chunk c of a row of entry e at chunk c ^ (e & 7)), so a linear copy lands in the
-// bank-conflict-free layout ldmatrix wants.  The warps' partials are
-// merged through shared memory, the splits by the merge kernel.  Nothing in the kernel waits on
-// another warp's progress except the two CTA barriers of prologue and epilogue.
+// its warps is an independent worker that takes every W-th BATCH of the list (32 keys: two 16-token
+// pages, or one 32-token page; W = splits in use * warps), copies exactly the entries that exist -
+// one contiguous run per page, key row and value row per entry - into its private two-slot ring
+// with 16-byte cp.async and runs scores, softmax and P.V over the whole batch at once (twice the
+// independent tensor-core work per dependent chain of a single page).  Pages are stored
+// pre-swizzled (16-byte chunk c of a row of entry e at chunk c ^ (e & 7)), so a linear copy lands
+// in the bank-conflict-free layout ldmatrix wants.
+//
+// Fused append: the entry a row feeds at this step is the last one of its subsequence's last page
+// and is not in the cache yet.  The warp that meets that page takes the row's key and value of this
+// head straight from the projection's output (rotating the key by the position tau + i in rotary
+// mode), puts them into its ring slot AND into the cache - every (page, head) block is met by
+// exactly one warp of the launch, so the cache is written once, without a race, and no separate
+// append launch exists.  Queries come from the same projection output (rotated likewise).
+//
+// Splits: the number of splits in use follows the list's length (a CTA whose split is not needed
+// leaves at once).  Warps merge through shared memory; split CTAs leave a partial record, take a
+// ticket, and the last one to arrive merges the records in split order (deterministic) and writes
+// the output - no merge launch, and no CTA ever waits for another.
 #include "pd_internal.h"
 
 namespace pd {
 
 constexpr int SW = 4;                      // worker warps per CTA
 constexpr int STHREADS = SW * 32;
-constexpr int SDEPTH = 2;                  // ring slots per warp: the page in use and the next one
+constexpr int SDEPTH = 2;                  // ring slots per warp: the batch in use and the next one
+constexpr int SKEYS = 16;                  // keys per batch: one 16-token page (a 32-token page is a batch of its own)
 constexpr int SMAXLIST = 256;              // page-list entries of one sequence held in shared memory
 constexpr int SMAXDIST = 512;
-constexpr int SMROW = kDh + 8;               // row stride of the merge scratch in floats (spreads the eight fragment rows over the banks)
+constexpr int SMROW = kDh + 8;             // row stride of the merge scratch in floats (spreads the eight fragment rows over the banks)
+constexpr int SBATCHES_PER_WARP = 3;       // batches a warp should get before another split is used
+constexpr int SBIAS_PER_THREAD = (SMAXDIST + STHREADS - 1) / STHREADS;
 
 __device__ __forceinline__ uint32_t s_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 // 16-byte asynchronous copy global -> shared
@@ -37,6 +52,7 @@ __device__ __forceinline__ void s_cp_async16(uint32_t dst, const void *src) {
 }
 __device__ __forceinline__ void s_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void s_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void s_st_shared_u32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
 __device__ __forceinline__ void s_ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -61,31 +77,48 @@ __device__ __forceinline__ uint32_t s_pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
-// Byte offset of 16-byte chunk `chunk` of entry `row`'s key row inside a block (256 bytes per
-// entry: swizzled key row, then swizzled value row at + 128).
+// Byte offset of 16-byte chunk `chunk` of key row `row` inside a batch slot (256 bytes per entry:
+// swizzled key row, then swizzled value row at + 128).  Pages are 16 or 32 entries, so the
+// swizzle phase (row & 7) of an entry is the same in the slot as in its page.
 __device__ __forceinline__ uint32_t s_swz(int row, int chunk) { return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4)); }
 
-// All lanes: copy the nv existing entries of one (page, head) block - nv * 256 contiguous bytes,
-// key row then value row per entry - into a ring slot.
+// All lanes: copy the first n entries of one (page, head) block - n * 256 contiguous bytes, key row
+// then value row per entry - to `dst`.
 template <int P>
-__device__ __forceinline__ void s_fetch_page(uint32_t slot, const __nv_bfloat16 *blk, int nv, int lane) {
+__device__ __forceinline__ void s_fetch_run(uint32_t dst, const __nv_bfloat16 *blk, int n, int lane) {
   const uint8_t *src = reinterpret_cast<const uint8_t *>(blk) + lane * 16;
-  const uint32_t dst = slot + lane * 16;
-  const int nchunks = nv * 16;                   // 16-byte chunks of the run
+  const int nchunks = n * 16;                    // 16-byte chunks of the run
 #pragma unroll
   for (int k = 0; k < P / 2; ++k)                // P * 16 chunks over 32 lanes
-    if (k * 32 + lane < nchunks) s_cp_async16(dst + k * 512, src + k * 512);
+    if (k * 32 + lane < nchunks) s_cp_async16(dst + lane * 16 + k * 512, src + k * 512);
+}
+
+// Query fragment word (two consecutive columns of row r) from the projection's output; rotary mode
+// rotates the pair by the row's position.
+__device__ __forceinline__ uint32_t s_load_q(const AttnArgs &a, size_t row, int col_in_head, int h, int pos) {
+  const size_t off = row * 3 * (size_t)a.dm.d + (size_t)h * kDh + col_in_head;
+  if (!a.qkv_f32) return *reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(a.qkv) + off);
+  float2 v = *reinterpret_cast<const float2 *>(reinterpret_cast<const float *>(a.qkv) + off);
+  if (a.rope_tab != nullptr) {
+    const float2 c = a.rope_tab[(size_t)pos * (kDh / 2) + col_in_head / 2];
+    const float t = v.x * c.x - v.y * c.y;
+    v.y = v.x * c.y + v.y * c.x; v.x = t;
+  }
+  return s_pack_bf16(v.x, v.y);
 }
 
 template <int MT, int P>   // MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens
-__global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
-  constexpr int NT = P / 8;                // 8-key score tiles per page
-  constexpr int KS = P / 16;               // 16-key steps of P.V per page
-  constexpr uint32_t SLOT = 2u * P * 128u; // keys + values of one page of one head
+__global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel(AttnArgs a) {
+  constexpr int BK = P > SKEYS ? P : SKEYS; // keys per batch
+  constexpr int PB = BK / P;               // pages per batch
+  constexpr int NT = BK / 8;               // 8-key score tiles per batch
+  constexpr int KS = BK / 16;              // 16-key steps of P.V per batch
+  constexpr uint32_t SSLOT = BK * 256u;    // keys + values of one batch of one head
   extern __shared__ __align__(128) uint8_t s_ring_raw[];
   __shared__ int4 plist_s[SMAXLIST];       // (page, entries, subsequence i', distance base of entry 0)
   __shared__ int rsub_s[16 * MT];          // subsequence of row r
   __shared__ float bias_s[SMAXDIST];
+  __shared__ int last_s;
 
   const Dims &dm = a.dm;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -95,84 +128,130 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
   const int g = lane >> 2, tig = lane & 3;
 
   // ---- ONE round of independent global loads, none waiting for another: active-row count, page
-  // list (first STHREADS entries), row -> subsequence, bias row of this head, query fragments.
-  // What turns out to be unused (rows beyond the active ones) is masked afterwards.
+  // list (first STHREADS entries), row -> subsequence, where every row's new entry goes, bias row of
+  // this head.  What turns out to be unused (rows beyond the active ones) is masked afterwards.
   const int S = a.st.n_active[b];
   const int n_list = a.st.plist_n[b];
   const int list_cap = dm.SM * dm.PPS;
   const int4 *pl = a.st.plist + (size_t)b * list_cap;
   int4 my_entry = make_int4(0, 0, 0, 0);
   if (tid < list_cap) my_entry = pl[tid];
-  // this warp's first two pages (entries g0 and g0 + W of the list), so that their copies can start
-  // before the CTA has assembled the list in shared memory
-  const int W = a.splits * SW, g0 = split * SW + warp;
-  const int4 first0 = g0 < list_cap ? pl[g0] : make_int4(0, 0, 0, 0);
-  const int4 first1 = g0 + W < list_cap ? pl[g0 + W] : make_int4(0, 0, 0, 0);
+  // the entries of this warp's first batch, so that its copies can start before the CTA has assembled
+  // the list in shared memory (its index does not depend on how many splits are in use)
+  const int g0 = split * SW + warp;
+  int4 e_first[PB];
+#pragma unroll
+  for (int pb = 0; pb < PB; ++pb) e_first[pb] = PB * g0 + pb < list_cap ? pl[PB * g0 + pb] : make_int4(0, 0, 0, 0);
   int my_rsub = 0;
   if (tid < dm.C) my_rsub = a.st.row_sub[row0 + tid];
+  // (page, slot, position tau + i, subsequence) of the entry row `lane` of this sequence appends at this step
+  const int4 meta = lane < dm.C ? a.st.row_meta[row0 + lane] : make_int4(-1, 0, 0, 0);
   const bool use_bias = a.bias_tab != nullptr;
-  float my_bias[SMAXDIST / STHREADS];
+  float my_bias[SBIAS_PER_THREAD];
 #pragma unroll
-  for (int k = 0; k < SMAXDIST / STHREADS; ++k) {
+  for (int k = 0; k < SBIAS_PER_THREAD; ++k) {
     const int dd = k * STHREADS + tid;
     my_bias[k] = (use_bias && dd < dm.n_dist) ? a.bias_tab[h * dm.n_dist + dd] : 0.f;
   }
-  const __nv_bfloat16 *qbuf = (const __nv_bfloat16 *)a.q;
-  uint32_t qf[MT][4][4];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-    const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
-    const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      qf[mt][kk][0] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
-      qf[mt][kk][1] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
-      qf[mt][kk][2] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
-      qf[mt][kk][3] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
-    }
-  }
 
+  // splits in use: enough that a warp gets about SBATCHES_PER_WARP batches, at most the launched ones
+  const int n_batches = (n_list + PB - 1) / PB;
+  const int n_eff = min(a.splits, max(1, (n_batches + SW * SBATCHES_PER_WARP - 1) / (SW * SBATCHES_PER_WARP)));
   if (S == 0) {   // nothing active: keep the output rows of this head defined
     if (split == 0)
       for (int idx = tid; idx < dm.C * kDh; idx += STHREADS)
         out[(size_t)(row0 + idx / kDh) * dm.d + h * kDh + idx % kDh] = __float2bfloat16_rn(0.f);
     return;
   }
-  const int n_mine = n_list > g0 ? (n_list - g0 + W - 1) / W : 0;
-  const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SLOT;
+  if (split >= n_eff) return;
+
+  // ---- query fragments of the active rows, from the projection's output
+  uint32_t qf[MT][4][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+    const int pos_lo = __shfl_sync(0xffffffffu, meta.z, r_lo & 31), pos_hi = __shfl_sync(0xffffffffu, meta.z, r_hi & 31);
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      qf[mt][kk][0] = r_lo < S ? s_load_q(a, row0 + r_lo, kk * 16 + 2 * tig, h, pos_lo) : 0u;
+      qf[mt][kk][1] = r_hi < S ? s_load_q(a, row0 + r_hi, kk * 16 + 2 * tig, h, pos_hi) : 0u;
+      qf[mt][kk][2] = r_lo < S ? s_load_q(a, row0 + r_lo, kk * 16 + 2 * tig + 8, h, pos_lo) : 0u;
+      qf[mt][kk][3] = r_hi < S ? s_load_q(a, row0 + r_hi, kk * 16 + 2 * tig + 8, h, pos_hi) : 0u;
+    }
+  }
+
+  const int W = n_eff * SW;
+  const int n_mine = n_batches > g0 ? (n_batches - g0 + W - 1) / W : 0;
+  const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SSLOT;
   const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
   const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
-  auto fetch = [&](int n, int4 e) { s_fetch_page<P>(my_ring + (n & 1) * SLOT, pool_lh + e.x * page_stride, e.y, lane); };
-  {
-    // The warp's ring starts out zeroed: value rows beyond a partly filled page's entries get weights
-    // of exactly 0 in P.V and must be finite, whatever the slot held before (later: earlier pages' data).
-    uint4 *ring = reinterpret_cast<uint4 *>(s_ring_raw + (size_t)warp * SDEPTH * SLOT);
+
+  // One page of a batch: the entries the cache holds are copied; if a row appends to this page at this step
+  // (its entry is the page's last), the warp makes that entry from the projection's output - key
+  // rotated in rotary mode - and places it in the slot and in the cache.
+  auto fetch_page = [&](uint32_t dst, int4 e) {
+    if (e.y <= 0) return;
+    const __nv_bfloat16 *blk = pool_lh + e.x * page_stride;
+    const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
+    int n_copy = e.y;
+    if (hit != 0u) {
+      const int c = __ffs(hit) - 1;
+      const int slot = __shfl_sync(0xffffffffu, meta.y, c), pos = __shfl_sync(0xffffffffu, meta.z, c);
+      n_copy = slot;                                           // the entries before the new one
+      const size_t off = (size_t)(row0 + c) * 3 * dm.d + dm.d + (size_t)h * kDh + 2 * lane;   // key columns 2 lane, 2 lane + 1
+      uint32_t k2, v2;
+      if (!a.qkv_f32) {
+        const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(a.qkv) + off;
+        k2 = *reinterpret_cast<const uint32_t *>(src);
+        v2 = *reinterpret_cast<const uint32_t *>(src + dm.d);
+      } else {
+        const float *src = reinterpret_cast<const float *>(a.qkv) + off;
+        float2 kf = *reinterpret_cast<const float2 *>(src);
+        const float2 vf = *reinterpret_cast<const float2 *>(src + dm.d);
+        if (a.rope_tab != nullptr) {
+          const float2 cs = a.rope_tab[(size_t)pos * (kDh / 2) + lane];
+          const float t = kf.x * cs.x - kf.y * cs.y;
+          kf.y = kf.x * cs.y + kf.y * cs.x; kf.x = t;
+        }
+        k2 = s_pack_bf16(kf.x, kf.y);
+        v2 = s_pack_bf16(vf.x, vf.y);
+      }
+      const uint32_t sa = dst + s_swz(slot, lane >> 2) + (lane & 3) * 4;
+      s_st_shared_u32(sa, k2);
+      s_st_shared_u32(sa + 128u, v2);
+      __nv_bfloat16 *cache = const_cast<__nv_bfloat16 *>(blk) + kv_entry_offset<__nv_bfloat16>(slot, 2 * lane, 0);
+      *reinterpret_cast<uint32_t *>(cache) = k2;
+      *reinterpret_cast<uint32_t *>(cache + kDh) = v2;         // the value row follows the key row of the same entry
+    }
+    s_fetch_run<P>(dst, blk, n_copy, lane);
+  };
+  // batch n of this warp = list entries PB * (g0 + n W) ...; `list` = the list in global memory (before the
+  // CTA's copy is complete) or in shared memory
+  auto fetch = [&](int n, const int4 *list) {
+    const int first = PB * (g0 + n * W);
+    const uint32_t dst = my_ring + (n & 1) * SSLOT;
 #pragma unroll
-    for (int i = 0; i < (int)(SDEPTH * SLOT / 16) / 32; ++i) ring[i * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
-    __syncwarp();                      // the zeros are in place before any lane's copy lands on them
-    if (n_mine > 0) fetch(0, first0);
-    s_cp_async_commit();
-    if (n_mine > 1) fetch(1, first1);
-    s_cp_async_commit();
+    for (int pb = 0; pb < PB; ++pb) {
+      const int4 e = first + pb < n_list ? list[first + pb] : make_int4(0, 0, 0, 0);
+      fetch_page(dst + pb * P * 256, e);
+    }
+  };
+  // Nothing is ever cleared: what a slot holds beyond a page's entries (anything) gets score -inf, and
+  // the value fragments of those keys are zeroed in registers after ldmatrix.
+  if (n_mine > 0) {
+#pragma unroll
+    for (int pb = 0; pb < PB; ++pb) fetch_page(my_ring + pb * P * 256, PB * g0 + pb < n_list ? e_first[pb] : make_int4(0, 0, 0, 0));
   }
+  s_cp_async_commit();
+  if (n_mine > 1) fetch(1, pl);
+  s_cp_async_commit();
   if (tid < SMAXLIST) plist_s[tid] = my_entry;
   for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
   if (tid < 16 * MT) rsub_s[tid] = my_rsub;
 #pragma unroll
-  for (int k = 0; k < SMAXDIST / STHREADS; ++k) bias_s[k * STHREADS + tid] = my_bias[k];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {   // rows at or beyond S carry no query
-    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      if (r_lo >= S) qf[mt][kk][0] = qf[mt][kk][2] = 0u;
-      if (r_hi >= S) qf[mt][kk][1] = qf[mt][kk][3] = 0u;
-    }
-  }
+  for (int k = 0; k < SBIAS_PER_THREAD; ++k)
+    if (k * STHREADS + tid < SMAXDIST) bias_s[k * STHREADS + tid] = my_bias[k];
   __syncthreads();
-
-  // ---- this warp's share of the page list is entries g0, g0 + W, ...; its first two pages are already on their way
 
   int rs[MT][2];                     // subsequence of rows g and g + 8 of every query tile
   int tile_last[MT];                 // subsequence of the tile's last active row (rows are sorted)
@@ -195,26 +274,35 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
   const float sl2 = dm.scale_log2e;
 
   for (int n = 0; n < n_mine; ++n) {
-    s_cp_async_wait<1>();              // everything but the newest group has landed: page n is in its slot
-    __syncwarp();
-    const int4 e = plist_s[g0 + n * W];
-    const int nv = e.y;                // entries of this page that exist
-    const int ksub = e.z;              // subsequence the page belongs to
-    const int d0 = e.w;                // distance base of its first entry: distance = d0 + i - key offset
-    const uint32_t kbase = my_ring + (n & 1) * SLOT, vbase = kbase + 128u;
-    // Dependency rule: a row of subsequence i sees this page iff i' <= i (every stored entry was
-    // generated before the current step).  A query tile none of whose rows sees it is skipped;
-    // a full page that every row sees needs no masking at all.
+    s_cp_async_wait<1>();              // everything but the newest group has landed: batch n is in its slot
+    __syncwarp();                      // (and the appended entries the lanes stored themselves are visible)
+    // per page of the batch: entries that exist, subsequence, distance base of its first entry
+    int nv[PB], ksub[PB], d0[PB];
+    const int first = PB * (g0 + n * W);
+#pragma unroll
+    for (int pb = 0; pb < PB; ++pb) {
+      const int4 e = first + pb < n_list ? plist_s[first + pb] : make_int4(0, 0, 0x7fffffff, 0);
+      nv[pb] = e.y; ksub[pb] = e.z; d0[pb] = e.w;
+    }
+    const uint32_t kbase = my_ring + (n & 1) * SSLOT, vbase = kbase + 128u;
+    // Dependency rule: a row of subsequence i sees a page iff i' <= i (every stored entry was
+    // generated before the current step).  The list is sorted by subsequence: a query tile none
+    // of whose rows sees the batch's first page is skipped; a batch of full pages that every row sees
+    // needs no masking at all.
     bool act[MT];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) act[mt] = tile_last[mt] >= ksub;
-    const bool plain = nv == P && sub_first >= ksub;
+    for (int mt = 0; mt < MT; ++mt) act[mt] = tile_last[mt] >= ksub[0];
+    bool plain = true;
+#pragma unroll
+    for (int pb = 0; pb < PB; ++pb) plain = plain && nv[pb] == P && sub_first >= ksub[pb];
 
-    // ---- scores: Q (16 x 64) . K^T (64 x P keys); two accumulators per tile halve the mma chain
+    // ---- scores: Q (16 x 64) . K^T (64 x 32 keys); two accumulators per tile halve the mma chain
     float sc[MT][NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      if (nt * 8 < nv) {
+      constexpr int per_page = P / 8;                    // score tiles per page
+      const int pb = nt / per_page, within = (nt % per_page) * 8;
+      if (within < nv[pb]) {
         const int key = nt * 8 + (lane & 7);
         uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
         s_ldsm_x4(kbase + s_swz(key, (lane >> 3)), b0, b1, b2, b3);        // dims 0..31
@@ -242,39 +330,35 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       if (!act[mt]) continue;
-      // distance of rows g / g+8 to the page's entry 0, minus this thread's first key column
-      const float *bp0 = bias_s + (d0 + rs[mt][0] - 2 * tig);
-      const float *bp1 = bias_s + (d0 + rs[mt][1] - 2 * tig);
       float mx0 = -INFINITY, mx1 = -INFINITY;
-      if (plain) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
+      for (int nt = 0; nt < NT; ++nt) {
+        constexpr int per_page = P / 8;
+        const int pb = nt / per_page, within = (nt % per_page) * 8 + 2 * tig;    // this thread's first key of the tile, inside its page
+        // distance of rows g / g + 8 to the page's entry 0, minus the key's offset in the page
+        const float *bp0 = bias_s + (d0[pb] + rs[mt][0] - within);
+        const float *bp1 = bias_s + (d0[pb] + rs[mt][1] - within);
+        if (plain) {
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
-            const float bias = use_bias ? ((x & 2) ? bp1 : bp0)[-(nt * 8 + (x & 1))] : 0.f;
+            const float bias = use_bias ? ((x & 2) ? bp1 : bp0)[-(x & 1)] : 0.f;
             sc[mt][nt][x] = fmaf(sc[mt][nt][x], sl2, bias);
           }
-          mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
-          mx1 = fmaxf(mx1, fmaxf(sc[mt][nt][2], sc[mt][nt][3]));
-        }
-      } else {
-        const bool see0 = rs[mt][0] >= ksub, see1 = rs[mt][1] >= ksub;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
+        } else {
+          const bool see0 = rs[mt][0] >= ksub[pb], see1 = rs[mt][1] >= ksub[pb];
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
-            const int key = nt * 8 + 2 * tig + (x & 1);
-            const bool vis = key < nv && ((x & 2) ? see1 : see0);
+            const bool vis = within + (x & 1) < nv[pb] && ((x & 2) ? see1 : see0);
             float v = -INFINITY;
             if (vis) {
-              const float bias = use_bias ? ((x & 2) ? bp1 : bp0)[-(nt * 8 + (x & 1))] : 0.f;
+              const float bias = use_bias ? ((x & 2) ? bp1 : bp0)[-(x & 1)] : 0.f;
               v = fmaf(sc[mt][nt][x], sl2, bias);
             }
             sc[mt][nt][x] = v;
           }
-          mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
-          mx1 = fmaxf(mx1, fmaxf(sc[mt][nt][2], sc[mt][nt][3]));
         }
+        mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
+        mx1 = fmaxf(mx1, fmaxf(sc[mt][nt][2], sc[mt][nt][3]));
       }
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
@@ -300,15 +384,27 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
         for (int dn = 0; dn < 8; ++dn) { o[mt][dn][0] *= cr0; o[mt][dn][1] *= cr0; o[mt][dn][2] *= cr1; o[mt][dn][3] *= cr1; }
       }
     }
-    // ---- O += P (16 x P keys) . V (P keys x 64)
+    // ---- O += P (16 x 32 keys) . V (32 keys x 64)
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      if (ks * 16 < nv) {
+      constexpr int per_page = P / 16;                   // 16-key steps per page
+      const int pb = ks / per_page, within = (ks % per_page) * 16;
+      if (within < nv[pb]) {
         const int vkey = ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+        // this lane's fragment halves hold keys k0, k0 + 1 (b0, b2) and k0 + 8, k0 + 9 (b1, b3) of the page;
+        // keys that do not exist have weight exactly 0 and must not contribute whatever the slot holds
+        const bool ragged = nv[pb] < within + 16;
+        uint32_t keep_a = 0xffffffffu, keep_b = 0xffffffffu;
+        if (ragged) {
+          const int k0 = within + 2 * tig;
+          keep_a = (k0 < nv[pb] ? 0x0000ffffu : 0u) | (k0 + 1 < nv[pb] ? 0xffff0000u : 0u);
+          keep_b = (k0 + 8 < nv[pb] ? 0x0000ffffu : 0u) | (k0 + 9 < nv[pb] ? 0xffff0000u : 0u);
+        }
 #pragma unroll
         for (int dp = 0; dp < 4; ++dp) {
           uint32_t b0, b1, b2, b3;
           s_ldsm_x4_t(vbase + s_swz(vkey, dp * 2 + (lane >> 4)), b0, b1, b2, b3);
+          if (ragged) { b0 &= keep_a; b1 &= keep_b; b2 &= keep_a; b3 &= keep_b; }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             if (!act[mt]) continue;
@@ -319,7 +415,7 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
       }
     }
     __syncwarp();   // every lane is done reading the slot
-    if (n + 2 < n_mine) fetch(n + 2, plist_s[g0 + (n + 2) * W]);
+    if (n + 2 < n_mine) fetch(n + 2, plist_s);
     s_cp_async_commit();
   }
   s_cp_async_wait<0>();
@@ -332,7 +428,7 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
       l_run[mt][hh] += __shfl_xor_sync(0xffffffffu, l_run[mt][hh], 1);
       l_run[mt][hh] += __shfl_xor_sync(0xffffffffu, l_run[mt][hh], 2);
     }
-  __syncthreads();   // every warp is past its last page: the ring can be reused
+  __syncthreads();   // every warp is past its last batch: the ring can be reused
   constexpr int ROWS = 16 * MT;
   float *mo = reinterpret_cast<float *>(s_ring_raw);          // [SW][ROWS][SMROW]
   float *mm = mo + SW * ROWS * SMROW;                           // [SW][ROWS]
@@ -383,7 +479,7 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
       const float2 v = *reinterpret_cast<const float2 *>(&mo[(w * ROWS + r) * SMROW + col]);
       O.x += v.x * wgt; O.y += v.y * wgt;
     }
-    if (a.splits == 1) {
+    if (n_eff == 1) {
       const float inv = 1.f / ml[r];
       *reinterpret_cast<__nv_bfloat162 *>(out + orow) = __floats2bfloat162_rn(O.x * inv, O.y * inv);
     } else {
@@ -392,10 +488,41 @@ __global__ void __launch_bounds__(STHREADS) self_attn_tc_kernel(AttnArgs a) {
       if (col == 0) { a.part_ml[pi * 2] = ml[ROWS + r]; a.part_ml[pi * 2 + 1] = ml[r]; }
     }
   }
+  if (n_eff == 1) return;
+
+  // ---- several splits: the CTA that arrives last for this (sequence, head) merges the records in split order
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int ticket = atomicAdd(&a.tickets[b * dm.H + h], 1);
+    last_s = ticket == n_eff - 1;
+    if (last_s) a.tickets[b * dm.H + h] = 0;     // zero again for the next launch (every other CTA of the pair has arrived)
+  }
+  __syncthreads();
+  if (!last_s) return;
+  __threadfence();
+  for (int idx = tid; idx < S * (kDh / 2); idx += STHREADS) {
+    const int r = idx / (kDh / 2), col = 2 * (idx % (kDh / 2));
+    const size_t p0 = ((size_t)(row0 + r) * dm.H + h) * a.splits;
+    float M = -INFINITY;
+    for (int s = 0; s < n_eff; ++s) M = fmaxf(M, __ldcg(&a.part_ml[(p0 + s) * 2]));
+    float L = 0.f;
+    float2 O = make_float2(0.f, 0.f);
+    for (int s = 0; s < n_eff; ++s) {
+      const float m = __ldcg(&a.part_ml[(p0 + s) * 2]);
+      if (m == -INFINITY) continue;
+      const float w = s_ex2(m - M);
+      L += __ldcg(&a.part_ml[(p0 + s) * 2 + 1]) * w;
+      const float2 v = __ldcg(reinterpret_cast<const float2 *>(&a.part_o[(p0 + s) * kDh + col]));
+      O.x += v.x * w; O.y += v.y * w;
+    }
+    const float inv = 1.f / L;
+    *reinterpret_cast<__nv_bfloat162 *>(out + (size_t)(row0 + r) * dm.d + h * kDh + col) = __floats2bfloat162_rn(O.x * inv, O.y * inv);
+  }
 }
 
 static int self_attn_tc_smem(int P, int mt) {
-  int ring = SW * SDEPTH * 2 * P * 128;
+  int ring = SW * SDEPTH * (P > SKEYS ? P : SKEYS) * 256;
   int merge = SW * 16 * mt * (SMROW + 2) * 4;
   return ring > merge ? ring : merge;
 }
@@ -403,6 +530,19 @@ static int self_attn_tc_smem(int P, int mt) {
 bool self_attn_tc_supported(const Dims &dm) {
   return dm.C <= 32 && (dm.P == 16 || dm.P == 32) && dm.SM * dm.PPS <= SMAXLIST &&
          (dm.pos_mode != PD_POS_T5_BIAS || dm.n_dist <= SMAXDIST);
+}
+
+// Splits to launch for `pairs` (sequence, head) pairs on a device with `sms` SMs: enough for the
+// longest page list a sequence can have (CTAs whose split the current lists do not need leave at
+// once), but never more CTAs than are resident at the same time - a second wave costs a whole
+// CTA lifetime, a longer walk per warp a fraction of one.
+int self_attn_tc_splits(const Dims &dm, int pairs, int sms) {
+  const int per = dm.P > SKEYS ? 1 : SKEYS / dm.P;       // pages per batch
+  const int batches = (dm.SM * dm.PPS + per - 1) / per;
+  int s = (batches + SW * SBATCHES_PER_WARP - 1) / (SW * SBATCHES_PER_WARP);
+  const int resident = (dm.C <= 16 ? 4 : 2) * sms;
+  if (s > resident / (pairs > 0 ? pairs : 1)) s = resident / (pairs > 0 ? pairs : 1);
+  return s < 1 ? 1 : (s > 8 ? 8 : s);
 }
 
 template <int MT, int P>
@@ -418,6 +558,9 @@ cudaError_t self_attn_tc_prepare() {
   return e;
 }
 
+// a.qkv = the projection's output [rows][3 d] (bf16, or fp32 with a.qkv_f32), a.rope_tab set in rotary
+// mode, a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed), a.part_o /
+// a.part_ml sized for a.splits records per (row, head).
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s) {
   dim3 grid(a.splits, a.dm.H, a.batch);
   const int mt = (a.dm.C + 15) / 16;

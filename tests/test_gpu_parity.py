@@ -319,6 +319,36 @@ def test_two_identical_decodes_give_identical_logits():
     dec.close()
 
 
+def test_split_self_attention_merges_in_the_launch_and_repeats_bit_for_bit():
+    """Long page lists with four splits per (sequence, head): the split CTAs leave partial records and the
+    last one to arrive merges them in split order, so twenty decodes of the same inputs must give the same
+    logits bit for bit whatever the arrival order - and the logits must be the oracle's."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = W.CONFIGS["summarisation"].scaled(name="split_merge", batch=3, ctx=100, sub_max=40, delta_t=1, max_sub_len=40,
+                                           length_dist=("uniform", 25, 40), time_max=90, **SMALL_BF16)
+    weights, mem, ctx_len = W.make_weights(wl), W.make_encoder_memory(wl), W.make_ctx_len(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch, self_splits=4)
+    mem_dev = dec.device_memory(mem)
+    n_steps = 45                                        # by then every sequence holds more than 64 pages
+
+    def logits_after(steps):
+        dec.encode_context(mem_dev, ctx_len, fl)
+        for _ in range(steps):
+            dec.step()
+        return dec.get_logits()[0].copy()
+
+    first = logits_after(n_steps)
+    assert dec.stats()["pages"] > 3 * 64
+    for _ in range(19):
+        again = logits_after(n_steps)
+        assert np.array_equal(first.view(np.int32), again.view(np.int32)), "two identical decodes gave different logits"
+    runs = parity.oracle_runs(wl, weights, {1: mem[1]}, ctx_len, fl)
+    stats = parity.replay_compare(dec, wl, mem_dev, ctx_len, fl, runs, max_steps=n_steps + 5)
+    assert stats["max_err"] < 2e-2 and stats["logits"] > 0
+    dec.close()
+
+
 FULL = [("bart_base", 2e-2), ("long_context", 2e-2), ("summarisation", 2e-2), ("keyphrase", 2e-2)]
 _ORACLE_CACHE = {}
 
