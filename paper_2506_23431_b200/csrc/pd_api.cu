@@ -277,6 +277,10 @@ bool make_ff_plan(pd_handle *h, int M, int N, int K) {
     h->own_launches++;                              \
   } while (0)
 
+bool self_tc(const pd_handle *h) { return h->cfg.dtype == PD_DTYPE_BF16 && self_attn_tc_supported(h->dm); }
+// Nothing to rotate: the projection rounds to bf16 itself and the attention kernel places the new cache entries.
+bool fused_append(const pd_handle *h) { return self_tc(h) && h->dm.pos_mode != PD_POS_ROPE; }
+
 AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   AttnArgs a;
   a.dm = h->dm; a.st = h->st; a.layer = layer; a.batch = h->batch;
@@ -292,12 +296,9 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.tickets = h->ptr<int32_t>(h->lay.state) + h->lay.w_xtick;
   a.bias_tab = h->cfg.pos_mode == PD_POS_T5_BIAS ? h->ptr<float>(h->lay.bias_tab) : nullptr;
   a.qkv = h->ptr<void>(h->lay.qkv);
-  a.qkv_f32 = h->cfg.pos_mode == PD_POS_ROPE ? 1 : 0;      // the projection rounds to bf16 itself when nothing is rotated
-  a.rope_tab = h->cfg.pos_mode == PD_POS_ROPE ? h->ptr<float2>(h->lay.rope_tab) : nullptr;
+  a.fused_append = self && fused_append(h) ? 1 : 0;
   return a;
 }
-
-bool self_tc(const pd_handle *h) { return h->cfg.dtype == PD_DTYPE_BF16 && self_attn_tc_supported(h->dm); }
 
 // Pipelined self-attention of one layer.  The tensor-core kernel appends the step's keys/values itself and
 // merges its splits in the same launch; the plain-ALU kernel follows the append kernel and, when split,
@@ -347,10 +348,10 @@ pd_status enqueue_step(pd_handle *h) {
   for (int l = 0; l < dm.L; ++l) {
     const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
     OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
-    if (self_tc(h)) {
-      // the attention kernel takes queries, keys and values straight from the projection's output and
-      // appends the new cache entries itself (bf16 from the projection when nothing is rotated)
-      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, dm.pos_mode == PD_POS_ROPE, 0.f));
+    if (fused_append(h)) {
+      // the attention kernel takes queries, keys and values straight from the projection's bf16 output and
+      // appends the new cache entries itself
+      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, false, 0.f));
     } else if (dt == PD_DTYPE_BF16 && dm.pos_mode != PD_POS_ROPE) {
       // nothing to rotate: the projection rounds to bf16 itself and the append only places the rows
       PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, false, 0.f));

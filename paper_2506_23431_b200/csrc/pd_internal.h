@@ -96,11 +96,10 @@ struct AttnArgs {
   int rel_buckets;
   const float *bias_tab;       // [H, n_dist]: rel_bias[h][bucket(dist)] * log2(e), or null
   int32_t *tickets;            // one arrival counter per (sequence, head), zero between launches
-  // tensor-core self-attention (the step's KV-append happens inside it): the projection's output
-  // [rows][3 d] (bf16, or fp32 when qkv_f32), and the (cos, sin) table in rotary mode (else null)
+  // tensor-core self-attention with the step's KV-append inside it (fused_append): the projection's
+  // output [rows][3 d] in bf16
   const void *qkv;
-  int qkv_f32;
-  const float2 *rope_tab;
+  int fused_append;
 };
 
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------

@@ -20,12 +20,14 @@
 // pre-swizzled (16-byte chunk c of a row of entry e at chunk c ^ (e & 7)), so a linear copy lands
 // in the bank-conflict-free layout ldmatrix wants.
 //
-// Fused append: the entry a row feeds at this step is the last one of its subsequence's last page
-// and is not in the cache yet.  The warp that meets that page takes the row's key and value of this
-// head straight from the projection's output (rotating the key by the position tau + i in rotary
-// mode), puts them into its ring slot AND into the cache - every (page, head) block is met by
+// Fused append (when nothing has to be rotated, i.e. with the T5 bias; the projection then writes
+// bf16 itself): the entry a row feeds at this step is the last one of its subsequence's last page
+// and is not in the cache yet.  The warp that meets that page copies the row's key and value of this
+// head straight from the projection's output into its ring slot (asynchronously, like the rest of
+// the page) and, once they have landed, on into the cache - every (page, head) block is met by
 // exactly one warp of the launch, so the cache is written once, without a race, and no separate
-// append launch exists.  Queries come from the same projection output (rotated likewise).
+// append launch exists.  Queries come from the same projection output.  In rotary mode the append
+// kernel rotates queries and keys first and this kernel reads the cache alone.
 //
 // Splits: the number of splits in use follows the list's length (a CTA whose split is not needed
 // leaves at once).  Warps merge through shared memory; split CTAs leave a partial record, take a
@@ -93,31 +95,27 @@ __device__ __forceinline__ void s_fetch_run(uint32_t dst, const __nv_bfloat16 *b
     if (k * 32 + lane < nchunks) s_cp_async16(dst + lane * 16 + k * 512, src + k * 512);
 }
 
-// Query fragment word (two consecutive columns of row r) from the projection's output; rotary mode
-// rotates the pair by the row's position.
-__device__ __forceinline__ uint32_t s_load_q(const AttnArgs &a, size_t row, int col_in_head, int h, int pos) {
-  const size_t off = row * 3 * (size_t)a.dm.d + (size_t)h * kDh + col_in_head;
-  if (!a.qkv_f32) return *reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(a.qkv) + off);
-  float2 v = *reinterpret_cast<const float2 *>(reinterpret_cast<const float *>(a.qkv) + off);
-  if (a.rope_tab != nullptr) {
-    const float2 c = a.rope_tab[(size_t)pos * (kDh / 2) + col_in_head / 2];
-    const float t = v.x * c.x - v.y * c.y;
-    v.y = v.x * c.y + v.y * c.x; v.x = t;
-  }
-  return s_pack_bf16(v.x, v.y);
+// Bytes of the rings (or of the merge scratch that reuses them, whichever is larger).
+__host__ __device__ constexpr int self_attn_tc_ring_bytes(int P, int mt) {
+  return SW * SDEPTH * (P > SKEYS ? P : SKEYS) * 256 > SW * 16 * mt * (SMROW + 2) * 4 ? SW * SDEPTH * (P > SKEYS ? P : SKEYS) * 256
+                                                                                      : SW * 16 * mt * (SMROW + 2) * 4;
 }
 
-template <int MT, int P>   // MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens
-__global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel(AttnArgs a) {
+// MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens; FUSED = the launch appends the
+// step's keys/values itself (queries, keys, values in a.qkv) instead of following the append kernel (queries in a.q)
+// OCC = CTAs per SM the register budget is set for: four leave the compiler 128 registers (nothing spills),
+// five 96 (more CTAs resident, which wins when there are more (sequence, head) pairs than four per SM)
+template <int MT, int P, bool FUSED, int OCC>
+__global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kernel(AttnArgs a) {
   constexpr int BK = P > SKEYS ? P : SKEYS; // keys per batch
   constexpr int PB = BK / P;               // pages per batch
   constexpr int NT = BK / 8;               // 8-key score tiles per batch
   constexpr int KS = BK / 16;              // 16-key steps of P.V per batch
   constexpr uint32_t SSLOT = BK * 256u;    // keys + values of one batch of one head
+  // dynamic shared memory: the warps' rings (reused as merge scratch), then the sequence's page list
+  // (page, entries, subsequence i', distance base of entry 0), then this head's bias row
   extern __shared__ __align__(128) uint8_t s_ring_raw[];
-  __shared__ int4 plist_s[SMAXLIST];       // (page, entries, subsequence i', distance base of entry 0)
   __shared__ int rsub_s[16 * MT];          // subsequence of row r
-  __shared__ float bias_s[SMAXDIST];
   __shared__ int last_s;
 
   const Dims &dm = a.dm;
@@ -129,11 +127,13 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
 
   // ---- ONE round of independent global loads, none waiting for another: active-row count, page
   // list (first STHREADS entries), row -> subsequence, where every row's new entry goes, bias row of
-  // this head.  What turns out to be unused (rows beyond the active ones) is masked afterwards.
+  // this head, query fragments.  What turns out to be unused (rows beyond the active ones) is masked afterwards.
   const int S = a.st.n_active[b];
   const int n_list = a.st.plist_n[b];
   const int list_cap = dm.SM * dm.PPS;
   const int4 *pl = a.st.plist + (size_t)b * list_cap;
+  int4 *plist_s = reinterpret_cast<int4 *>(s_ring_raw + self_attn_tc_ring_bytes(P, MT));
+  float *bias_s = reinterpret_cast<float *>(plist_s + list_cap);
   int4 my_entry = make_int4(0, 0, 0, 0);
   if (tid < list_cap) my_entry = pl[tid];
   // the entries of this warp's first batch, so that its copies can start before the CTA has assembled
@@ -145,13 +145,29 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
   int my_rsub = 0;
   if (tid < dm.C) my_rsub = a.st.row_sub[row0 + tid];
   // (page, slot, position tau + i, subsequence) of the entry row `lane` of this sequence appends at this step
-  const int4 meta = lane < dm.C ? a.st.row_meta[row0 + lane] : make_int4(-1, 0, 0, 0);
+  const int4 meta = (FUSED && lane < dm.C) ? a.st.row_meta[row0 + lane] : make_int4(-1, 0, 0, 0);
   const bool use_bias = a.bias_tab != nullptr;
   float my_bias[SBIAS_PER_THREAD];
 #pragma unroll
   for (int k = 0; k < SBIAS_PER_THREAD; ++k) {
     const int dd = k * STHREADS + tid;
     my_bias[k] = (use_bias && dd < dm.n_dist) ? a.bias_tab[h * dm.n_dist + dd] : 0.f;
+  }
+  const __nv_bfloat16 *qsrc = FUSED ? (const __nv_bfloat16 *)a.qkv : (const __nv_bfloat16 *)a.q;
+  const size_t qstride = FUSED ? 3 * (size_t)dm.d : (size_t)dm.d;
+  uint32_t qf[MT][4][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+    const __nv_bfloat16 *q_lo = qsrc + (size_t)(row0 + r_lo) * qstride + h * kDh + 2 * tig;
+    const __nv_bfloat16 *q_hi = qsrc + (size_t)(row0 + r_hi) * qstride + h * kDh + 2 * tig;
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      qf[mt][kk][0] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
+      qf[mt][kk][1] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
+      qf[mt][kk][2] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
+      qf[mt][kk][3] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
+    }
   }
 
   // splits in use: enough that a warp gets about SBATCHES_PER_WARP batches, at most the launched ones
@@ -165,21 +181,6 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
   }
   if (split >= n_eff) return;
 
-  // ---- query fragments of the active rows, from the projection's output
-  uint32_t qf[MT][4][4];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-    const int pos_lo = __shfl_sync(0xffffffffu, meta.z, r_lo & 31), pos_hi = __shfl_sync(0xffffffffu, meta.z, r_hi & 31);
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      qf[mt][kk][0] = r_lo < S ? s_load_q(a, row0 + r_lo, kk * 16 + 2 * tig, h, pos_lo) : 0u;
-      qf[mt][kk][1] = r_hi < S ? s_load_q(a, row0 + r_hi, kk * 16 + 2 * tig, h, pos_hi) : 0u;
-      qf[mt][kk][2] = r_lo < S ? s_load_q(a, row0 + r_lo, kk * 16 + 2 * tig + 8, h, pos_lo) : 0u;
-      qf[mt][kk][3] = r_hi < S ? s_load_q(a, row0 + r_hi, kk * 16 + 2 * tig + 8, h, pos_hi) : 0u;
-    }
-  }
-
   const int W = n_eff * SW;
   const int n_mine = n_batches > g0 ? (n_batches - g0 + W - 1) / W : 0;
   const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SSLOT;
@@ -187,41 +188,23 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
   const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
 
   // One page of a batch: the entries the cache holds are copied; if a row appends to this page at this step
-  // (its entry is the page's last), the warp makes that entry from the projection's output - key
-  // rotated in rotary mode - and places it in the slot and in the cache.
+  // (its entry is the page's last), that entry comes from the projection's output: 8 + 8 chunks of 16 bytes.
   auto fetch_page = [&](uint32_t dst, int4 e) {
     if (e.y <= 0) return;
     const __nv_bfloat16 *blk = pool_lh + e.x * page_stride;
-    const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
     int n_copy = e.y;
-    if (hit != 0u) {
-      const int c = __ffs(hit) - 1;
-      const int slot = __shfl_sync(0xffffffffu, meta.y, c), pos = __shfl_sync(0xffffffffu, meta.z, c);
-      n_copy = slot;                                           // the entries before the new one
-      const size_t off = (size_t)(row0 + c) * 3 * dm.d + dm.d + (size_t)h * kDh + 2 * lane;   // key columns 2 lane, 2 lane + 1
-      uint32_t k2, v2;
-      if (!a.qkv_f32) {
-        const __nv_bfloat16 *src = reinterpret_cast<const __nv_bfloat16 *>(a.qkv) + off;
-        k2 = *reinterpret_cast<const uint32_t *>(src);
-        v2 = *reinterpret_cast<const uint32_t *>(src + dm.d);
-      } else {
-        const float *src = reinterpret_cast<const float *>(a.qkv) + off;
-        float2 kf = *reinterpret_cast<const float2 *>(src);
-        const float2 vf = *reinterpret_cast<const float2 *>(src + dm.d);
-        if (a.rope_tab != nullptr) {
-          const float2 cs = a.rope_tab[(size_t)pos * (kDh / 2) + lane];
-          const float t = kf.x * cs.x - kf.y * cs.y;
-          kf.y = kf.x * cs.y + kf.y * cs.x; kf.x = t;
+    if (FUSED) {
+      const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
+      if (hit != 0u) {
+        const int c = __ffs(hit) - 1;
+        const int slot = __shfl_sync(0xffffffffu, meta.y, c);
+        n_copy = slot;                                         // the entries before the new one
+        if (lane < 16) {                                       // lanes 0-7: the key row's chunks, 8-15: the value row's
+          const __nv_bfloat16 *src = (const __nv_bfloat16 *)a.qkv + (size_t)(row0 + c) * 3 * dm.d + (lane < 8 ? 1 : 2) * (size_t)dm.d +
+                                     (size_t)h * kDh + (lane & 7) * 8;
+          s_cp_async16(dst + s_swz(slot, lane & 7) + (lane < 8 ? 0u : 128u), src);
         }
-        k2 = s_pack_bf16(kf.x, kf.y);
-        v2 = s_pack_bf16(vf.x, vf.y);
       }
-      const uint32_t sa = dst + s_swz(slot, lane >> 2) + (lane & 3) * 4;
-      s_st_shared_u32(sa, k2);
-      s_st_shared_u32(sa + 128u, v2);
-      __nv_bfloat16 *cache = const_cast<__nv_bfloat16 *>(blk) + kv_entry_offset<__nv_bfloat16>(slot, 2 * lane, 0);
-      *reinterpret_cast<uint32_t *>(cache) = k2;
-      *reinterpret_cast<uint32_t *>(cache + kDh) = v2;         // the value row follows the key row of the same entry
     }
     s_fetch_run<P>(dst, blk, n_copy, lane);
   };
@@ -245,12 +228,12 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
   s_cp_async_commit();
   if (n_mine > 1) fetch(1, pl);
   s_cp_async_commit();
-  if (tid < SMAXLIST) plist_s[tid] = my_entry;
+  if (tid < list_cap) plist_s[tid] = my_entry;
   for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
   if (tid < 16 * MT) rsub_s[tid] = my_rsub;
 #pragma unroll
   for (int k = 0; k < SBIAS_PER_THREAD; ++k)
-    if (k * STHREADS + tid < SMAXDIST) bias_s[k * STHREADS + tid] = my_bias[k];
+    if (use_bias && k * STHREADS + tid < dm.n_dist) bias_s[k * STHREADS + tid] = my_bias[k];
   __syncthreads();
 
   int rs[MT][2];                     // subsequence of rows g and g + 8 of every query tile
@@ -283,6 +266,21 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
     for (int pb = 0; pb < PB; ++pb) {
       const int4 e = first + pb < n_list ? plist_s[first + pb] : make_int4(0, 0, 0x7fffffff, 0);
       nv[pb] = e.y; ksub[pb] = e.z; d0[pb] = e.w;
+      if (FUSED && e.y > 0) {
+        // the entry a row appended to this page has landed in the slot: on into the cache (same swizzled place)
+        const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
+        if (hit != 0u) {
+          const int slot = __shfl_sync(0xffffffffu, meta.y, __ffs(hit) - 1);
+          if (lane < 16) {
+            const uint32_t off = s_swz(slot, lane & 7) + (lane < 8 ? 0u : 128u);
+            uint4 v;
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                         : "r"(my_ring + (n & 1) * SSLOT + pb * P * 256 + off));
+            uint8_t *cache = reinterpret_cast<uint8_t *>(const_cast<__nv_bfloat16 *>(pool_lh + e.x * page_stride)) + off;
+            *reinterpret_cast<uint4 *>(cache) = v;
+          }
+        }
+      }
     }
     const uint32_t kbase = my_ring + (n & 1) * SSLOT, vbase = kbase + 128u;
     // Dependency rule: a row of subsequence i sees a page iff i' <= i (every stored entry was
@@ -521,11 +519,11 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? 4 : 2) self_attn_tc_kernel
   }
 }
 
-static int self_attn_tc_smem(int P, int mt) {
-  int ring = SW * SDEPTH * (P > SKEYS ? P : SKEYS) * 256;
-  int merge = SW * 16 * mt * (SMROW + 2) * 4;
-  return ring > merge ? ring : merge;
+static int self_attn_tc_smem(const Dims &dm) {
+  const int mt = (dm.C + 15) / 16;
+  return self_attn_tc_ring_bytes(dm.P, mt) + dm.SM * dm.PPS * (int)sizeof(int4) + (dm.pos_mode == PD_POS_T5_BIAS ? dm.n_dist * 4 : 0);
 }
+static int self_attn_tc_max_smem(int P, int mt) { return self_attn_tc_ring_bytes(P, mt) + SMAXLIST * (int)sizeof(int4) + SMAXDIST * 4; }
 
 bool self_attn_tc_supported(const Dims &dm) {
   return dm.C <= 32 && (dm.P == 16 || dm.P == 32) && dm.SM * dm.PPS <= SMAXLIST &&
@@ -540,14 +538,22 @@ int self_attn_tc_splits(const Dims &dm, int pairs, int sms) {
   const int per = dm.P > SKEYS ? 1 : SKEYS / dm.P;       // pages per batch
   const int batches = (dm.SM * dm.PPS + per - 1) / per;
   int s = (batches + SW * SBATCHES_PER_WARP - 1) / (SW * SBATCHES_PER_WARP);
-  const int resident = (dm.C <= 16 ? 4 : 2) * sms;
+  // CTAs an SM holds: five by registers (two with 32 rows), and what 227 KB of shared memory allow
+  const int by_smem = (227 * 1024) / (self_attn_tc_smem(dm) + 1024 + 256);
+  const int per_sm = dm.C <= 16 ? (by_smem < 5 ? by_smem : 5) : (by_smem < 2 ? by_smem : 2);
+  const int resident = (per_sm < 1 ? 1 : per_sm) * sms;
   if (s > resident / (pairs > 0 ? pairs : 1)) s = resident / (pairs > 0 ? pairs : 1);
   return s < 1 ? 1 : (s > 8 ? 8 : s);
 }
 
 template <int MT, int P>
 static cudaError_t prepare_one() {
-  return cudaFuncSetAttribute(self_attn_tc_kernel<MT, P>, cudaFuncAttributeMaxDynamicSharedMemorySize, self_attn_tc_smem(P, MT));
+  const int smem = self_attn_tc_max_smem(P, MT);
+  cudaError_t e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, false, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, true, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  return e;
 }
 
 cudaError_t self_attn_tc_prepare() {
@@ -558,18 +564,29 @@ cudaError_t self_attn_tc_prepare() {
   return e;
 }
 
-// a.qkv = the projection's output [rows][3 d] (bf16, or fp32 with a.qkv_f32), a.rope_tab set in rotary
-// mode, a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed), a.part_o /
+// a.fused_append: a.qkv = the projection's output [rows][3 d] in bf16 (else a.q = the queries the append
+// kernel left), a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed), a.part_o /
 // a.part_ml sized for a.splits records per (row, head).
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s) {
   dim3 grid(a.splits, a.dm.H, a.batch);
   const int mt = (a.dm.C + 15) / 16;
-  const int smem = self_attn_tc_smem(a.dm.P, mt);
-  if (mt == 1 && a.dm.P == 16) self_attn_tc_kernel<1, 16><<<grid, STHREADS, smem, s>>>(a);
-  else if (mt == 2 && a.dm.P == 16) self_attn_tc_kernel<2, 16><<<grid, STHREADS, smem, s>>>(a);
-  else if (mt == 1 && a.dm.P == 32) self_attn_tc_kernel<1, 32><<<grid, STHREADS, smem, s>>>(a);
-  else if (mt == 2 && a.dm.P == 32) self_attn_tc_kernel<2, 32><<<grid, STHREADS, smem, s>>>(a);
+  const int smem = self_attn_tc_smem(a.dm);
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const bool roomy = (long long)a.splits * a.dm.H * a.batch <= 4LL * sms;      // all CTAs resident at four per SM
+#define PD_SELF_LAUNCH(MT_, P_)                                                                            \
+  do {                                                                                                   \
+    if (a.fused_append && roomy) self_attn_tc_kernel<MT_, P_, true, 4><<<grid, STHREADS, smem, s>>>(a);   \
+    else if (a.fused_append) self_attn_tc_kernel<MT_, P_, true, 5><<<grid, STHREADS, smem, s>>>(a);       \
+    else if (roomy) self_attn_tc_kernel<MT_, P_, false, 4><<<grid, STHREADS, smem, s>>>(a);               \
+    else self_attn_tc_kernel<MT_, P_, false, 5><<<grid, STHREADS, smem, s>>>(a);                          \
+  } while (0)
+  if (mt == 1 && a.dm.P == 16) PD_SELF_LAUNCH(1, 16);
+  else if (mt == 2 && a.dm.P == 16) PD_SELF_LAUNCH(2, 16);
+  else if (mt == 1 && a.dm.P == 32) PD_SELF_LAUNCH(1, 32);
+  else if (mt == 2 && a.dm.P == 32) PD_SELF_LAUNCH(2, 32);
   else return cudaErrorInvalidValue;
+#undef PD_SELF_LAUNCH
   return cudaGetLastError();
 }
 
