@@ -30,12 +30,11 @@ import numpy as np
 
 from paper_2506_23431_b200 import workload as W
 
-# DRAM traffic / algorithmic bytes of the two attention kernels, from the ncu capture summarised in
-# profiles/attention_kernels_summarisation_batch16.md (dram__bytes_read.sum + dram__bytes_write.sum
-# of one launch over the bytes the method must move).  Both kernels read every sequence's
-# keys/values once, so the ratio carries over to other batch sizes.  Set to None when a kernel
-# changes after its counters were taken.
-TRAFFIC_RATIO = {"cross_attn": 1.03, "self_attn": 1.03}
+# DRAM traffic / algorithmic bytes of the two attention kernels, from an ncu capture of one launch each
+# (dram__bytes_read.sum + dram__bytes_write.sum over the bytes the method must move).  Both kernels
+# read every sequence's keys/values once, so the ratio carries over to other batch sizes.  None =
+# the kernel has changed since its counters were taken.
+TRAFFIC_RATIO = {"cross_attn": None, "self_attn": None}
 
 METRIC = "decoded tokens/s per B200"
 UNIT = "tokens/s"
@@ -208,6 +207,40 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this same command (one process per
+    GPU) through torch.distributed.run on the loopback address and hand back its exit code.  Rank 0's
+    JSON line goes to stdout as usual; NCCL's own log (communicator size included) goes to stderr."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def spawn_check(args):
+    """Every rank joins the process group and one MAX / SUM reduction; rank 0 reports how many took part."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    device = "cpu"
+    if args.backend == "nccl":
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        device = "cuda"
+    if world > 1:
+        dist.init_process_group(args.backend)
+    t, c = reduce_over_ranks([float(rank)], [1], dist if world > 1 else None, device)
+    if rank == 0:
+        print(json.dumps({"spawn_check": True, "n_ranks": c[0], "max_rank": t[0], "world_size": world, "backend": args.backend}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -220,8 +253,12 @@ def main():
                     help="time-steps of batch row 0 the CPU oracle decodes for cpu_baseline (256 = its whole decode on every config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--sequential", action="store_true",
-                    help="also time the sequential decoder (sub_max = 1) on the same targets and report the speed-up")
+    ap.add_argument("--no-sequential", action="store_true",
+                    help="skip the sequential decoder (sub_max = 1 on the same targets), which is otherwise timed beside the "
+                         "pipelined one at N = 1 for the speed-up the paper's tables report")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend for N > 1")
+    ap.add_argument("--spawn-check", action="store_true",
+                    help="start the ranks, reduce one number over them, report the rank count and exit (no decode)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
     ap.add_argument("--single-decode", action="store_true",
                     help="run exactly one encode + decode and exit (no timing): the command profilers are pointed at")
@@ -232,6 +269,11 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
+    if args.spawn_check:
+        spawn_check(args)
         return
     if args.warmup < 3:
         args.warmup = 3
@@ -246,7 +288,7 @@ def main():
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.init_process_group(args.backend, device_id=torch.device("cuda", local_rank))
 
     def barrier():
         if dist is not None:
@@ -408,21 +450,25 @@ def main():
             "roofline": roofline, "roofline_self_attn": roofline_self, "roofline_vocab": roofline_vocab,
             "kernel_ms_per_decode": kernel_ms}
 
-    if rank == 0 and world == 1 and args.sequential:
+    att = [r["frac"] for r in (roofline, roofline_self) if r]
+    if att:
+        line["roofline_min_attention_frac"] = min(att)
+    if rank == 0 and world == 1 and not args.no_sequential:
         # the same targets decoded by the ordinary sequential decoder (sub_max = 1) with the same library
         dec.close()
         swl, sfl = sequential_workload(wl, fl)
         sdec = PipelinedDecoder(swl.hyper(), weights, swl.batch, device=local_rank, use_graph=not args.no_graph,
                                 store_logits=False)
         s_ms = []
-        for k in range(args.warmup + args.steps):
+        s_warm, s_steps = 1, min(2, args.steps)          # a sequential decode takes several times a pipelined one
+        for k in range(s_warm + s_steps):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             sdec.encode_context(mem_dev, ctx_len, sfl)
             a.record(sdec.stream)
             sdec.run(poll_every=8)
             b.record(sdec.stream)
             torch.cuda.synchronize()
-            if k >= args.warmup:
+            if k >= s_warm:
                 s_ms.append(a.elapsed_time(b))
         sst = sdec.stats()
         sdec.close()

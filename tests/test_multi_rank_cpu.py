@@ -68,3 +68,17 @@ def test_rank_workloads_are_a_partition_by_independent_seeds():
     a, b = bench.rank_workload(wl, 0), bench.rank_workload(wl, 3)
     assert a == wl and b.seed != wl.seed and b.batch == wl.batch
     assert not np.array_equal(W.make_forced_len(a), W.make_forced_len(b))
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment starts two ranks by itself (gloo here,
+    NCCL on the GPU machine); rank 0 alone reports, and it saw both."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--backend", "gloo", "--spawn-check"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    res = json.loads(lines[0])
+    assert res["n_ranks"] == 2 and res["world_size"] == 2 and res["max_rank"] == 1.0
