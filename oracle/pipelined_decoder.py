@@ -29,6 +29,13 @@ What follows the paper and what is a reading of it:
   they are pinned only against a separately written textbook causal decoder (sub_max = 1).
 * The terminator of an ended subsequence is output only; it is never fed back and never
   becomes a key (a reading).  eos and sep both end a subsequence.
+* `e4m3_round`, `quantize_context_kv` - an option of this build, not of the paper (hp["kv_c_dtype"] =
+  "e4m3"): the cross-attention keys/values of Eq. 1's encoder memory are stored as 8-bit floats
+  (OCP FP8 E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest
+  finite value 448) with one scale per (layer, head, keys | values) of a sequence, and attention
+  runs over the de-quantised values.  The rounding decisions are taken in the precision the CUDA
+  path takes them in (bf16 projections, float32 scale arithmetic); everything after that is
+  float64 as elsewhere.
 """
 from __future__ import annotations
 
@@ -165,6 +172,44 @@ def rope_rotate(x: np.ndarray, pos: int, theta: float) -> np.ndarray:
     return out
 
 
+def bf16_round(a: np.ndarray) -> np.ndarray:
+    """float32 values rounded to the nearest bfloat16 (ties to even), as float32: bfloat16 keeps the
+    upper 16 bits of a float32."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    u = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return u.view(np.float32)
+
+
+E4M3_MAX = 448.0
+
+
+def e4m3_round(a: np.ndarray) -> np.ndarray:
+    """Round to the nearest value of the E4M3 grid, ties to the even mantissa, saturating at +-448.
+    The grid: +-2^(e-7) * (1 + m/8) for e = 1..15 (m = 0..7, without e = 15, m = 7, which is NaN), and
+    the subnormals +-2^-6 * m/8.  Below 2^-6 the spacing is 2^-9; in [2^k, 2^(k+1)) it is 2^(k-3)."""
+    x = np.asarray(a, dtype=np.float64)
+    mag = np.minimum(np.abs(x), E4M3_MAX)
+    k = np.floor(np.log2(np.maximum(mag, 2.0 ** -6)))          # exponent of the binade (subnormals share 2^-6's spacing)
+    step = 2.0 ** (k - 3)
+    q = np.rint(mag / step) * step                               # np.rint rounds halves to even, and mag / step is exact
+    return np.copysign(np.minimum(q, E4M3_MAX), x)
+
+
+def quantize_context_kv(kv: np.ndarray, ctx_rows: int):
+    """kv [N, dh] (one head's keys or values of one sequence, float64).  Returns (the de-quantised
+    array, scale).  Decisions in the CUDA path's precision: the projection is rounded to bfloat16, the
+    scale is max|.| / 448 in float32 (1 when everything is zero), a value's code is
+    e4m3_round(float32(value) * float32(448 / max|.|))."""
+    v = bf16_round(np.asarray(kv, dtype=np.float64).astype(np.float32))[:ctx_rows]
+    amax = np.float32(np.abs(v).max()) if v.size else np.float32(0)
+    if amax == 0:
+        return np.zeros(v.shape, dtype=np.float64), 1.0
+    inv = np.float32(E4M3_MAX) / amax
+    scale = amax / np.float32(E4M3_MAX)
+    codes = e4m3_round((v * inv).astype(np.float32))
+    return codes.astype(np.float64) * np.float64(scale), float(scale)
+
+
 def masked_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, mask: np.ndarray, scale: float,
                      bias: Optional[np.ndarray] = None) -> np.ndarray:
     """softmax(scale * q.k + bias) over exactly the visible keys, times V.
@@ -213,7 +258,11 @@ class PipelinedDecoderOracle:
         ctx = []
         for l in range(self.L):
             kv = mem @ self.w[f"l{l}.wkv_c"]
-            ctx.append((self._heads(kv[:, :hd]), self._heads(kv[:, hd:])))
+            K, V = self._heads(kv[:, :hd]), self._heads(kv[:, hd:])
+            if self.hp.get("kv_c_dtype", "same") == "e4m3":
+                K = np.stack([quantize_context_kv(K[h], ctx_len)[0] for h in range(self.H)])
+                V = np.stack([quantize_context_kv(V[h], ctx_len)[0] for h in range(self.H)])
+            ctx.append((K, V))
         return ctx
 
     # ---- the dependency rule and the positional term, by brute force over all token pairs
