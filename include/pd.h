@@ -55,6 +55,7 @@ typedef enum {
 
 enum { PD_DTYPE_FP32 = 0, PD_DTYPE_BF16 = 1 };
 enum { PD_POS_T5_BIAS = 0, PD_POS_ROPE = 1 };
+enum { PD_KV_SAME = 0, PD_KV_E4M3 = 1 };
 /* per-subsequence flags returned by pd_collect */
 enum { PD_FLAG_COMPLETE = 1, PD_FLAG_TRUNCATED = 2, PD_FLAG_CAPPED = 4 };
 /* intermediate buffers readable with pd_debug_read (values of the last layer of the last step) */
@@ -90,6 +91,13 @@ typedef struct {
                              bf16 path the vocabulary projection keeps the logits on chip (only the
                              greedy choice of Eq. 4 leaves the kernel) and pd_get_logits returns
                              PD_ERR_STATE; the fp32 path stores them either way                    */
+  int32_t kv_c_dtype;     /* storage of the cross-attention keys/values (the projected encoder memory, the
+                             dominant byte term of a step).  PD_KV_SAME: cfg.dtype.  PD_KV_E4M3 (bf16 path,
+                             at most 32 rows per sequence, max_ctx a multiple of 16): 8-bit floats (1-4-3,
+                             largest value 448) with one fp32 scale per (layer, sequence, head, keys | values)
+                             = max|.| / 448 over the sequence's context; attention runs over the de-quantised
+                             values - half the bytes per step, logits within the same tolerance of an oracle
+                             that quantises likewise                                                  */
   int32_t device;         /* CUDA device ordinal                                                */
 } pd_config;
 

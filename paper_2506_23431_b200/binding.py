@@ -36,7 +36,7 @@ class PdConfig(C.Structure):
                                          "bos_id", "eos_id", "sep_id", "pos_mode", "rel_buckets", "rel_max_dist")] + \
                [(n, C.c_float) for n in ("rope_theta", "attn_scale", "norm_eps")] + \
                [(n, C.c_int32) for n in ("page_tokens", "pool_pages", "self_splits", "cross_splits", "use_graph",
-                                         "store_logits", "device")]
+                                         "store_logits", "kv_c_dtype", "device")]
 
 
 class PdWeights(C.Structure):
@@ -107,7 +107,7 @@ def _p(a: Optional[np.ndarray], typ=_i32p):
 
 
 def make_config(hp: Dict, max_batch: int, device: int = 0, use_graph: bool = True, self_splits: int = 0,
-                cross_splits: int = 0, pool_pages: int = 0, store_logits: bool = True) -> PdConfig:
+                cross_splits: int = 0, pool_pages: int = 0, store_logits: bool = True, kv_c_dtype: Optional[str] = None) -> PdConfig:
     """pd_config from a plain hyper-parameter dict (keys as in Workload.hyper())."""
     c = PdConfig()
     for k in ("n_layers", "d_model", "n_heads", "d_head", "d_ff", "vocab", "sub_max", "delta_t", "time_max",
@@ -118,6 +118,8 @@ def make_config(hp: Dict, max_batch: int, device: int = 0, use_graph: bool = Tru
     c.rope_theta, c.attn_scale, c.norm_eps = float(hp["rope_theta"]), float(hp["attn_scale"]), float(hp["norm_eps"])
     c.pool_pages, c.self_splits, c.cross_splits = pool_pages, self_splits, cross_splits
     c.use_graph, c.store_logits, c.device = int(use_graph), int(store_logits), device
+    kv = hp.get("kv_c_dtype", "same") if kv_c_dtype is None else kv_c_dtype
+    c.kv_c_dtype = 1 if kv == "e4m3" else 0
     return c
 
 

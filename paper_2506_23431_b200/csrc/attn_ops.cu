@@ -66,7 +66,7 @@ pd_status cross_attention_enqueue(int dtype, int batch, int rows_per_seq, int n_
     CUtensorMap tmap;
     if (encode_ctx_kv_tensor_map(&tmap, kv, (uint64_t)batch * n_heads * 2 * max_ctx, nullptr) != cudaSuccess) return PD_ERR_CUDA;
     if (cross_attn_tma_prepare() != cudaSuccess) return PD_ERR_CUDA;
-    return launch_cross_attn_tma(a, tmap, cross_attn_ctas(), s) == cudaSuccess ? PD_OK : PD_ERR_CUDA;
+    return launch_cross_attn_tma(a, tmap, tmap, cross_attn_ctas(), s) == cudaSuccess ? PD_OK : PD_ERR_CUDA;
   }
   e = launch_attn_core(a, dtype, false, s);
   if (e != cudaSuccess) return PD_ERR_CUDA;

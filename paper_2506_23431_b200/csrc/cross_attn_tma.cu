@@ -17,16 +17,29 @@
 // partial record, takes a ticket, and the CTA that arrives last for that (sequence, head) merges
 // all records in CTA order (deterministic) and writes the output - no CTA ever waits for another.
 // Every mbarrier wait is bounded: on expiry the kernel records PD_ERR_TIMEOUT and drains.
+//
+// 8-bit variant (FP8 = true): the context keys/values are E4M3 codes with one scale per (layer,
+// sequence, head, keys | values) - half the bytes of the dominant term of a decode step.  Keys are
+// stored [position][64] (a 128-key tile is 64 lines of 128 bytes), values transposed [dim][position],
+// so that both reach the tensor cores through plain ldmatrix: a thread's 32-bit fragment word holds
+// four consecutive codes (four dims of a key, or four keys of a dim), widened to two f16 pairs in
+// registers (cvt.rn.f16x2.e4m3x2, exact).  The order of the sixteen dims (keys) inside a k16 step is
+// therefore 4 tig + {0, 1} | 4 tig + {2, 3} instead of 2 tig + {0, 1} | 2 tig + 8 + {0, 1}; queries
+// (score columns) are loaded with the same permutation, which a contraction does not see.  Queries and
+// softmax weights go through f16 (exact for bf16 queries in f16's range; 11 bits for the weights), the
+// key scale is folded into the score scale and the value scale into the final 1 / l.  Stages are 16 KB,
+// so the ring is six deep.
+#include <cuda_fp16.h>
+
 #include "pd_internal.h"
 
 namespace pd {
 
 constexpr int XK = 128;                   // keys per tile
-constexpr int XSTAGES = 3;
+constexpr int XRING_BYTES = 96 * 1024;    // three 32 KB stages (bf16) or six 16 KB stages (8-bit)
+constexpr int XMAX_STAGES = 6;
 constexpr int XCW = 4;                    // consumer warps
 constexpr int XTHREADS = (XCW + 1) * 32;
-constexpr int XTILE_BYTES = XK * kDh * 2; // 16 KB
-constexpr int XSTAGE_BYTES = 2 * XTILE_BYTES;
 constexpr int XMIN_TILES = 4;              // fewest tiles worth a CTA of its own
 constexpr int XMIN_WHOLE = 64;             // fewest CTAs for which whole (sequence, head) segments per CTA still beat cutting the tile list
 constexpr int XLONG_SEG = 24;              // tiles from which a segment is worth two CTAs when there are fewer segments than SMs
@@ -34,7 +47,7 @@ constexpr int XMAXB = 256;                // sequences per launch the tile prefi
 constexpr int XREC_WORDS = 36;            // per lane and 16-row tile: 32 output values, 2 maxima, 2 sums
 constexpr int XREC_FLOATS = XREC_WORDS * 32;
 constexpr int XSCRATCH_BYTES = 2 * XREC_FLOATS * 4;   // two records for the warp tree merge
-constexpr int XSMEM = XSTAGES * XSTAGE_BYTES + XSCRATCH_BYTES + 128 /*barriers*/ + 1024 /*alignment slack*/;
+constexpr int XSMEM = XRING_BYTES + XSCRATCH_BYTES + 128 /*barriers*/ + 1024 /*alignment slack*/;
 constexpr uint32_t XSPIN_LIMIT = 1u << 24;
 
 int cross_attn_tma_smem_bytes() { return XSMEM; }
@@ -76,6 +89,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tma
       ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tmap, uint32_t bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -90,6 +109,29 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+// two E4M3 codes (the low or the high half of a fragment word) -> f16 pair; every E4M3 value is an f16 value
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t word, int high) {
+  uint32_t r;
+  const unsigned short v = (unsigned short)(high ? (word >> 16) : (word & 0xffffu));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
+  return r;
+}
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
+  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&w);
+  const __half2 hh = __float22half2_rn(__bfloat1622float2(b));
+  return *reinterpret_cast<const uint32_t *>(&hh);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -165,8 +207,14 @@ struct TileCursor {
   }
 };
 
-template <int MT>   // MT = 16-row query tiles (rows per sequence <= 16 * MT)
-__global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap, AttnArgs a) {
+// MT = 16-row query tiles (rows per sequence <= 16 * MT); FP8 = keys/values are E4M3 codes (tmap: the keys'
+// 128-byte lines, tmap_v: the transposed values), else bf16 (tmap alone: rows of 64 values)
+template <int MT, bool FP8>
+__global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                  const __grid_constant__ CUtensorMap tmap_v, AttnArgs a) {
+  constexpr int XTILE_BYTES = XK * kDh * (FP8 ? 1 : 2);    // keys (or values) of one tile: 8 or 16 KB
+  constexpr int XSTAGE_BYTES = 2 * XTILE_BYTES;
+  constexpr int XSTAGES = XRING_BYTES / XSTAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int pfx_s[XMAXB + 1];
   __shared__ int aseq_s[XMAXB];             // the a-th sequence that has an active row
@@ -264,9 +312,16 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         if (!mbar_wait(bar_empty + 8 * s, (u & 1u) ^ 1u)) { atomicExch(&a.st.hdr[HDR_STATUS], (int)PD_ERR_TIMEOUT); break; }
         mbar_expect_tx(bar_full + 8 * s, XSTAGE_BYTES);
         const uint32_t dst = base + s * XSTAGE_BYTES;
-        const int y = (int)(ctx_kv_offset(a.layer, dm.B, cur.b, H, cur.h, 0, dm.ctx) / kDh) + cur.tile * XK;
-        tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, y);                         // K tile
-        tma_load_2d(dst + XTILE_BYTES, &tmap, bar_full + 8 * s, 0, y + dm.ctx);  // V tile
+        if (FP8) {
+          // block (layer, sequence, head) = max_ctx * 64 bytes of keys, then as many of transposed values
+          const int blk = (((a.layer * dm.B + cur.b) * H + cur.h) << 1);
+          tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, blk * (dm.ctx >> 1) + cur.tile * (XK / 2));    // 64 lines = 128 keys
+          tma_load_3d(dst + XTILE_BYTES, &tmap_v, bar_full + 8 * s, cur.tile * XK, 0, blk + 1);       // 64 dims x 128 keys
+        } else {
+          const int y = (int)(ctx_kv_offset(a.layer, dm.B, cur.b, H, cur.h, 0, dm.ctx) / kDh) + cur.tile * XK;
+          tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, y);                         // K tile
+          tma_load_2d(dst + XTILE_BYTES, &tmap, bar_full + 8 * s, 0, y + dm.ctx);  // V tile
+        }
         if (++cur.tile == cur.nt) cur.next_segment(pfx_s, batch, H);
       }
     }
@@ -288,18 +343,36 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
     const int my_end = min(hi, seg_end);
     const int S = nact_s[b], ctx_len = min(max(a.st.ctx_len[b], 1), dm.ctx);
     const int row0 = b * dm.C;
+    float seg_sl2 = sl2, seg_vscale = 1.f;          // 8-bit: the key scale joins the score scale, the value scale the final 1 / l
+    if (FP8) {
+      const float2 sc2 = *reinterpret_cast<const float2 *>(a.kv_scale + ((((size_t)a.layer * dm.B + b) * H + h) << 1));
+      seg_sl2 = sl2 * sc2.x; seg_vscale = sc2.y;
+    }
     uint32_t qf[MT][4][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-      const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
-      const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
+      if (FP8) {
+        // f16 queries, dims 4 tig + {0, 1} | 4 tig + {2, 3} of every 16: the order the key codes come in
+        const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 4 * tig;
+        const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 4 * tig;
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk) {
-        qf[mt][kk][0] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
-        qf[mt][kk][1] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
-        qf[mt][kk][2] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
-        qf[mt][kk][3] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
+        for (int kk = 0; kk < 4; ++kk) {
+          const uint2 lo = r_lo < S ? *reinterpret_cast<const uint2 *>(q_lo + kk * 16) : make_uint2(0u, 0u);
+          const uint2 hi = r_hi < S ? *reinterpret_cast<const uint2 *>(q_hi + kk * 16) : make_uint2(0u, 0u);
+          qf[mt][kk][0] = bf16x2_to_f16x2(lo.x); qf[mt][kk][2] = bf16x2_to_f16x2(lo.y);
+          qf[mt][kk][1] = bf16x2_to_f16x2(hi.x); qf[mt][kk][3] = bf16x2_to_f16x2(hi.y);
+        }
+      } else {
+        const __nv_bfloat16 *q_lo = qbuf + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
+        const __nv_bfloat16 *q_hi = qbuf + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          qf[mt][kk][0] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
+          qf[mt][kk][1] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
+          qf[mt][kk][2] = r_lo < S ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
+          qf[mt][kk][3] = r_hi < S ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
+        }
       }
     }
     TileAcc acc[MT];
@@ -326,16 +399,32 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         for (int nt = 0; nt < 4; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
-        const int key = kb + nt * 8 + (lane & 7);
+        if (FP8) {
+          // column c of score tile nt = 2 ks + u is key 16 ks + 4 (c >> 1) + 2 u + (c & 1) of this warp's 32: the
+          // order in which the value codes of a 16-key step come out of ldmatrix (see the P.V loop)
+          const int c = lane & 7;
+          const int key = kb + 16 * (nt >> 1) + 4 * (c >> 1) + 2 * (nt & 1) + (c & 1);
+          const int line = key >> 1, chunk = ((key & 1) << 2) + (lane >> 3);       // two keys per 128-byte line
+          uint32_t r[4];
+          ldsm_x4(kbase + (uint32_t)(line * 128 + ((chunk ^ (line & 7)) << 4)), r[0], r[1], r[2], r[3]);   // all 64 dims of 8 keys
 #pragma unroll
-        for (int kp = 0; kp < 2; ++kp) {      // two k16 steps per ldmatrix.x4
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(kbase + swz(key, kp * 4 + (lane >> 3)), b0, b1, b2, b3);
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t b0 = e4m3x2_to_f16x2(r[j], 0), b1 = e4m3x2_to_f16x2(r[j], 1);
 #pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            mma_bf16(sc[mt][nt], qf[mt][2 * kp][0], qf[mt][2 * kp][1], qf[mt][2 * kp][2], qf[mt][2 * kp][3], b0, b1);
-            mma_bf16(sc[mt][nt], qf[mt][2 * kp + 1][0], qf[mt][2 * kp + 1][1], qf[mt][2 * kp + 1][2],
-                     qf[mt][2 * kp + 1][3], b2, b3);
+            for (int mt = 0; mt < MT; ++mt) mma_f16(sc[mt][nt], qf[mt][j][0], qf[mt][j][1], qf[mt][j][2], qf[mt][j][3], b0, b1);
+          }
+        } else {
+          const int key = kb + nt * 8 + (lane & 7);
+#pragma unroll
+          for (int kp = 0; kp < 2; ++kp) {      // two k16 steps per ldmatrix.x4
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(kbase + swz(key, kp * 4 + (lane >> 3)), b0, b1, b2, b3);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+              mma_bf16(sc[mt][nt], qf[mt][2 * kp][0], qf[mt][2 * kp][1], qf[mt][2 * kp][2], qf[mt][2 * kp][3], b0, b1);
+              mma_bf16(sc[mt][nt], qf[mt][2 * kp + 1][0], qf[mt][2 * kp + 1][1], qf[mt][2 * kp + 1][2],
+                       qf[mt][2 * kp + 1][3], b2, b3);
+            }
           }
         }
       }
@@ -348,8 +437,9 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float v = sc[mt][nt][e] * sl2;
-            if (ragged && key0 + nt * 8 + 2 * tig + (e & 1) >= ctx_len) v = -INFINITY;
+            float v = sc[mt][nt][e] * seg_sl2;
+            const int kidx = FP8 ? key0 + 16 * (nt >> 1) + 4 * tig + 2 * (nt & 1) + (e & 1) : key0 + nt * 8 + 2 * tig + (e & 1);
+            if (ragged && kidx >= ctx_len) v = -INFINITY;
             sc[mt][nt][e] = v;
           }
           mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
@@ -370,8 +460,8 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
           float p0 = ex2f(sc[mt][nt][0] - ref0), p1 = ex2f(sc[mt][nt][1] - ref0);
           float p2 = ex2f(sc[mt][nt][2] - ref1), p3 = ex2f(sc[mt][nt][3] - ref1);
           s0 += p0 + p1; s1 += p2 + p3;
-          pf[mt][nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-          pf[mt][nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+          pf[mt][nt >> 1][(nt & 1) * 2 + 0] = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
+          pf[mt][nt >> 1][(nt & 1) * 2 + 1] = FP8 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
         }
         A.l0 = A.l0 * c0 + s0;
         A.l1 = A.l1 * c1 + s1;
@@ -381,6 +471,27 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         }
       }
       // ---- O += P (16 x 32 keys) . V (32 keys x 64)
+      if (FP8) {
+        // transposed values: a line is one dim, a 16-byte chunk sixteen keys; positions at or beyond ctx_len
+        // hold zero codes (written so, or filled by the copy beyond max_ctx), so nothing needs masking
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const int chunk = (kb + ks * 16) >> 4;
+#pragma unroll
+          for (int dq = 0; dq < 2; ++dq) {      // four 8-wide slices of the head per ldmatrix.x4
+            const int dim = (dq * 4 + (lane >> 3)) * 8 + (lane & 7);
+            uint32_t r[4];
+            ldsm_x4(vbase + (uint32_t)(dim * 128 + ((chunk ^ (dim & 7)) << 4)), r[0], r[1], r[2], r[3]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t b0 = e4m3x2_to_f16x2(r[j], 0), b1 = e4m3x2_to_f16x2(r[j], 1);
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt)
+                mma_f16(acc[mt].o[dq * 4 + j], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b0, b1);
+            }
+          }
+        }
+      } else {
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
         const int key = kb + ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
@@ -402,6 +513,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
             mma_bf16(acc[mt].o[2 * dp + 1], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b2, b3);
           }
         }
+      }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_empty + 8 * s);
@@ -456,7 +568,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         for (int mt = 0; mt < MT; ++mt) {
           const TileAcc &A = acc[mt];
           const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-          const float i0 = 1.f / A.l0, i1 = 1.f / A.l1;
+          const float i0 = seg_vscale / A.l0, i1 = seg_vscale / A.l1;
           __nv_bfloat16 *o_lo = out + (size_t)(row0 + r_lo) * dm.d + h * kDh + 2 * tig;
           __nv_bfloat16 *o_hi = out + (size_t)(row0 + r_hi) * dm.d + h * kDh + 2 * tig;
 #pragma unroll
@@ -505,18 +617,62 @@ int cross_attn_ctas() {
   return 2 * sms < kMaxCrossCtas ? 2 * sms : kMaxCrossCtas;
 }
 
-cudaError_t cross_attn_tma_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(cross_attn_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+// Tensor maps of the 8-bit context keys/values, n_blocks = layers * sequences * heads blocks of
+// max_ctx * 64 bytes of keys followed by max_ctx * 64 bytes of transposed values.  Keys: the whole buffer
+// as lines of 128 bytes (two keys each), boxes of 64 lines; values: [block][64 dims][max_ctx], boxes of
+// 128 keys x 64 dims.  Both with the 128-byte swizzle; reads beyond max_ctx are filled with zeros.
+cudaError_t encode_ctx_kv8_tensor_maps(CUtensorMap *map_k, CUtensorMap *map_v, const void *base, uint64_t n_blocks, uint64_t ctx,
+                                       int *driver_code) {
+  typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  if (driver_code) *driver_code = 0;
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(cross_attn_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+  if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+  {
+    cuuint64_t gdim[2] = {128, (cuuint64_t)(n_blocks * 2 * ctx * kDh / 128)};
+    cuuint64_t gstride[1] = {128};
+    cuuint32_t box[2] = {128, (cuuint32_t)(XK / 2)};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = ((EncodeFn)fn)(map_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { if (driver_code) *driver_code = (int)r; return cudaErrorInvalidValue; }
+  }
+  {
+    cuuint64_t gdim[3] = {(cuuint64_t)ctx, (cuuint64_t)kDh, (cuuint64_t)(n_blocks * 2)};
+    cuuint64_t gstride[2] = {(cuuint64_t)ctx, (cuuint64_t)ctx * kDh};
+    cuuint32_t box[3] = {(cuuint32_t)XK, (cuuint32_t)kDh, 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = ((EncodeFn)fn)(map_v, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), gdim, gstride, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { if (driver_code) *driver_code = (int)r; return cudaErrorInvalidValue; }
+  }
+  return cudaSuccess;
+}
+
+cudaError_t cross_attn_tma_prepare() {
+  cudaError_t e = cudaFuncSetAttribute(cross_attn_tma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+  return e;
 }
 
 // n_ctas persistent CTAs (two per SM); a.part_o holds cross_attn_tma_partial_bytes(n_ctas, C),
 // a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed).
-cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, int n_ctas, cudaStream_t s) {
+// 8-bit keys/values (a.kv_scale set): tmap = the keys' lines, tmap_v = the transposed values; else tmap alone.
+cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, const CUtensorMap &tmap_v, int n_ctas, cudaStream_t s) {
   int mt = (a.dm.C + 15) / 16;
-  if (mt == 1) cross_attn_tma_kernel<1><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, a);
-  else if (mt == 2) cross_attn_tma_kernel<2><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, a);
+  const bool fp8 = a.kv_scale != nullptr;
+  if (mt == 1 && !fp8) cross_attn_tma_kernel<1, false><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
+  else if (mt == 2 && !fp8) cross_attn_tma_kernel<2, false><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
+  else if (mt == 1) cross_attn_tma_kernel<1, true><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
+  else if (mt == 2) cross_attn_tma_kernel<2, true><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }

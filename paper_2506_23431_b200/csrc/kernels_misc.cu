@@ -1,5 +1,7 @@
 // Small kernels of the decode step: state reset, embedding gather, RMSNorm, ReLU,
 // KV-append with the positional write.
+#include <cuda_fp8.h>
+
 #include "pd_internal.h"
 
 namespace pd {
@@ -316,6 +318,88 @@ cudaError_t launch_ctx_kv_relayout(const Dims &dm, int b0, int batch, int layer,
                                    cudaStream_t s) {
   const int esize = dtype == PD_DTYPE_BF16 ? 2 : 4;
   ctx_kv_relayout_kernel<<<148 * 8, 256, 0, s>>>(dm, b0, batch, layer, esize, (const uint4 *)proj, (uint4 *)kv_c);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// 8-bit storage of the context keys/values (E4M3, one scale per (layer, sequence, head, keys | values)).
+// proj holds [position][k of all heads | v of all heads] in bf16 for sequences b0 .. b0 + nb - 1.
+// Pass 1: scale = max|.| / 448 over the positions below ctx_len (1 when all are zero).
+__global__ void __launch_bounds__(256) ctx_kv_amax_kernel(Dims dm, int b0, int layer, const __nv_bfloat16 *__restrict__ proj,
+                                                          const int32_t *__restrict__ ctx_len, float *__restrict__ scale,
+                                                          float *__restrict__ amax) {
+  __shared__ float red[8];
+  const int h = blockIdx.x >> 1, kv = blockIdx.x & 1, b = blockIdx.y;
+  const int n = min(max(ctx_len[b0 + b], 0), dm.ctx);
+  const __nv_bfloat16 *base = proj + (size_t)b * dm.ctx * 2 * dm.d + (size_t)kv * dm.d + (size_t)h * kDh;
+  float m = 0.f;
+  for (int idx = threadIdx.x; idx < n * 8; idx += 256) {               // one 16-byte chunk (8 values) per thread and iteration
+    const int pos = idx >> 3, c = idx & 7;
+    const uint4 v = *reinterpret_cast<const uint4 *>(base + (size_t)pos * 2 * dm.d + c * 8);
+    const __nv_bfloat162 *p2 = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) m = fmaxf(m, fmaxf(fabsf(__low2float(p2[j])), fabsf(__high2float(p2[j]))));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]);
+    const size_t i = ((((size_t)layer * dm.B + b0 + b) * dm.H + h) << 1) + kv;
+    scale[i] = m > 0.f ? __fdiv_rn(m, 448.f) : 1.f;
+    amax[i] = m;
+  }
+}
+
+// Pass 2: codes.  Keys as [position][64] (two keys per 128-byte line), values transposed as [dim][max_ctx],
+// both inside the block of (layer, sequence, head): keys at + 0, values at + max_ctx * 64 bytes.  A value's
+// code is the nearest E4M3 number (ties to even, saturating) of value * (448 / max|.|), the product
+// rounded to fp32; positions at or beyond ctx_len become zeros.
+__global__ void __launch_bounds__(256) ctx_kv_quant_kernel(Dims dm, int b0, int layer, const __nv_bfloat16 *__restrict__ proj,
+                                                           const int32_t *__restrict__ ctx_len, const float *__restrict__ amax,
+                                                           uint8_t *__restrict__ kv8) {
+  __shared__ uint8_t vt[64][80];                      // this tile's value codes, [position][dim], rows padded to 80 bytes
+  const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int n = min(max(ctx_len[b0 + b], 0), dm.ctx);
+  const size_t blk = (((size_t)layer * dm.B + b0 + b) * dm.H + h) * 2;
+  const float mk = amax[blk], mv = amax[blk + 1];
+  const float ik = mk > 0.f ? __fdiv_rn(448.f, mk) : 1.f, iv = mv > 0.f ? __fdiv_rn(448.f, mv) : 1.f;
+  uint8_t *kblock = kv8 + blk * (size_t)dm.ctx * kDh, *vblock = kblock + (size_t)dm.ctx * kDh;
+  const int t = threadIdx.x, pl = t >> 2, c = t & 3;          // position within the tile, 16-value chunk
+  const int pos = tile * 64 + pl;
+  const __nv_bfloat16 *row = proj + ((size_t)b * dm.ctx + pos) * 2 * dm.d + (size_t)h * kDh + c * 16;
+  uint32_t kc[4] = {0u, 0u, 0u, 0u}, vc[4] = {0u, 0u, 0u, 0u};
+  if (pos < n) {
+    uint4 kin[2], vin[2];
+    kin[0] = *reinterpret_cast<const uint4 *>(row); kin[1] = *reinterpret_cast<const uint4 *>(row + 8);
+    vin[0] = *reinterpret_cast<const uint4 *>(row + dm.d); vin[1] = *reinterpret_cast<const uint4 *>(row + dm.d + 8);
+    const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(kin), *v2 = reinterpret_cast<const __nv_bfloat162 *>(vin);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float2 kf = make_float2(__fmul_rn(__low2float(k2[j]), ik), __fmul_rn(__high2float(k2[j]), ik));
+      const float2 vf = make_float2(__fmul_rn(__low2float(v2[j]), iv), __fmul_rn(__high2float(v2[j]), iv));
+      kc[j >> 1] |= (uint32_t)__nv_cvt_float2_to_fp8x2(kf, __NV_SATFINITE, __NV_E4M3) << (16 * (j & 1));
+      vc[j >> 1] |= (uint32_t)__nv_cvt_float2_to_fp8x2(vf, __NV_SATFINITE, __NV_E4M3) << (16 * (j & 1));
+    }
+  }
+  if (pos < dm.ctx) *reinterpret_cast<uint4 *>(kblock + (size_t)pos * kDh + c * 16) = make_uint4(kc[0], kc[1], kc[2], kc[3]);
+  *reinterpret_cast<uint4 *>(&vt[pl][c * 16]) = make_uint4(vc[0], vc[1], vc[2], vc[3]);
+  __syncthreads();
+  // transposed write: thread = (dim, 16 positions)
+  const int dim = t >> 2, p0 = (t & 3) * 16;
+  uint32_t o[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int j = 0; j < 16; ++j) o[j >> 2] |= (uint32_t)vt[p0 + j][dim] << (8 * (j & 3));
+  if (tile * 64 + p0 < dm.ctx)                       // max_ctx is a multiple of 16: a chunk is inside or outside as a whole
+    *reinterpret_cast<uint4 *>(vblock + (size_t)dim * dm.ctx + tile * 64 + p0) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// scale, amax: [layer][sequence][head][keys | values] fp32 each.
+cudaError_t launch_ctx_kv_quantize(const Dims &dm, int b0, int batch, int layer, const void *proj, const int32_t *ctx_len_dev,
+                                   float *scale, float *amax, void *kv8, cudaStream_t s) {
+  ctx_kv_amax_kernel<<<dim3(dm.H * 2, batch), 256, 0, s>>>(dm, b0, layer, (const __nv_bfloat16 *)proj, ctx_len_dev, scale, amax);
+  ctx_kv_quant_kernel<<<dim3((dm.ctx + 63) / 64, dm.H, batch), 256, 0, s>>>(dm, b0, layer, (const __nv_bfloat16 *)proj, ctx_len_dev,
+                                                                            amax, (uint8_t *)kv8);
   return cudaGetLastError();
 }
 

@@ -25,7 +25,7 @@ struct Layout {
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
       w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, w_crow, state_words;
   Region state, plist, row_meta, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
-      ffn, logits, vpart_val, vpart_idx, vterm, part_o, part_ml, kv_c, kv_pool, enc_stage, proj_stage, cublas_ws;
+      ffn, logits, vpart_val, vpart_idx, vterm, part_o, part_ml, kv_c, kv_scale, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
 };
 
@@ -43,6 +43,8 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   for (int v : ids) if (v < 0 || v >= c.vocab) return false;
   if (c.self_splits < 0 || c.self_splits > 32 || c.cross_splits < 0 || c.cross_splits > 32) return false;
   if (c.store_logits != 0 && c.store_logits != 1) return false;
+  if (c.kv_c_dtype != PD_KV_SAME && c.kv_c_dtype != PD_KV_E4M3) return false;
+  if (c.kv_c_dtype == PD_KV_E4M3 && (c.dtype != PD_DTYPE_BF16 || (c.max_ctx % 16) != 0)) return false;
   if (!(c.attn_scale > 0.f) || !(c.norm_eps >= 0.f)) return false;
   dm.L = c.n_layers; dm.d = c.d_model; dm.H = c.n_heads; dm.ff = c.d_ff; dm.V = c.vocab;
   dm.B = c.max_batch; dm.ctx = c.max_ctx; dm.SM = c.sub_max; dm.dt = c.delta_t; dm.T = c.time_max;
@@ -59,6 +61,7 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   dm.pos_mode = c.pos_mode;
   dm.n_dist = c.time_max + c.sub_max + 2;
   if (c.pos_mode == PD_POS_T5_BIAS && dm.n_dist > 512) return false;
+  if (c.kv_c_dtype == PD_KV_E4M3 && dm.C > 32) return false;          // the 8-bit keys/values are read by the tensor-core kernel only
   dm.scale_log2e = c.attn_scale * 1.4426950408889634f;
   dm.eps = c.norm_eps;
   max_splits = 32;
@@ -117,7 +120,13 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
     reg(L.part_o, split_bytes > flat_bytes ? split_bytes : flat_bytes);
   }
   reg(L.part_ml, M * dm.H * max_splits * 2 * 4);
-  reg(L.kv_c, (size_t)dm.L * B * dm.ctx * 2 * dm.d * e);
+  if (c.kv_c_dtype == PD_KV_E4M3) {
+    reg(L.kv_c, (size_t)dm.L * B * dm.ctx * 2 * dm.d);                       // one byte per value
+    reg(L.kv_scale, (size_t)dm.L * B * dm.H * 2 * sizeof(float) * 2);        // scales, then the maxima they come from
+  } else {
+    reg(L.kv_c, (size_t)dm.L * B * dm.ctx * 2 * dm.d * e);
+    reg(L.kv_scale, 0);
+  }
   reg(L.kv_pool, (size_t)dm.L * dm.pool * 2 * dm.H * dm.P * kDh * e);
   reg(L.enc_stage, B * dm.ctx * dm.d * e);
   reg(L.proj_stage, B * dm.ctx * 2 * dm.d * e);
@@ -146,8 +155,9 @@ struct pd_handle {
   DecState st;
   std::vector<const void *> layer_w;
   pd_weights w;
-  CUtensorMap tmap_kvc;
+  CUtensorMap tmap_kvc, tmap_kvc_v;   // context keys/values (8-bit storage: the keys' lines and the transposed values)
   bool have_tmap = false;
+  bool kv8 = false;
   CUtensorMap vmap_a, vmap_b;      // hidden rows and lm_head for the tcgen05 vocabulary projection
   bool vocab_tc = false;
   // pd_generate_host: host-to-device copies of the encoder memory run on a stream of their own, in
@@ -297,6 +307,7 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.bias_tab = h->cfg.pos_mode == PD_POS_T5_BIAS ? h->ptr<float>(h->lay.bias_tab) : nullptr;
   a.qkv = h->ptr<void>(h->lay.qkv);
   a.fused_append = self && fused_append(h) ? 1 : 0;
+  a.kv_scale = (!self && h->kv8) ? h->ptr<float>(h->lay.kv_scale) : nullptr;
   return a;
 }
 
@@ -322,7 +333,7 @@ pd_status enqueue_cross_attention(pd_handle *h, int layer) {
   const int dt = h->cfg.dtype;
   AttnArgs a = attn_args(h, layer, false);
   if (dt == PD_DTYPE_BF16 && h->have_tmap && cross_attn_tma_supported(h->dm, h->batch)) {
-    CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, h->cross_ctas, h->stream));   // merges its own partials
+    CU_TRY(h, launch_cross_attn_tma(a, h->tmap_kvc, h->kv8 ? h->tmap_kvc_v : h->tmap_kvc, h->cross_ctas, h->stream));   // merges its own partials
     h->own_launches++;
     return PD_OK;
   }
@@ -419,7 +430,9 @@ int t5_bucket(int dist, int num_buckets, int max_dist) {
 pd_status make_tensor_map(pd_handle *h) {
   const Dims &dm = h->dm;
   int code = 0;
-  cudaError_t e = encode_ctx_kv_tensor_map(&h->tmap_kvc, h->ptr<void>(h->lay.kv_c), (uint64_t)dm.L * dm.B * dm.H * 2 * dm.ctx, &code);
+  cudaError_t e = h->kv8 ? encode_ctx_kv8_tensor_maps(&h->tmap_kvc, &h->tmap_kvc_v, h->ptr<void>(h->lay.kv_c), (uint64_t)dm.L * dm.B * dm.H,
+                                                      (uint64_t)dm.ctx, &code)
+                         : encode_ctx_kv_tensor_map(&h->tmap_kvc, h->ptr<void>(h->lay.kv_c), (uint64_t)dm.L * dm.B * dm.H * 2 * dm.ctx, &code);
   if (e != cudaSuccess) return fail(h, PD_ERR_CUDA, std::string("tensor map for the context keys/values: ") + cudaGetErrorString(e) +
                                                     " (driver code " + std::to_string(code) + ")");
   h->have_tmap = true;
@@ -531,6 +544,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
       (launch_build_bias_table(dm, weights->rel_bias, cfg->rel_buckets, h->ptr<int32_t>(L.dist_bucket), h->ptr<float>(L.bias_tab),
                                h->stream) != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess))
     return bail(PD_ERR_CUDA);
+  h->kv8 = cfg->kv_c_dtype == PD_KV_E4M3;
   if (cfg->dtype == PD_DTYPE_BF16 && dm.C <= 32) {
     pd_status s = make_tensor_map(h);
     if (s != PD_OK) return bail(s);
@@ -626,7 +640,14 @@ pd_status encode_project(pd_handle *h, const void *enc_mem, int b0, int nb) {
   for (int l = 0; l < dm.L; ++l) {
     PD_TRY(gemm(h, false, nb * dm.ctx, 2 * dm.d, dm.d, enc_mem, h->layer_w[(size_t)l * kLayerTensors + 5],
                 h->ptr<void>(L.proj_stage), false, 0.f));
-    OWN(h, PD_PROF_OTHER, launch_ctx_kv_relayout(dm, b0, nb, l, h->cfg.dtype, h->ptr<void>(L.proj_stage), h->ptr<void>(L.kv_c), h->stream));
+    if (h->kv8) {
+      float *scale = h->ptr<float>(L.kv_scale);
+      OWN(h, PD_PROF_OTHER, launch_ctx_kv_quantize(dm, b0, nb, l, h->ptr<void>(L.proj_stage), h->st.ctx_len, scale,
+                                                   scale + (size_t)dm.L * dm.B * dm.H * 2, h->ptr<void>(L.kv_c), h->stream));
+      h->own_launches++;   // two launches
+    } else {
+      OWN(h, PD_PROF_OTHER, launch_ctx_kv_relayout(dm, b0, nb, l, h->cfg.dtype, h->ptr<void>(L.proj_stage), h->ptr<void>(L.kv_c), h->stream));
+    }
   }
   return PD_OK;
 }

@@ -100,6 +100,8 @@ struct AttnArgs {
   // output [rows][3 d] in bf16
   const void *qkv;
   int fused_append;
+  // cross-attention over 8-bit keys/values: [layer][sequence][head][keys | values] fp32 scales (else null)
+  const float *kv_scale;
 };
 
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
@@ -121,7 +123,11 @@ cudaError_t launch_ctx_kv_relayout(const Dims &dm, int b0, int batch, int layer,
 cudaError_t launch_attn_core(const AttnArgs &a, int dtype, bool self, cudaStream_t s);
 cudaError_t launch_attn_merge(const AttnArgs &a, int dtype, cudaStream_t s);
 constexpr int kMaxCrossCtas = 320;      // persistent cross-attention CTAs (two per SM) the scratch is sized for
-cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, int n_ctas, cudaStream_t s);
+cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, const CUtensorMap &tmap_v, int n_ctas, cudaStream_t s);
+cudaError_t encode_ctx_kv8_tensor_maps(CUtensorMap *map_k, CUtensorMap *map_v, const void *base, uint64_t n_blocks, uint64_t ctx,
+                                       int *driver_code);
+cudaError_t launch_ctx_kv_quantize(const Dims &dm, int b0, int batch, int layer, const void *proj, const int32_t *ctx_len_dev,
+                                   float *scale, float *amax, void *kv8, cudaStream_t s);
 size_t cross_attn_tma_partial_bytes(int n_ctas, int rows_per_seq);
 bool cross_attn_tma_supported(const Dims &dm, int batch);
 int cross_attn_ctas();                  // 2 x SM count of the current device, capped at kMaxCrossCtas

@@ -55,6 +55,7 @@ class Workload:
     weight_std: float = 0.02
     rel_bias_std: float = 0.5
     norm_gain_std: float = 0.0   # 0 => all norm gains are exactly 1
+    kv_c_dtype: str = "same"     # "e4m3": cross-attention keys/values stored as 8-bit floats (an option of the build)
 
     @property
     def attn_scale(self) -> float:

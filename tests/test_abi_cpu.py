@@ -69,6 +69,7 @@ def test_invalid_configurations_are_rejected_on_the_host():
     assert ws(dtype=7) == 0
     assert ws(sep_id=10 ** 6) == 0
     assert ws(pos_mode=3) == 0
+    assert ws(kv_c_dtype=1) == 0                       # 8-bit context keys/values need the bf16 path
     assert B._lib.pd_workspace_bytes(None) == 0
     # pd_init refuses null pointers and bad configs before touching CUDA
     h = C.c_void_p()

@@ -319,6 +319,30 @@ def test_two_identical_decodes_give_identical_logits():
     dec.close()
 
 
+@pytest.mark.parametrize("pos_mode", [W.POS_T5_BIAS, W.POS_ROPE])
+def test_small_bf16_with_e4m3_context_keys_values(pos_mode):
+    """The 8-bit storage of the cross-attention keys/values against the oracle that quantises likewise:
+    ragged contexts (a context of less than one tile, a tile edge, zero-filled tails), three layers."""
+    wl = W.CONFIGS["bart_base"].scaled(name="small_e4m3", batch=4, ctx=304, sub_max=6, delta_t=2, max_sub_len=40,
+                                       length_dist=("uniform", 1, 40), time_max=60, pos_mode=pos_mode, kv_c_dtype="e4m3",
+                                       **dict(SMALL_BF16, n_layers=3))
+    weights, mem, _, dec, rows = make(wl)
+    ctx_len = np.array([304, 100, 257, 129], dtype=np.int32)
+    fl = W.make_forced_len(wl)
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, fl)
+    stats = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    assert stats["max_err"] < 2e-2 and stats["choices"] > 0
+    dec.close()
+
+
+def test_small_bf16_e4m3_two_query_tiles_and_long_context():
+    """Twenty rows per sequence (two 16-row query tiles) over 2000 context positions: several CTAs per
+    (sequence, head) segment, partial records merged by ticket, all on 8-bit keys/values."""
+    wl = W.CONFIGS["keyphrase"].scaled(name="small_kp8", batch=2, ctx=2000, sub_max=24, delta_t=1, max_sub_len=19,
+                                       length_dist=("uniform", 3, 19), time_max=48, kv_c_dtype="e4m3", **SMALL_BF16)
+    check(wl, ragged=True, free_run=False)
+
+
 def test_split_self_attention_merges_in_the_launch_and_repeats_bit_for_bit():
     """Long page lists with four splits per (sequence, head): the split CTAs leave partial records and the
     last one to arrive merges them in split order, so twenty decodes of the same inputs must give the same
@@ -399,6 +423,21 @@ def test_full_size_configs_with_ragged_contexts(name, tol):
     s = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs, use_logits=False)
     assert s["choices"] > 0
     dec.close()
+
+
+def test_full_size_summarisation_with_e4m3_context_keys_values():
+    """The largest configuration with the 8-bit storage of the context keys/values (half of a step's dominant
+    byte term), logits element by element against the oracle that quantises likewise."""
+    from paper_2506_23431_b200.binding import PipelinedDecoder
+    wl = W.CONFIGS["summarisation"].scaled(kv_c_dtype="e4m3")
+    weights, mem = W.make_weights(wl), W.make_encoder_memory(wl)
+    ctx_len, fl = W.make_ctx_len(wl, ragged=True), W.make_forced_len(wl)
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in (0, wl.batch - 1)}, ctx_len, fl)
+    dec = PipelinedDecoder(wl.hyper(), weights, wl.batch)
+    s = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    assert s["max_err"] <= 2e-2 and s["choices"] > 0
+    dec.close()
+    print(f"summarisation e4m3: max logit error {s['max_err']:.3e}, {s['choices']} choices, {s['low_margin']} below margin")
 
 
 @pytest.mark.parametrize("store_logits", [True, False])
