@@ -266,6 +266,8 @@ def main():
                     help="run exactly one encode + decode and exit (no timing): the command profilers are pointed at")
     ap.add_argument("--time-steps", type=int, default=0,
                     help="with --single-decode: stop after this many time-steps (0 = until done)")
+    ap.add_argument("--kv-c-dtype", default="same", choices=["same", "e4m3"],
+                    help="storage of the cross-attention keys/values for the main measurement (profiling the 8-bit kernel)")
     ap.add_argument("--self-splits", type=int, default=0)
     ap.add_argument("--cross-splits", type=int, default=0)
     args = ap.parse_args()
@@ -300,6 +302,8 @@ def main():
     wl = W.CONFIGS[args.config]
     if args.batch > 0:
         wl = wl.scaled(batch=args.batch)
+    if args.kv_c_dtype != "same":
+        wl = wl.scaled(kv_c_dtype=args.kv_c_dtype)
     weights = W.make_weights(wl)                 # replicated on every rank
     wl_data = rank_workload(wl, rank)            # this rank's sequences
     mem = W.make_encoder_memory(wl_data)

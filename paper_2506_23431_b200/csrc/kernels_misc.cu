@@ -351,7 +351,9 @@ __global__ void __launch_bounds__(256) ctx_kv_amax_kernel(Dims dm, int b0, int l
   }
 }
 
-// Pass 2: codes.  Keys as [position][64] (two keys per 128-byte line), values transposed as [dim][max_ctx],
+// Pass 2: codes.  Keys as [position][64] (two keys per 128-byte line; inside every group of 16 positions
+// key g sits at place 8 * ((g >> 1) & 1) + 2 * (g >> 2) + (g & 1): the order the attention kernel's score
+// tiles take them in, which keeps its ldmatrix rows in different banks), values transposed as [dim][max_ctx],
 // both inside the block of (layer, sequence, head): keys at + 0, values at + max_ctx * 64 bytes.  A value's
 // code is the nearest E4M3 number (ties to even, saturating) of value * (448 / max|.|), the product
 // rounded to fp32; positions at or beyond ctx_len become zeros.
@@ -382,7 +384,8 @@ __global__ void __launch_bounds__(256) ctx_kv_quant_kernel(Dims dm, int b0, int 
       vc[j >> 1] |= (uint32_t)__nv_cvt_float2_to_fp8x2(vf, __NV_SATFINITE, __NV_E4M3) << (16 * (j & 1));
     }
   }
-  if (pos < dm.ctx) *reinterpret_cast<uint4 *>(kblock + (size_t)pos * kDh + c * 16) = make_uint4(kc[0], kc[1], kc[2], kc[3]);
+  const int g16 = pos & 15, place = (pos & ~15) | ((((g16 >> 1) & 1) << 3) + ((g16 >> 2) << 1) + (g16 & 1));
+  if (pos < dm.ctx) *reinterpret_cast<uint4 *>(kblock + (size_t)place * kDh + c * 16) = make_uint4(kc[0], kc[1], kc[2], kc[3]);
   *reinterpret_cast<uint4 *>(&vt[pl][c * 16]) = make_uint4(vc[0], vc[1], vc[2], vc[3]);
   __syncthreads();
   // transposed write: thread = (dim, 16 positions)
