@@ -207,6 +207,51 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def continuous_batching(dec, wl: W.Workload, mem_dev, ctx_len, fl, queue_factor: int = 4, poll_every: int = 4):
+    """A queue of queue_factor x batch sequences decoded through the batch's rows: whenever a row's sequence has
+    ended (looked at every poll_every steps), its streams are collected and the next sequence of the queue is
+    admitted into the row (pd_admit: context projection of that sequence + row reset, inside the timed region).
+    The queue repeats the workload's sequences, so the token count is queue_factor x the one-shot count.
+    Steady-state throughput of a serving loop, beside the one-shot decode of a single batch."""
+    import torch
+    B = wl.batch
+    n_queue = queue_factor * B
+    seqs = [mem_dev[q].contiguous() for q in range(B)]
+    out = None
+    for _ in range(2):                                       # one warm-up pass, one timed
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dec.encode_context(mem_dev, ctx_len, fl)
+        torch.cuda.synchronize()
+        a.record(dec.stream)
+        row_live = [True] * B
+        next_q, steps, collected_tokens = B, 0, 0
+        while any(row_live):
+            for _ in range(poll_every):
+                dec.step()
+            steps += poll_every
+            done, _ = dec.rows_done()
+            for row in range(B):
+                if row_live[row] and done[row]:
+                    res = dec.collect_row(row)
+                    collected_tokens += int(res["lens"][: res["n_sub"]].sum()) + res["n_sub"]
+                    if next_q < n_queue:
+                        q = next_q % B
+                        dec.admit(row, seqs[q], int(ctx_len[q]), fl[q])
+                        next_q += 1
+                    else:
+                        row_live[row] = False
+        b.record(dec.stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b)
+        tokens = int(dec.stats()["tokens"])
+        assert tokens == collected_tokens, "tokens counted on the device differ from the collected streams"
+        out = {"value": tokens / (ms * 1e-3), "unit": UNIT, "rows": B, "queue": n_queue, "tokens": tokens, "time_steps": steps,
+               "ms_per_time_step": ms / steps, "tokens_per_time_step": tokens / steps, "poll_every": poll_every,
+               "note": "steady-state serving loop: context projection of every admitted sequence, row resets and the "
+                       "polling synchronisations are inside the timed region; the first batch's projection is not"}
+    return out
+
+
 def spawn_ranks(n: int) -> int:
     """`python bench.py --gpus N` without a launcher: start N ranks of this same command (one process per
     GPU) through torch.distributed.run on the loopback address and hand back its exit code.  Rank 0's
@@ -256,6 +301,8 @@ def main():
     ap.add_argument("--no-sequential", action="store_true",
                     help="skip the sequential decoder (sub_max = 1 on the same targets), which is otherwise timed beside the "
                          "pipelined one at N = 1 for the speed-up the paper's tables report")
+    ap.add_argument("--no-queue", action="store_true",
+                    help="skip the continuous-batching leg (a queue of 4 x batch sequences through the batch's rows)")
     ap.add_argument("--no-kv8", action="store_true",
                     help="skip the extra decode with the cross-attention keys/values stored as 8-bit floats (reported as e4m3_context_kv)")
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend for N > 1")
@@ -459,6 +506,8 @@ def main():
     att = [r["frac"] for r in (roofline, roofline_self) if r]
     if att:
         line["roofline_min_attention_frac"] = min(att)
+    if rank == 0 and world == 1 and not args.no_queue:
+        line["continuous_batching"] = continuous_batching(dec, wl, mem_dev, ctx_len, fl, poll_every=4)
     if rank == 0 and world == 1 and not args.no_kv8 and wl.dtype == "bf16" and wl.ctx % 16 == 0 and dec.rows_per_seq <= 32:
         # the same job with the cross-attention keys/values stored as 8-bit floats (an option of the build; the headline stays bf16)
         dec.close()

@@ -161,6 +161,28 @@ PD_API pd_status pd_done(pd_handle *h, int32_t *all_done);
 PD_API pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags,
                      int32_t *steps);
 
+/* Continuous batching: a new sequence in a row whose sequence has ended, between two steps (Algorithm 1
+ * runs per sequence; rows only share the step clock).  The row starts over as pd_encode_context would leave
+ * it - state cleared, subsequence 1 admitted, its own step counter at 1 for the coming pd_step, its pages its
+ * own again - and the context's keys/values are projected into the row's slice.  The other rows carry on
+ * untouched; the result of the row's sequence is what the sequence gives decoded alone.  Take the previous
+ * sequence's result first (pd_collect_row).
+ *   row        0 .. batch-1 of the last pd_encode_context; its sequence should have ended (pd_rows_done)
+ *   enc_mem    device [max_ctx, d_model] of cfg.dtype;  ctx_len 1..max_ctx;  forced_len host [sub_max] or NULL
+ * Needs the default page pool (cfg.pool_pages = 0), else PD_ERR_UNSUPPORTED.  Enqueues on the handle's stream;
+ * call it between pd_step calls (not while pd_run is running).  pd_run / pd_done report "all done" again only
+ * when every row's current sequence has ended. */
+PD_API pd_status pd_admit(pd_handle *h, int32_t row, const void *enc_mem, int32_t ctx_len, const int32_t *forced_len);
+
+/* done[b] = 1 when row b's current sequence has ended (host [batch]); steps[b] (host [batch] or NULL) = the step
+ * of the sequence's own clock at which it stopped.  Synchronises; returns a pending device error if any. */
+PD_API pd_status pd_rows_done(pd_handle *h, int32_t *done, int32_t *steps);
+
+/* pd_collect for one row: tokens host [sub_max, max_sub_len], lens [sub_max], n_sub [1], flags [sub_max],
+ * steps [1] (any may be NULL).  Synchronises. */
+PD_API pd_status pd_collect_row(pd_handle *h, int32_t row, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags,
+                                int32_t *steps);
+
 /* Whole Algorithm 1 from host buffers: copies enc_mem (host [batch, max_ctx, d_model], dtype;
  * pinned memory lets the copy overlap) to the device in chunks of sequences on a copy stream of
  * the handle's own while the context projection of the chunks already there runs on the handle's
@@ -171,7 +193,8 @@ PD_API pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const 
                            int32_t *flags, int32_t *steps);
 
 /* Schedule trace: active_mask[(t-1)*batch + b] has bit i-1 set iff subsequence i of sequence b
- * emitted a token at step t.  Host [time_max, batch].  Synchronises. */
+ * emitted a token at step t of the sequence's own clock (a row's column starts over with pd_admit).
+ * Host [time_max, batch].  Synchronises. */
 PD_API pd_status pd_get_trace(pd_handle *h, uint64_t *active_mask);
 
 /* Parity/debug: fp32 logits of the last executed step, host [rows, vocab] with

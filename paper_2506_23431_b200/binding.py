@@ -54,6 +54,9 @@ _SIGS = {
     "pd_run": (C.c_int, [_H, C.c_int32, _i32p]),
     "pd_done": (C.c_int, [_H, _i32p]),
     "pd_collect": (C.c_int, [_H, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "pd_admit": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int32, _i32p]),
+    "pd_rows_done": (C.c_int, [_H, _i32p, _i32p]),
+    "pd_collect_row": (C.c_int, [_H, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "pd_generate_host": (C.c_int, [_H, C.c_void_p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "pd_get_trace": (C.c_int, [_H, C.POINTER(C.c_uint64)]),
     "pd_get_logits": (C.c_int, [_H, C.POINTER(C.c_float), _i32p]),
@@ -238,6 +241,31 @@ class PipelinedDecoder:
         steps = np.empty((b,), np.int32)
         self._check(_lib.pd_collect(self._h, _p(tokens), _p(lens), _p(n_sub), _p(flags), _p(steps)), "pd_collect")
         return {"tokens": tokens, "lens": lens, "n_sub": n_sub, "flags": flags, "steps": steps}
+
+    def admit(self, row: int, enc_mem, ctx_len: int, forced_len=None):
+        """A new sequence in `row` (whose sequence has ended): enc_mem torch CUDA tensor [ctx, d] of the model dtype."""
+        if tuple(enc_mem.shape) != (self.cfg.max_ctx, self.cfg.d_model) or enc_mem.dtype != self.tdtype \
+                or not enc_mem.is_contiguous() or not enc_mem.is_cuda:
+            raise ValueError("enc_mem must be a contiguous CUDA tensor [max_ctx, d_model] of the model dtype")
+        fl = None if forced_len is None else _np_i32(forced_len, (self.cfg.sub_max,))
+        self.stream.wait_stream(self.torch.cuda.current_stream(self.device))
+        self._keep.append(enc_mem)
+        self._check(_lib.pd_admit(self._h, int(row), C.c_void_p(enc_mem.data_ptr()), int(ctx_len), _p(fl)), "pd_admit")
+
+    def rows_done(self):
+        done = np.empty((self.batch,), np.int32)
+        steps = np.empty((self.batch,), np.int32)
+        self._check(_lib.pd_rows_done(self._h, _p(done), _p(steps)), "pd_rows_done")
+        return done, steps
+
+    def collect_row(self, row: int):
+        sm, msl = self.cfg.sub_max, self.cfg.max_sub_len
+        tokens = np.empty((sm, msl), np.int32)
+        lens = np.empty((sm,), np.int32)
+        flags = np.empty((sm,), np.int32)
+        n_sub, steps = np.empty((1,), np.int32), np.empty((1,), np.int32)
+        self._check(_lib.pd_collect_row(self._h, int(row), _p(tokens), _p(lens), _p(n_sub), _p(flags), _p(steps)), "pd_collect_row")
+        return {"tokens": tokens, "lens": lens, "n_sub": int(n_sub[0]), "flags": flags, "steps": int(steps[0])}
 
     def generate_host(self, enc_mem_host, ctx_len, forced_len=None):
         """enc_mem_host: host buffer (torch CPU tensor, ideally pinned, or numpy array) of the model

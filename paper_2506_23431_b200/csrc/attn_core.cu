@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(NT) attn_core_kernel(AttnArgs a) {
   // (the stand-alone op reads caller-written counts: clamped, so that no access leaves the tensors)
   const int S = min(max(a.st.n_active[b], 0), min(dm.C, kMaxRows));
   const int row0 = b * dm.C;
-  const int t = SELF ? a.st.hdr[HDR_STEP_T] : 0;
+  const int t = SELF ? a.st.hdr[HDR_STEP_T] - a.st.t0[b] : 0;        // the sequence's own step
   const T *qbuf = (const T *)a.q;
   T *out = (T *)a.out;
 

@@ -38,10 +38,11 @@ __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_
     st.start[b * dm.SM] = 1;
     st.state[b * dm.SM] = SUB_ACTIVE;
     st.row_sub[b * dm.C] = 1;
-    st.page_table[(size_t)b * dm.SM * dm.PPS] = (int32_t)b;   // pages 0..batch-1 go to the first subsequences
-    st.plist[(size_t)b * dm.SM * dm.PPS] = make_int4((int)b, 1, 1, -1);  // step 1: bos of subsequence 1 at position 1, d0 = 0 - 1
+    const int pg = dm.pool_static ? (int)b * dm.SM * dm.PPS : (int)b;    // bump allocation: pages 0..batch-1 go to the first subsequences
+    st.page_table[(size_t)b * dm.SM * dm.PPS] = pg;
+    st.plist[(size_t)b * dm.SM * dm.PPS] = make_int4(pg, 1, 1, -1);      // step 1: bos of subsequence 1 at position 1, d0 = 0 - 1
     st.plist_n[b] = 1;
-    st.row_meta[b * dm.C] = make_int4((int)b, 0, 1, 1);                  // bos goes to slot 0 of that page, position 0 + 1
+    st.row_meta[b * dm.C] = make_int4(pg, 0, 1, 1);                      // bos goes to slot 0 of that page, position 0 + 1
     for (int c = 1; c < dm.C; ++c) st.row_meta[b * dm.C + c] = make_int4(0, 0, 0, 0);
   }
   if (gid == 0) {
@@ -50,6 +51,46 @@ __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_
     st.hdr[HDR_PAGE_BUMP] = batch;
     if (batch > dm.pool) st.hdr[HDR_STATUS] = PD_ERR_POOL_EXHAUSTED;
   }
+}
+
+// A new sequence in row b between two steps (the initialisation of Algorithm 1 for this row alone): the row's
+// state as reset_state leaves it, with the row's step origin at the step before the coming one, so that the
+// coming step is its step 1.  Only with the static page mapping (the row's pages are its own).
+__global__ void admit_row_kernel(Dims dm, DecState st, int b, int ctx_len, const int32_t *forced_len) {
+  const int tid = threadIdx.x, n = blockDim.x;
+  const int SM = dm.SM, C = dm.C, NPT = dm.SM * dm.PPS;
+  for (int i = tid; i < SM; i += n) {
+    const int sidx = b * SM + i;
+    st.forced_len[sidx] = forced_len ? forced_len[i] : -1;
+    st.last_tok[sidx] = dm.bos;
+    st.start[sidx] = i == 0 ? 1 : 0; st.len[sidx] = 0; st.state[sidx] = i == 0 ? SUB_ACTIVE : SUB_NONE; st.flag[sidx] = 0;
+  }
+  for (int i = tid; i < SM * (dm.MSL + 1); i += n) st.chosen[(size_t)b * SM * (dm.MSL + 1) + i] = -1;
+  for (int i = tid; i < SM * dm.MSL; i += n) st.tokens[(size_t)b * SM * dm.MSL + i] = -1;
+  for (int i = tid; i < NPT; i += n) st.page_table[(size_t)b * NPT + i] = 0;
+  for (int c = tid; c < C; c += n) {
+    st.row_sub[b * C + c] = c == 0 ? 1 : 0; st.prev_row_sub[b * C + c] = 0; st.row_tok[b * C + c] = 0;
+    st.row_meta[b * C + c] = make_int4(0, 0, 0, 0);
+  }
+  for (int t = tid; t < dm.T; t += n) st.trace[(size_t)t * dm.B + b] = 0ull;
+  __syncthreads();
+  if (tid == 0) {
+    const int pg = b * NPT;
+    st.ctx_len[b] = ctx_len;
+    st.k[b] = 1; st.n_active[b] = 1; st.steps[b] = 0; st.seq_ticket[b] = 0;
+    st.page_table[(size_t)b * NPT] = pg;
+    st.plist[(size_t)b * NPT] = make_int4(pg, 1, 1, -1);
+    st.plist_n[b] = 1;
+    st.row_meta[b * C] = make_int4(pg, 0, 1, 1);
+    st.t0[b] = st.hdr[HDR_STEP_T] - 1;
+    if (st.done[b]) { st.done[b] = 0; atomicSub(&st.hdr[HDR_N_DONE], 1); }
+    st.hdr[HDR_ALL_DONE] = 0;
+  }
+}
+
+cudaError_t launch_admit_row(const Dims &dm, const DecState &st, int row, int ctx_len, const int32_t *forced_len_dev, cudaStream_t s) {
+  admit_row_kernel<<<1, 256, 0, s>>>(dm, st, row, ctx_len, forced_len_dev);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, const int32_t *ctx_len_dev,

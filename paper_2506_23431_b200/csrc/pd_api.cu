@@ -23,7 +23,7 @@ struct Region { size_t off = 0, bytes = 0; };
 struct Layout {
   // integer state (offsets in int32 words from the start of the state block)
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
-      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, w_crow, state_words;
+      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, w_crow, w_t0, state_words;
   Region state, plist, row_meta, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
       ffn, logits, vpart_val, vpart_idx, vterm, part_o, part_ml, kv_c, kv_scale, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
@@ -55,6 +55,7 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   dm.PPS = (c.max_sub_len + 1 + dm.P - 1) / dm.P;
   long long worst = (long long)c.max_batch * c.sub_max * dm.PPS;
   dm.pool = c.pool_pages > 0 ? c.pool_pages : (int)worst;
+  dm.pool_static = c.pool_pages == 0 ? 1 : 0;
   if (c.pool_pages < 0 || worst > 0x7fffffffLL) return false;
   if ((long long)c.n_layers * c.max_batch * c.n_heads * 2 * c.max_ctx > 0x7fffffffLL) return false;   // rows of the context K/V tensor map
   dm.bos = c.bos_id; dm.eos = c.eos_id; dm.sep = c.sep_id;
@@ -78,6 +79,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   L.w_plist_n = take(B);
   L.w_xtick = take(B * dm.H);
   L.w_crow = take(B);
+  L.w_t0 = take(B);
   L.w_k = take(B); L.w_done = take(B); L.w_steps = take(B); L.w_nact = take(B); L.w_ctx = take(B); L.w_ticket = take(B);
   L.w_start = take(B * SM); L.w_len = take(B * SM); L.w_state = take(B * SM); L.w_flag = take(B * SM);
   L.w_last = take(B * SM); L.w_forced = take(B * SM);
@@ -518,7 +520,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   st.hdr = sb + L.w_hdr; st.stats = reinterpret_cast<unsigned long long *>(sb + L.w_stats);
   st.trace = reinterpret_cast<unsigned long long *>(sb + L.w_trace);
   st.k = sb + L.w_k; st.done = sb + L.w_done; st.steps = sb + L.w_steps; st.n_active = sb + L.w_nact;
-  st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket; st.crow = sb + L.w_crow;
+  st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket; st.crow = sb + L.w_crow; st.t0 = sb + L.w_t0;
   st.plist_n = sb + L.w_plist_n; st.plist = h->ptr<int4>(L.plist); st.row_meta = h->ptr<int4>(L.row_meta);
   st.start = sb + L.w_start; st.len = sb + L.w_len; st.state = sb + L.w_state; st.flag = sb + L.w_flag;
   st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced;
@@ -747,6 +749,47 @@ pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_su
   if (n_sub) CU_TRY(h, cudaMemcpyAsync(n_sub, h->st.k, nb * 4, cudaMemcpyDeviceToHost, s));
   if (flags) CU_TRY(h, cudaMemcpyAsync(flags, h->st.flag, nb * dm.SM * 4, cudaMemcpyDeviceToHost, s));
   if (steps) CU_TRY(h, cudaMemcpyAsync(steps, h->st.steps, nb * 4, cudaMemcpyDeviceToHost, s));
+  return device_status(h);
+}
+
+pd_status pd_admit(pd_handle *h, int32_t row, const void *enc_mem, int32_t ctx_len, const int32_t *forced_len) {
+  if (!h) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_admit before pd_encode_context");
+  const Dims &dm = h->dm;
+  if (!enc_mem || row < 0 || row >= h->batch || ctx_len < 1 || ctx_len > dm.ctx) return fail(h, PD_ERR_ARG, "pd_admit: bad argument");
+  if (!dm.pool_static)
+    return fail(h, PD_ERR_UNSUPPORTED, "pd_admit needs the default page pool (pool_pages = 0): a row's pages are then its own and start over with it");
+  if (forced_len)
+    for (int i = 0; i < dm.SM; ++i)
+      if (forced_len[i] > dm.MSL) return fail(h, PD_ERR_ARG, "pd_admit: forced_len exceeds max_sub_len");
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  const Layout &L = h->lay;
+  int32_t *fl_dev = h->ptr<int32_t>(L.forced_in) + (size_t)row * dm.SM;
+  if (forced_len) CU_TRY(h, cudaMemcpyAsync(fl_dev, forced_len, (size_t)dm.SM * 4, cudaMemcpyHostToDevice, h->stream));
+  OWN(h, PD_PROF_OTHER, launch_admit_row(dm, h->st, row, ctx_len, forced_len ? fl_dev : nullptr, h->stream));
+  return encode_project(h, enc_mem, row, 1);
+}
+
+pd_status pd_rows_done(pd_handle *h, int32_t *done, int32_t *steps) {
+  if (!h || !done) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_rows_done before pd_encode_context");
+  CU_TRY(h, cudaMemcpyAsync(done, h->st.done, (size_t)h->batch * 4, cudaMemcpyDeviceToHost, h->stream));
+  if (steps) CU_TRY(h, cudaMemcpyAsync(steps, h->st.steps, (size_t)h->batch * 4, cudaMemcpyDeviceToHost, h->stream));
+  return device_status(h);
+}
+
+pd_status pd_collect_row(pd_handle *h, int32_t row, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags, int32_t *steps) {
+  if (!h) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_collect_row before pd_encode_context");
+  if (row < 0 || row >= h->batch) return fail(h, PD_ERR_ARG, "pd_collect_row: bad row");
+  const Dims &dm = h->dm;
+  cudaStream_t s = h->stream;
+  const size_t r = (size_t)row;
+  if (tokens) CU_TRY(h, cudaMemcpyAsync(tokens, h->st.tokens + r * dm.SM * dm.MSL, (size_t)dm.SM * dm.MSL * 4, cudaMemcpyDeviceToHost, s));
+  if (lens) CU_TRY(h, cudaMemcpyAsync(lens, h->st.len + r * dm.SM, (size_t)dm.SM * 4, cudaMemcpyDeviceToHost, s));
+  if (n_sub) CU_TRY(h, cudaMemcpyAsync(n_sub, h->st.k + r, 4, cudaMemcpyDeviceToHost, s));
+  if (flags) CU_TRY(h, cudaMemcpyAsync(flags, h->st.flag + r * dm.SM, (size_t)dm.SM * 4, cudaMemcpyDeviceToHost, s));
+  if (steps) CU_TRY(h, cudaMemcpyAsync(steps, h->st.steps + r, 4, cudaMemcpyDeviceToHost, s));
   return device_status(h);
 }
 

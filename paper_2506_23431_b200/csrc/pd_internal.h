@@ -57,6 +57,7 @@ struct Dims {
   int P;        // page_tokens
   int PPS;      // pages per subsequence
   int pool;     // pool pages
+  int pool_static;  // the pool holds the worst case: page j of subsequence i of sequence b is page (b SM + i - 1) PPS + j, nothing is allocated
   int bos, eos, sep;
   int pos_mode;
   int n_dist;   // entries of the distance -> bucket table
@@ -69,6 +70,7 @@ struct DecState {
   int32_t *hdr;                 // [HDR_WORDS]
   unsigned long long *stats;    // [PD_STAT_COUNT]
   int32_t *k, *done, *steps, *n_active, *ctx_len, *seq_ticket;        // [B]
+  int32_t *t0;                  // [B] the sequence's step origin: its own step t = header step - t0 (0 unless it was admitted later)
   int32_t *crow;                // [B] first row of the sequence among the step's active rows packed back to back
   int32_t *plist_n;             // [B] entries of the sequence's page list for the coming step
   int4 *row_meta;               // [B*C] per row: (page, slot in it, position tau + i) of the entry the coming step appends, subsequence i (0 = unused row)
@@ -107,6 +109,7 @@ struct AttnArgs {
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
 cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, const int32_t *ctx_len_dev,
                                const int32_t *forced_len_dev, size_t state_words, int32_t *state_base, cudaStream_t s);
+cudaError_t launch_admit_row(const Dims &dm, const DecState &st, int row, int ctx_len, const int32_t *forced_len_dev, cudaStream_t s);
 cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x,
                          cudaStream_t s);
 cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, const void *gain, void *out,

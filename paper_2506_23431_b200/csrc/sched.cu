@@ -56,7 +56,8 @@ __device__ __forceinline__ SeqScalars stage_in(const Dims &dm, const DecState &s
   const int tid = threadIdx.x, nthr = blockDim.x;
   const int C = dm.C, SM = dm.SM, NPT = dm.SM * dm.PPS;
   SeqScalars sc;
-  sc.t = st.hdr[HDR_STEP_T]; sc.nact = st.n_active[b]; sc.k = st.k[b]; sc.done = st.done[b]; sc.status = st.hdr[HDR_STATUS];
+  sc.t = st.hdr[HDR_STEP_T] - st.t0[b];        // the sequence's own step (Algorithm 1 runs per sequence)
+  sc.nact = st.n_active[b]; sc.k = st.k[b]; sc.done = st.done[b]; sc.status = st.hdr[HDR_STATUS];
   for (int c = tid; c < C; c += nthr) v.row_sub[c] = st.row_sub[b * C + c];
   for (int i = tid; i < SM; i += nthr) {
     const int sidx = b * SM + i;
@@ -177,8 +178,10 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqS
       const unsigned nb = __ballot_sync(FULL, need);
       int pg0 = 0;
       if (nb != 0u) {
-        if (lane == 0) pg0 = atomicAdd(&st.hdr[HDR_PAGE_BUMP], __popc(nb));
-        pg0 = __shfl_sync(FULL, pg0, 0);
+        if (!dm.pool_static) {
+          if (lane == 0) pg0 = atomicAdd(&st.hdr[HDR_PAGE_BUMP], __popc(nb));
+          pg0 = __shfl_sync(FULL, pg0, 0);
+        }
         pages += __popc(nb);
       }
       if (on) {
@@ -186,7 +189,7 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqS
           atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_STATE);
         } else {
           if (need) {
-            int pg = pg0 + __popc(nb & lt_mask);
+            int pg = dm.pool_static ? (b * SM + i - 1) * dm.PPS + p / P : pg0 + __popc(nb & lt_mask);
             if (pg >= dm.pool) { atomicExch(&st.hdr[HDR_STATUS], (int)PD_ERR_POOL_EXHAUSTED); pg = 0; }
             v.page_table[(i - 1) * dm.PPS + p / P] = pg;
           }
