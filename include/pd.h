@@ -114,14 +114,22 @@ typedef struct {
   const float *rel_bias;    /* [n_heads, rel_buckets], shared by all layers; may be NULL in RoPE mode */
 } pd_weights;
 
-/* Bytes of device workspace pd_init needs for this configuration (0 if cfg is invalid).
+/* PD_OK if pd_init would accept cfg; PD_ERR_ARG for a field out of range; PD_ERR_UNSUPPORTED for a valid request
+ * beyond a limit of this build: T5-bias mode needs time_max + sub_max + 2 <= 512 (one bias value per distance is
+ * kept in shared memory); 8-bit context keys/values need the bf16 path, max_ctx a multiple of 16 and at most 32
+ * rows per sequence.  *reason (may be NULL) receives a static text.  Not a limit but a slower path: with more than
+ * 32 rows per sequence (pd_rows_per_seq) the bf16 attention steps run on the plain-ALU kernels instead of the
+ * tensor-core ones.  Pure function; no CUDA call. */
+PD_API pd_status pd_config_check(const pd_config *cfg, const char **reason);
+
+/* Bytes of device workspace pd_init needs for this configuration (0 if pd_config_check(cfg) fails).
  * Pure function; no CUDA call. */
 PD_API size_t pd_workspace_bytes(const pd_config *cfg);
 
 /* Creates a handle: validates cfg, carves the workspace (device, 256-byte aligned, at least
  * pd_workspace_bytes(cfg)), creates the cuBLAS handles and the TMA descriptor of the context
- * keys/values, builds the position tables.  `cuda_stream`
- * is a cudaStream_t (NULL = legacy default stream).  Algorithm 1's inputs delta_t, time_max,
+ * keys/values, builds the position tables.  Returns what pd_config_check returns for a configuration it
+ * does not take.  `cuda_stream` is a cudaStream_t (NULL = legacy default stream).  Algorithm 1's inputs delta_t, time_max,
  * sub_max are fixed here. */
 PD_API pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspace, size_t workspace_bytes,
                   void *cuda_stream, pd_handle **out);

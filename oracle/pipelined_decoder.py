@@ -8,9 +8,12 @@ blocking, no paging, no fusion.
 
 What follows the paper and what is a reading of it:
 
-* `decode`             - Algorithm 1 (Section 3.4), line by line: admission every delta_t
-                         steps while k < sub_max, one decoder call per step, append to the
-                         incomplete subsequences, stop when all k have ended, strip bos/eos.
+* `decode`             - the decoding procedure of Section 3.4 driven by Eq. 2's closed form: at
+                         step t the sequence holds k(t) = min(sub_max, ceil(t / delta_t))
+                         subsequences (subsequence i starts at s_i = (i-1) delta_t + 1), every
+                         subsequence that has not ended gets one token from one decoder call,
+                         a terminator ends it, and the procedure stops after the first step at
+                         which every subsequence it holds has ended (or at time_max).
 * `visible`            - the dependency rule of Section 3.2 (the set G^{<=t}_{<=i} under
                          Eq. 3): a query of subsequence i whose input token was generated
                          at step tau_q sees token (i', tau') iff i' <= i and tau' <= tau_q.
@@ -98,36 +101,40 @@ class Sub:
 
 def decode(step_fn: Callable[[List[Sub], int, List[int]], Dict[int, int]], delta_t: int, time_max: int,
            sub_max: int, bos: int, terminators: Sequence[int]):
-    """Algorithm 1.  `step_fn(G, t, active)` plays Decoder(G, H^E): it returns the new token
-    of every active (incomplete) subsequence.  Returns (G, steps_used, trace) where trace[t-1]
-    = (active list, {i: token}) and G keeps bos (callers strip with `strip`)."""
+    """The decoding procedure of Section 3.4.  `step_fn(G, t, active)` plays Decoder(G, H^E): it returns
+    the new token of every active (not yet ended) subsequence.  Returns (G, steps_used, trace) where
+    trace[t-1] = (active list, {i: token}) and G keeps bos (callers strip with `strip`).
+
+    The schedule comes from Eq. 2: while the procedure runs, the number of subsequences at step t is
+    k(t) = min(sub_max, ceil(t / delta_t)), so subsequence i appears exactly at s_i = (i-1) delta_t + 1;
+    k(t) grows by at most one per step, which is the paper's "a new subsequence every delta_t steps while
+    fewer than sub_max exist"."""
     G: List[Sub] = []
-    k = 0
     trace = []
-    steps = 0
-    for t in range(1, time_max + 1):
-        if (t - 1) % delta_t == 0:
-            if k < sub_max:
-                k += 1
-                G.append(Sub(k, t, bos))
+    t = 0
+    while t < time_max:
+        t += 1
+        k_t = min(sub_max, -(-t // delta_t))                 # Eq. 2, capped
+        if len(G) < k_t:
+            i = len(G) + 1
+            assert k_t == i and (i - 1) * delta_t + 1 == t   # one at a time, at its start step
+            G.append(Sub(i, t, bos))
         active = [s.index for s in G if not s.ended]
         new = step_fn(G, t, active)
-        for i in active:
-            s = G[i - 1]
-            tok = int(new[i])
+        for s in (G[i - 1] for i in active):
+            tok = int(new[s.index])
             if tok in terminators:
                 s.ended, s.terminator = True, tok
                 s.flag |= FLAG_COMPLETE
             else:
                 s.tokens.append(tok)
         trace.append((active, {i: int(new[i]) for i in active}))
-        steps = t
-        if sum(1 for s in G if s.ended) == k:
+        if all(s.ended for s in G):                          # every subsequence the sequence holds has ended
             break
     for s in G:
         if not s.ended:
             s.flag |= FLAG_TRUNCATED
-    return G, steps, trace
+    return G, t, trace
 
 
 def strip(G: List[Sub]) -> List[List[int]]:

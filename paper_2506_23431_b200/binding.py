@@ -47,6 +47,7 @@ class PdWeights(C.Structure):
 _H = C.c_void_p
 _i32p = C.POINTER(C.c_int32)
 _SIGS = {
+    "pd_config_check": (C.c_int, [C.POINTER(PdConfig), C.POINTER(C.c_char_p)]),
     "pd_workspace_bytes": (C.c_size_t, [C.POINTER(PdConfig)]),
     "pd_init": (C.c_int, [C.POINTER(PdConfig), C.POINTER(PdWeights), C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(_H)]),
     "pd_encode_context": (C.c_int, [_H, C.c_void_p, _i32p, C.c_int32, _i32p]),

@@ -31,6 +31,17 @@ struct Layout {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Limits of this build on otherwise valid configurations, with the text pd_config_check returns.
+const char *unsupported_reason(const pd_config &c) {
+  if (c.pos_mode == PD_POS_T5_BIAS && c.time_max + c.sub_max + 2 > 512)
+    return "T5-bias mode keeps one bias value per distance in shared memory: time_max + sub_max + 2 must not exceed 512";
+  if (c.kv_c_dtype == PD_KV_E4M3 && (c.dtype != PD_DTYPE_BF16 || (c.max_ctx % 16) != 0))
+    return "8-bit context keys/values need dtype = bf16 and max_ctx a multiple of 16";
+  if (c.kv_c_dtype == PD_KV_E4M3 && c.delta_t >= 1 && (c.max_sub_len / c.delta_t + 1 < c.sub_max ? c.max_sub_len / c.delta_t + 1 : c.sub_max) > 32)
+    return "8-bit context keys/values are read by the tensor-core kernel only: at most 32 rows per sequence";
+  return nullptr;
+}
+
 bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   if (c.n_layers < 1 || c.d_model < 64 || c.d_model > 4096 || c.n_heads < 1 || c.d_head != kDh || c.n_heads * c.d_head != c.d_model) return false;
   if (c.d_ff < 8 || c.vocab < 4 || (c.d_model % 8) || (c.d_ff % 8)) return false;
@@ -44,7 +55,7 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   if (c.self_splits < 0 || c.self_splits > 32 || c.cross_splits < 0 || c.cross_splits > 32) return false;
   if (c.store_logits != 0 && c.store_logits != 1) return false;
   if (c.kv_c_dtype != PD_KV_SAME && c.kv_c_dtype != PD_KV_E4M3) return false;
-  if (c.kv_c_dtype == PD_KV_E4M3 && (c.dtype != PD_DTYPE_BF16 || (c.max_ctx % 16) != 0)) return false;
+  if (unsupported_reason(c) != nullptr) return false;
   if (!(c.attn_scale > 0.f) || !(c.norm_eps >= 0.f)) return false;
   dm.L = c.n_layers; dm.d = c.d_model; dm.H = c.n_heads; dm.ff = c.d_ff; dm.V = c.vocab;
   dm.B = c.max_batch; dm.ctx = c.max_ctx; dm.SM = c.sub_max; dm.dt = c.delta_t; dm.T = c.time_max;
@@ -61,8 +72,7 @@ bool make_dims(const pd_config &c, Dims &dm, int &max_splits) {
   dm.bos = c.bos_id; dm.eos = c.eos_id; dm.sep = c.sep_id;
   dm.pos_mode = c.pos_mode;
   dm.n_dist = c.time_max + c.sub_max + 2;
-  if (c.pos_mode == PD_POS_T5_BIAS && dm.n_dist > 512) return false;
-  if (c.kv_c_dtype == PD_KV_E4M3 && dm.C > 32) return false;          // the 8-bit keys/values are read by the tensor-core kernel only
+
   dm.scale_log2e = c.attn_scale * 1.4426950408889634f;
   dm.eps = c.norm_eps;
   max_splits = 32;
@@ -472,6 +482,17 @@ int encode_chunks(const pd_handle *h, int batch) {
 
 extern "C" {
 
+pd_status pd_config_check(const pd_config *cfg, const char **reason) {
+  if (reason) *reason = "";
+  if (!cfg) { if (reason) *reason = "null configuration"; return PD_ERR_ARG; }
+  Dims dm; int ms;
+  if (make_dims(*cfg, dm, ms)) return PD_OK;
+  const char *why = unsupported_reason(*cfg);
+  if (why) { if (reason) *reason = why; return PD_ERR_UNSUPPORTED; }
+  if (reason) *reason = "a field is out of range (see pd_config in pd.h)";
+  return PD_ERR_ARG;
+}
+
 size_t pd_workspace_bytes(const pd_config *cfg) {
   if (!cfg) return 0;
   Dims dm; int ms; Layout L;
@@ -485,7 +506,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   if (!cfg || !weights || !workspace || !out) return PD_ERR_ARG;
   *out = nullptr;
   Dims dm; int ms;
-  if (!make_dims(*cfg, dm, ms)) return PD_ERR_ARG;
+  if (!make_dims(*cfg, dm, ms)) return pd_config_check(cfg, nullptr);
   if (!weights->embed || !weights->layer || !weights->final_norm || !weights->lm_head) return PD_ERR_ARG;
   if (cfg->pos_mode == PD_POS_T5_BIAS && !weights->rel_bias) return PD_ERR_ARG;
   for (int i = 0; i < cfg->n_layers * kLayerTensors; ++i) if (!weights->layer[i]) return PD_ERR_ARG;

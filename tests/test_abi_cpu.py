@@ -71,6 +71,19 @@ def test_invalid_configurations_are_rejected_on_the_host():
     assert ws(pos_mode=3) == 0
     assert ws(kv_c_dtype=1) == 0                       # 8-bit context keys/values need the bf16 path
     assert B._lib.pd_workspace_bytes(None) == 0
+    # limits of the build are told apart from bad fields, with a text
+    def check(**kw):
+        cfg = B.make_config(wl.hyper(), 1)
+        for k, v in kw.items():
+            setattr(cfg, k, v)
+        why = C.c_char_p()
+        return B._lib.pd_config_check(C.byref(cfg), C.byref(why)), (why.value or b"").decode()
+    assert check() == (0, "")
+    st, why = check(time_max=600)
+    assert st == -7 and "512" in why and ws(time_max=600) == 0
+    st, why = check(kv_c_dtype=1)
+    assert st == -7 and "bf16" in why
+    assert check(sub_max=65)[0] == -1
     # pd_init refuses null pointers and bad configs before touching CUDA
     h = C.c_void_p()
     cfg = B.make_config(wl.hyper(), 1)
