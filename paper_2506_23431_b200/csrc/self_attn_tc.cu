@@ -44,7 +44,9 @@ constexpr int SKEYS = 16;                  // keys per batch: one 16-token page 
 constexpr int SMAXLIST = 256;              // page-list entries of one sequence held in shared memory
 constexpr int SMAXDIST = 512;
 constexpr int SMROW = kDh + 8;             // row stride of the merge scratch in floats (spreads the eight fragment rows over the banks)
-constexpr int SBATCHES_PER_WARP = 3;       // batches a warp should get before another split is used
+// Pages a warp walks before another split is used: a page costs a warp ~0.75 us, a split ~4 us of fixed cost
+// (partial records, fence, ticket, the last CTA's read-back), so a split pays once it saves about six pages per warp.
+constexpr int SBATCHES_PER_WARP = 10;
 constexpr int SBIAS_PER_THREAD = (SMAXDIST + STHREADS - 1) / STHREADS;
 
 __device__ __forceinline__ uint32_t s_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
