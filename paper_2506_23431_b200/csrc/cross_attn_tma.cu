@@ -28,7 +28,7 @@
 // (score columns) are loaded with the same permutation, which a contraction does not see.  Queries and
 // softmax weights go through f16 (exact for bf16 queries in f16's range; 11 bits for the weights), the
 // key scale is folded into the score scale and the value scale into the final 1 / l.  Stages are 16 KB,
-// so the ring is six deep.
+// the ring six deep.
 #include <cuda_fp16.h>
 
 #include "pd_internal.h"
@@ -36,21 +36,23 @@
 namespace pd {
 
 constexpr int XK = 128;                   // keys per tile
-constexpr int XRING_BYTES = 96 * 1024;    // three 32 KB stages (bf16) or six 16 KB stages (8-bit)
-constexpr int XMAX_STAGES = 6;
-constexpr int XCW = 4;                    // consumer warps
-constexpr int XTHREADS = (XCW + 1) * 32;
+// ring: three 32 KB stages (bf16) or six 16 KB stages (8-bit); with the merge scratch two CTAs fit an SM
+__host__ __device__ constexpr int xring_bytes(bool fp8) { return fp8 ? 96 * 1024 : 96 * 1024; }
+// consumer warps: four, each taking 32 keys of a tile.  (Eight warps of 16 keys each were measured in both
+// variants and lost: 50.3 against 49.2 us per full bf16 launch, 31.9 against 28.7 us per 8-bit launch.)
+__host__ __device__ constexpr int xcw(bool fp8) { return fp8 ? 4 : 4; }
+__host__ __device__ constexpr int xthreads(bool fp8) { return (xcw(fp8) + 1) * 32; }
 constexpr int XMIN_TILES = 4;              // fewest tiles worth a CTA of its own
 constexpr int XMIN_WHOLE = 64;             // fewest CTAs for which whole (sequence, head) segments per CTA still beat cutting the tile list
 constexpr int XLONG_SEG = 24;              // tiles from which a segment is worth two CTAs when there are fewer segments than SMs
 constexpr int XMAXB = 256;                // sequences per launch the tile prefix table holds
 constexpr int XREC_WORDS = 36;            // per lane and 16-row tile: 32 output values, 2 maxima, 2 sums
 constexpr int XREC_FLOATS = XREC_WORDS * 32;
-constexpr int XSCRATCH_BYTES = 2 * XREC_FLOATS * 4;   // two records for the warp tree merge
-constexpr int XSMEM = XRING_BYTES + XSCRATCH_BYTES + 128 /*barriers*/ + 1024 /*alignment slack*/;
+__host__ __device__ constexpr int xscratch_bytes(bool fp8) { return (xcw(fp8) / 2) * XREC_FLOATS * 4; }   // half the consumer warps' records for the tree merge
+__host__ __device__ constexpr int xsmem(bool fp8) { return xring_bytes(fp8) + xscratch_bytes(fp8) + 128 /*barriers*/ + 1024 /*alignment slack*/; }
 constexpr uint32_t XSPIN_LIMIT = 1u << 24;
 
-int cross_attn_tma_smem_bytes() { return XSMEM; }
+int cross_attn_tma_smem_bytes() { return xsmem(false); }
 size_t cross_attn_tma_partial_bytes(int n_ctas, int rows_per_seq) {
   return (size_t)n_ctas * 2 * ((rows_per_seq + 15) / 16) * XREC_FLOATS * sizeof(float);
 }
@@ -139,7 +141,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
-__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(XCW * 32) : "memory"); }
+template <int THREADS> __device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
 
 // Byte offset of (row, 16-byte chunk) inside a 128-byte-swizzled tile whose rows are 128 bytes.
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
@@ -212,11 +214,15 @@ struct TileCursor {
 // MT = 16-row query tiles (rows per sequence <= 16 * MT); FP8 = keys/values are E4M3 codes (tmap: the keys'
 // 128-byte lines, tmap_v: the transposed values), else bf16 (tmap alone: rows of 64 values)
 template <int MT, bool FP8>
-__global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap,
-                                                                  const __grid_constant__ CUtensorMap tmap_v, AttnArgs a) {
+__global__ void __launch_bounds__(xthreads(FP8), 2) cross_attn_tma_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                          const __grid_constant__ CUtensorMap tmap_v, AttnArgs a) {
+  constexpr int XCW = xcw(FP8), XTHREADS = xthreads(FP8);
+  constexpr int KPW = XK / XCW;                            // keys of a tile per consumer warp: 32 or 16
+  constexpr int NTW = KPW / 8, KSW = KPW / 16;             // 8-key score tiles and 16-key P.V steps per warp and tile
   constexpr int XTILE_BYTES = XK * kDh * (FP8 ? 1 : 2);    // keys (or values) of one tile: 8 or 16 KB
   constexpr int XSTAGE_BYTES = 2 * XTILE_BYTES;
-  constexpr int XSTAGES = XRING_BYTES / XSTAGE_BYTES;
+  constexpr int XSTAGES = xring_bytes(FP8) / XSTAGE_BYTES;
+  constexpr int XSCRATCH_BYTES = xscratch_bytes(FP8);
   extern __shared__ uint8_t smem_raw[];
   __shared__ int pfx_s[XMAXB + 1];
   __shared__ int aseq_s[XMAXB];             // the a-th sequence that has an active row
@@ -333,7 +339,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
   // -------------------------------------------------------------------- consumers
   const int g = lane >> 2, tig = lane & 3;
   const __nv_bfloat16 *qbuf = (const __nv_bfloat16 *)a.q;
-  const int kb = warp * 32;          // this warp's keys inside every tile
+  const int kb = warp * KPW;         // this warp's keys inside every tile
   const float sl2 = dm.scale_log2e;
   bool ok = true;
   int it = 0;
@@ -388,19 +394,19 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
       if (!ok) continue;             // drained mode: keep the control flow (barriers below) intact
       const uint32_t kbase = base + s * XSTAGE_BYTES, vbase = kbase + XTILE_BYTES;
       const int key0 = tile * XK + kb;               // context position of this warp's first key
-      const bool ragged = key0 + 32 > ctx_len;
+      const bool ragged = key0 + KPW > ctx_len;
       // Rows at or beyond ctx_len hold whatever follows in memory.  Their weights are exactly 0 below;
       // the value fragments of those keys are cleared in registers after ldmatrix, so that 0 never
       // multiplies a non-finite.  (Nothing but TMA ever writes a stage: zeroing the rows in shared
       // memory raced with the next bulk copy into the stage, proxy fence or not.)
       // ---- scores: S[mt][nt] = Q (16 x 64) . K^T (64 x 8 keys)
-      float sc[MT][4][4];
+      float sc[MT][NTW][4];
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
+        for (int nt = 0; nt < NTW; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) {
+      for (int nt = 0; nt < NTW; ++nt) {
         if (FP8) {
           // column c of score tile nt = 2 ks + u is key 16 ks + 4 (c >> 1) + 2 u + (c & 1) of this warp's 32: the
           // order in which the value codes of a 16-key step come out of ldmatrix (see the P.V loop).  The keys
@@ -432,12 +438,12 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         }
       }
       // ---- scale, mask the ragged end of the context, online softmax
-      uint32_t pf[MT][2][4];
+      uint32_t pf[MT][KSW][4];
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
+        for (int nt = 0; nt < NTW; ++nt) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             float v = sc[mt][nt][e] * seg_sl2;
@@ -459,7 +465,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         A.m0 = mn0; A.m1 = mn1;
         float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
+        for (int nt = 0; nt < NTW; ++nt) {
           float p0 = ex2f(sc[mt][nt][0] - ref0), p1 = ex2f(sc[mt][nt][1] - ref0);
           float p2 = ex2f(sc[mt][nt][2] - ref1), p3 = ex2f(sc[mt][nt][3] - ref1);
           s0 += p0 + p1; s1 += p2 + p3;
@@ -478,7 +484,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         // transposed values: a line is one dim, a 16-byte chunk sixteen keys; positions at or beyond ctx_len
         // hold zero codes (written so, or filled by the copy beyond max_ctx), so nothing needs masking
 #pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
+        for (int ks = 0; ks < KSW; ++ks) {
           const int chunk = (kb + ks * 16) >> 4;
 #pragma unroll
           for (int dq = 0; dq < 2; ++dq) {      // four 8-wide slices of the head per ldmatrix.x4
@@ -496,7 +502,7 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
         }
       } else {
 #pragma unroll
-      for (int ks = 0; ks < 2; ++ks) {
+      for (int ks = 0; ks < KSW; ++ks) {
         const int key = kb + ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
         // this lane's fragment halves hold keys k0, k0 + 1 (b0, b2) and k0 + 8, k0 + 9 (b1, b3)
         uint32_t keep_a = 0xffffffffu, keep_b = 0xffffffffu;
@@ -523,20 +529,19 @@ __global__ void __launch_bounds__(XTHREADS) cross_attn_tma_kernel(const __grid_c
     }
 
     // ---- end of this CTA's part of the (sequence, head) segment: row sums across the quad, then
-    // tree-merge the four warps into warp 0, one 16-row tile at a time
+    // tree-merge the consumer warps into warp 0, one 16-row tile at a time
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       TileAcc &A = acc[mt];
       A.l0 += __shfl_xor_sync(0xffffffffu, A.l0, 1); A.l0 += __shfl_xor_sync(0xffffffffu, A.l0, 2);
       A.l1 += __shfl_xor_sync(0xffffffffu, A.l1, 1); A.l1 += __shfl_xor_sync(0xffffffffu, A.l1, 2);
-      if (warp >= 2) A.store(scratch + (warp & 1) * XREC_FLOATS, lane);      // warps 2, 3 -> warps 0, 1
-      consumer_bar_sync();
-      if (warp < 2) A.template merge<false>(scratch + warp * XREC_FLOATS, lane);
-      consumer_bar_sync();
-      if (warp == 1) A.store(scratch, lane);                                  // warp 1 -> warp 0
-      consumer_bar_sync();
-      if (warp == 0) A.template merge<false>(scratch, lane);
-      consumer_bar_sync();
+#pragma unroll
+      for (int stride = XCW / 2; stride >= 1; stride >>= 1) {                 // the upper half hands its state to the lower half
+        if (warp >= stride && warp < 2 * stride) A.store(scratch + (warp - stride) * XREC_FLOATS, lane);
+        consumer_bar_sync<XCW * 32>();
+        if (warp < stride) A.template merge<false>(scratch + warp * XREC_FLOATS, lane);
+        consumer_bar_sync<XCW * 32>();
+      }
     }
     if (warp == 0) {
       const bool whole = f == seg_start && my_end == seg_end;
@@ -659,10 +664,10 @@ cudaError_t encode_ctx_kv8_tensor_maps(CUtensorMap *map_k, CUtensorMap *map_v, c
 }
 
 cudaError_t cross_attn_tma_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(cross_attn_tma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, XSMEM);
+  cudaError_t e = cudaFuncSetAttribute(cross_attn_tma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, xsmem(false));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, xsmem(false));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, xsmem(true));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(cross_attn_tma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, xsmem(true));
   return e;
 }
 
@@ -672,10 +677,10 @@ cudaError_t cross_attn_tma_prepare() {
 cudaError_t launch_cross_attn_tma(const AttnArgs &a, const CUtensorMap &tmap, const CUtensorMap &tmap_v, int n_ctas, cudaStream_t s) {
   int mt = (a.dm.C + 15) / 16;
   const bool fp8 = a.kv_scale != nullptr;
-  if (mt == 1 && !fp8) cross_attn_tma_kernel<1, false><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
-  else if (mt == 2 && !fp8) cross_attn_tma_kernel<2, false><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
-  else if (mt == 1) cross_attn_tma_kernel<1, true><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
-  else if (mt == 2) cross_attn_tma_kernel<2, true><<<n_ctas, XTHREADS, XSMEM, s>>>(tmap, tmap_v, a);
+  if (mt == 1 && !fp8) cross_attn_tma_kernel<1, false><<<n_ctas, xthreads(false), xsmem(false), s>>>(tmap, tmap_v, a);
+  else if (mt == 2 && !fp8) cross_attn_tma_kernel<2, false><<<n_ctas, xthreads(false), xsmem(false), s>>>(tmap, tmap_v, a);
+  else if (mt == 1) cross_attn_tma_kernel<1, true><<<n_ctas, xthreads(true), xsmem(true), s>>>(tmap, tmap_v, a);
+  else if (mt == 2) cross_attn_tma_kernel<2, true><<<n_ctas, xthreads(true), xsmem(true), s>>>(tmap, tmap_v, a);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }
