@@ -209,6 +209,9 @@ __global__ void __launch_bounds__(RN_THREADS) rmsnorm_packed_kernel(int d, float
                                                                     T *__restrict__ out) {
   __shared__ float red[RN_THREADS / 32];
   __shared__ int redi[RN_THREADS / 32];
+  // the vocabulary projection that follows may start its set-up and its first lm_head copies now (it waits for
+  // this kernel's rows where it needs them)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int b = blockIdx.x / C, c = blockIdx.x % C;
   int before = 0;
   for (int bb = threadIdx.x; bb < b; bb += RN_THREADS) before += st.n_active[bb];

@@ -170,7 +170,7 @@ struct pd_handle {
   CUtensorMap tmap_kvc, tmap_kvc_v;   // context keys/values (8-bit storage: the keys' lines and the transposed values)
   bool have_tmap = false;
   bool kv8 = false;
-  CUtensorMap vmap_a, vmap_b;      // hidden rows and lm_head for the tcgen05 vocabulary projection
+  VocabMaps vmaps;                 // hidden rows and lm_head for the tcgen05 vocabulary projection
   bool vocab_tc = false;
   // pd_generate_host: host-to-device copies of the encoder memory run on a stream of their own, in
   // chunks of sequences, so that the context projection of one chunk overlaps the copy of the next
@@ -421,7 +421,7 @@ pd_status enqueue_step(pd_handle *h) {
     va.logits = h->cfg.store_logits ? logits : nullptr;
     va.status = h->st.hdr + HDR_STATUS;
     OWN(h, PD_PROF_OTHER, launch_rmsnorm_packed(dm, h->st, h->batch, dt, x, h->w.final_norm, hb, s));
-    OWN(h, PD_PROF_VOCAB, launch_vocab_tc(h->vmap_a, h->vmap_b, va, s));
+    OWN(h, PD_PROF_VOCAB, launch_vocab_tc(h->vmaps, va, s));
     OWN(h, PD_PROF_ARGMAX_SCHED, launch_pick_sched(dm, h->st, h->batch, vocab_tc_tiles(dm.V), va.part_val, va.part_idx, va.term_val,
                                                    h->ptr<int32_t>(h->lay.teacher), s));
     return PD_OK;
@@ -577,7 +577,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   if (cfg->dtype == PD_DTYPE_BF16 && self_attn_tc_supported(dm) && self_attn_tc_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);
   if (cfg->dtype == PD_DTYPE_BF16 && vocab_tc_supported(dm.d, dm.V) && reinterpret_cast<uintptr_t>(weights->lm_head) % 16 == 0) {
     int code = 0;
-    if (encode_vocab_maps(&h->vmap_a, &h->vmap_b, h->ptr<void>(L.hbuf), (uint64_t)dm.B * dm.C, weights->lm_head, (uint64_t)dm.V,
+    if (encode_vocab_maps(&h->vmaps, h->ptr<void>(L.hbuf), (uint64_t)dm.B * dm.C, weights->lm_head, (uint64_t)dm.V,
                           (uint64_t)dm.d, &code) != cudaSuccess)
       return bail(PD_ERR_CUDA);
     if (vocab_tc_prepare() != cudaSuccess) return bail(PD_ERR_CUDA);

@@ -156,6 +156,7 @@ struct VocabArgs {
   int m_fixed;               // number of rows when n_active is null
   int V, K;                  // vocabulary size, model width (a multiple of 64)
   int rows_cap;              // row stride of the partial arrays (>= the largest row count)
+  int wn;                    // vocabulary ids per CTA (set by the launcher: vocab_tc_slice(V))
   int eos, sep;              // ids kept out of the maxima (their logits go to term_val); -1 = none
   float *part_val;           // [tiles][rows_cap] maximum of the row over the tile's ids
   int32_t *part_idx;         // [tiles][rows_cap] the id that holds it (lowest on ties; INT_MAX = none)
@@ -163,12 +164,14 @@ struct VocabArgs {
   float *logits;             // [rows][V] fp32, or null when nobody reads them
   int32_t *status;           // error word (PD_ERR_TIMEOUT on an expired wait)
 };
+struct VocabMaps { CUtensorMap a, a32, b; };   // hidden rows (128-row and 32-row boxes), lm_head (one slice per box)
+int vocab_tc_slice(int V);
 int vocab_tc_tiles(int V);
 bool vocab_tc_supported(int K, int V);
 cudaError_t vocab_tc_prepare();          // once per device, outside any stream capture
-cudaError_t encode_vocab_maps(CUtensorMap *map_a, CUtensorMap *map_b, const void *hidden, uint64_t rows, const void *lm_head,
-                              uint64_t vocab, uint64_t K, int *driver_code);
-cudaError_t launch_vocab_tc(const CUtensorMap &map_a, const CUtensorMap &map_b, const VocabArgs &a, cudaStream_t s);
+cudaError_t encode_vocab_maps(VocabMaps *m, const void *hidden, uint64_t rows, const void *lm_head, uint64_t vocab, uint64_t K,
+                              int *driver_code);
+cudaError_t launch_vocab_tc(const VocabMaps &m, const VocabArgs &a, cudaStream_t s);
 
 // ---- skinny-M linear layers on tcgen05 (linear_tc.cu) --------------------------------------------
 enum { LIN_EPI_STORE = 0,   // out = bf16(acc * row_scale)

@@ -71,8 +71,8 @@ pd_status pd_vocab_argmax(int32_t rows, int32_t d_model, int32_t vocab, const vo
   uint8_t *base = reinterpret_cast<uint8_t *>(scratch);
   if (cudaMemsetAsync(base, 0, kOpHeaderBytes, s) != cudaSuccess) return PD_ERR_CUDA;    // status word
 
-  CUtensorMap map_a, map_b;
-  if (encode_vocab_maps(&map_a, &map_b, hidden, (uint64_t)rows, lm_head, (uint64_t)vocab, (uint64_t)d_model, nullptr) != cudaSuccess)
+  VocabMaps maps;
+  if (encode_vocab_maps(&maps, hidden, (uint64_t)rows, lm_head, (uint64_t)vocab, (uint64_t)d_model, nullptr) != cudaSuccess)
     return PD_ERR_CUDA;
   if (vocab_tc_prepare() != cudaSuccess) return PD_ERR_CUDA;
   VocabArgs a;
@@ -83,7 +83,7 @@ pd_status pd_vocab_argmax(int32_t rows, int32_t d_model, int32_t vocab, const vo
   a.term_val = reinterpret_cast<float *>(base + L.off_term);
   a.logits = logits;
   a.status = reinterpret_cast<int32_t *>(base) + HDR_STATUS;
-  if (launch_vocab_tc(map_a, map_b, a, s) != cudaSuccess) return PD_ERR_CUDA;
+  if (launch_vocab_tc(maps, a, s) != cudaSuccess) return PD_ERR_CUDA;
   const int warps = 8;
   vocab_reduce_kernel<<<(rows + warps - 1) / warps, warps * 32, 0, s>>>(rows, vocab_tc_tiles(vocab), rows, a.part_val, a.part_idx,
                                                                          best_id, best_val);
