@@ -122,28 +122,39 @@ cudaError_t launch_build_bias_table(const Dims &dm, const float *rel_bias, int r
 // ---------------------------------------------------------------------------------------------
 // Embedding gather: row (b, c) takes the embedding of the last token of its subsequence (the
 // decoder input of Eq. 3); unused rows are zero so that they stay zero through the layer stack.
+// The first layer's RMSNorm of the row rides along (the CTA holds the whole row): h = norm(x) * gain.
 template <typename T>
-__global__ void embed_kernel(Dims dm, DecState st, const T *__restrict__ embed, float *__restrict__ x) {
+__global__ void __launch_bounds__(128) embed_kernel(Dims dm, DecState st, const T *__restrict__ embed, float *__restrict__ x,
+                                                    const T *__restrict__ gain, T *__restrict__ h) {
+  __shared__ float red[4];
   int r = blockIdx.x;
   int b = r / dm.C;
   int i = st.row_sub[r];
   float *xr = x + (size_t)r * dm.d;
+  T *hr = h + (size_t)r * dm.d;
   if (i <= 0) {
-    for (int c = threadIdx.x; c < dm.d; c += blockDim.x) xr[c] = 0.f;
+    for (int c = threadIdx.x; c < dm.d; c += blockDim.x) { xr[c] = 0.f; hr[c] = from_f<T>(0.f); }
     return;
   }
   int tok = st.last_tok[b * dm.SM + i - 1];
   const T *e = embed + (size_t)tok * dm.d;
-  for (int c = threadIdx.x; c < dm.d; c += blockDim.x) xr[c] = to_f<T>(e[c]);
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < dm.d; c += blockDim.x) { const float v = to_f<T>(e[c]); xr[c] = v; ss += v * v; }
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  const float inv = rsqrtf((red[0] + red[1] + red[2] + red[3]) / (float)dm.d + dm.eps);
+  for (int c = threadIdx.x; c < dm.d; c += blockDim.x) hr[c] = from_f<T>(to_f<T>(e[c]) * inv * to_f<T>(gain[c]));
 }
 
-cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x,
-                         cudaStream_t s) {
+// gain, h: the first layer's norm gain and the buffer its normalised rows go to (the input of that layer's Q/K/V projection)
+cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x, const void *gain,
+                         void *h, cudaStream_t s) {
   int rows = batch * dm.C;
   if (dtype == PD_DTYPE_BF16)
-    embed_kernel<__nv_bfloat16><<<rows, 128, 0, s>>>(dm, st, (const __nv_bfloat16 *)embed, x);
+    embed_kernel<__nv_bfloat16><<<rows, 128, 0, s>>>(dm, st, (const __nv_bfloat16 *)embed, x, (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)h);
   else
-    embed_kernel<float><<<rows, 128, 0, s>>>(dm, st, (const float *)embed, x);
+    embed_kernel<float><<<rows, 128, 0, s>>>(dm, st, (const float *)embed, x, (const float *)gain, (float *)h);
   return cudaGetLastError();
 }
 

@@ -2,8 +2,7 @@
 // 5th-generation tensor cores (bf16, sm_100a):  acc[m][n] = sum_k A[m][k] * W[n][k]  for the few
 // hundred packed active rows m of a decode step against a weight matrix that is streamed from HBM
 // exactly once, with the work that surrounds the product in the layer fused into the epilogue
-// (row scale of the preceding RMSNorm, ReLU, residual add + the next norm's inputs, KV-append with
-// the positional write).
+// (row scale of the preceding RMSNorm, ReLU, residual add + the next norm's inputs).
 //
 // The products are tiny (a few MB of weights, a few hundred rows), so the kernel is built around
 // latency, not flops:
@@ -140,7 +139,7 @@ __device__ __forceinline__ uint2 l_pack4(float a, float b, float c, float d) {
 // ---- the epilogue of one (row, four columns) group --------------------------------------------------
 // v = the four sums of columns n .. n + 3 of packed row m.  `ss` accumulates the squares of what the
 // residual epilogue writes (the next RMSNorm's input).
-__device__ __forceinline__ void l_epilogue4(const LinearArgs &a, int m, int n, float4 v, float inv, const int4 &meta, float &ss) {
+__device__ __forceinline__ void l_epilogue4(const LinearArgs &a, int m, int n, float4 v, float inv, float &ss) {
   switch (a.epi) {
     case LIN_EPI_STORE:
     case LIN_EPI_RELU: {
@@ -156,27 +155,6 @@ __device__ __forceinline__ void l_epilogue4(const LinearArgs &a, int m, int n, f
       const __nv_bfloat162 g0 = *reinterpret_cast<const __nv_bfloat162 *>(&gbits.x), g1 = *reinterpret_cast<const __nv_bfloat162 *>(&gbits.y);
       *reinterpret_cast<uint2 *>(a.xg + (size_t)m * a.N + n) =
           l_pack4(v.x * __low2float(g0), v.y * __high2float(g0), v.z * __low2float(g1), v.w * __high2float(g1));
-      break;
-    }
-    case LIN_EPI_QKV: {
-      // columns q | k | v (each d wide, head-major); meta = (page, slot, position tau + i, subsequence) of the row
-      v.x *= inv; v.y *= inv; v.z *= inv; v.w *= inv;
-      const int sect = n / a.d, col = n - sect * a.d;
-      const int head = col / kDh, dd = col % kDh;
-      if (a.rope && sect < 2) {
-        const float2 c0 = a.rope_tab[(size_t)meta.z * (kDh / 2) + dd / 2], c1 = a.rope_tab[(size_t)meta.z * (kDh / 2) + dd / 2 + 1];
-        float t;
-        t = v.x * c0.x - v.y * c0.y; v.y = v.x * c0.y + v.y * c0.x; v.x = t;
-        t = v.z * c1.x - v.w * c1.y; v.w = v.z * c1.y + v.w * c1.x; v.z = t;
-      }
-      const uint2 bits = l_pack4(v.x, v.y, v.z, v.w);
-      if (sect == 0) {
-        *reinterpret_cast<uint2 *>(a.q_out + (size_t)m * a.d + col) = bits;
-      } else {
-        __nv_bfloat16 *dst = a.kv_pool + kv_block_offset(a.layer, a.pool, meta.x, a.H, head, a.P) +
-                             kv_entry_offset<__nv_bfloat16>(meta.y, dd, sect - 1);
-        *reinterpret_cast<uint2 *>(dst) = bits;
-      }
       break;
     }
   }
@@ -385,8 +363,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           float sc = 1.f;
 #pragma unroll
           for (int jj = 0; jj < LT_MT_MAX; ++jj) if (jj == j) sc = inv[jj];
-          int4 meta = make_int4(0, 0, 0, 0);
-          if (a.epi == LIN_EPI_QKV) meta = a.prow_meta[m];
           float ss = 0.f;
           const float4 *buf = reinterpret_cast<const float4 *>(red + (size_t)(j - j0) * tile_bytes) + row;
           for (int g = 0; g < ng; ++g) {
@@ -409,7 +385,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
               }
               v.x += x0.x; v.y += x0.y; v.z += x0.z; v.w += x0.w;
             }
-            l_epilogue4(a, m, n, v, sc, meta, ss);
+            l_epilogue4(a, m, n, v, sc, ss);
           }
           if (a.epi == LIN_EPI_RESID && a.ssq_out != nullptr) a.ssq_out[(size_t)(n_tile * ks + (int)rank) * a.rows_cap + m] = ss;
         }

@@ -367,10 +367,10 @@ pd_status enqueue_step(pd_handle *h) {
   void *ffn = h->ptr<void>(h->lay.ffn);
   float *logits = h->ptr<float>(h->lay.logits);
 
-  OWN(h, PD_PROF_OTHER, launch_embed(dm, h->st, h->batch, dt, h->w.embed, x, s));
+  OWN(h, PD_PROF_OTHER, launch_embed(dm, h->st, h->batch, dt, h->w.embed, x, h->layer_w[0], hb, s));   // with the first layer's norm
   for (int l = 0; l < dm.L; ++l) {
     const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
-    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
+    if (l > 0) OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
     if (fused_append(h)) {
       // the attention kernel takes queries, keys and values straight from the projection's bf16 output and
       // appends the new cache entries itself

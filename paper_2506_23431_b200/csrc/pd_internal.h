@@ -110,8 +110,8 @@ struct AttnArgs {
 cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, const int32_t *ctx_len_dev,
                                const int32_t *forced_len_dev, size_t state_words, int32_t *state_base, cudaStream_t s);
 cudaError_t launch_admit_row(const Dims &dm, const DecState &st, int row, int ctx_len, const int32_t *forced_len_dev, cudaStream_t s);
-cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x,
-                         cudaStream_t s);
+cudaError_t launch_embed(const Dims &dm, const DecState &st, int batch, int dtype, const void *embed, float *x, const void *gain,
+                         void *h, cudaStream_t s);
 cudaError_t launch_rmsnorm(const Dims &dm, int rows, int dtype, const float *x, const void *gain, void *out,
                            cudaStream_t s);
 cudaError_t launch_rmsnorm_packed(const Dims &dm, const DecState &st, int batch, int dtype, const float *x, const void *gain,
@@ -176,8 +176,7 @@ cudaError_t launch_vocab_tc(const VocabMaps &m, const VocabArgs &a, cudaStream_t
 // ---- skinny-M linear layers on tcgen05 (linear_tc.cu) --------------------------------------------
 enum { LIN_EPI_STORE = 0,   // out = bf16(acc * row_scale)
        LIN_EPI_RELU = 1,    // out = bf16(max(acc * row_scale, 0))
-       LIN_EPI_RESID = 2,   // x += acc (fp32 residual stream); xg = bf16(x * gain_next); partial sums of x^2 per row
-       LIN_EPI_QKV = 3 };   // q | k | v columns: scale, rotary positions (optional), q to its buffer, k and v to the row's cache slot
+       LIN_EPI_RESID = 2 }; // x += acc (fp32 residual stream); xg = bf16(x * gain_next); partial sums of x^2 per row
 struct LinearArgs {
   int K, N;                  // the weight is [N][K] (K contiguous)
   int BN, ksplit;            // columns per CTA; CTAs (one cluster) along K
@@ -193,11 +192,6 @@ struct LinearArgs {
   __nv_bfloat16 *xg;         // RESID: bf16 [rows][N] = x * gain_next (input of the next layer's GEMM)
   const __nv_bfloat16 *gain_next;  // RESID: [N]
   float *ssq_out;            // RESID: [(N / BN) * ksplit][rows_cap] partial sums of squares of the new x, or null
-  // QKV
-  __nv_bfloat16 *q_out, *kv_pool;
-  const int4 *prow_meta;     // per packed row: (page, slot, position tau + i, subsequence)
-  const float2 *rope_tab;
-  int layer, pool, H, P, d, rope;
   int32_t *status;           // error word (PD_ERR_TIMEOUT on an expired wait)
 };
 int linear_tc_smem_bytes();
