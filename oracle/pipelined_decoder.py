@@ -32,6 +32,10 @@ What follows the paper and what is a reading of it:
   they are pinned only against a separately written textbook causal decoder (sub_max = 1).
 * The terminator of an ended subsequence is output only; it is never fed back and never
   becomes a key (a reading).  eos and sep both end a subsequence.
+* `PipelinedDecoderOracle.teacher_forward`  - Section 3.3, Eq. 6: one pass over the whole target
+                         (every subsequence as [bos, Y_i], inputs given) under the dense dependency
+                         mask; returns the logits of every position and the loss
+                         L = - sum_(i,t) log P(target_i^(t+1) | targets seen under the rule; H^E).
 * `e4m3_round`, `quantize_context_kv` - an option of this build, not of the paper (hp["kv_c_dtype"] =
   "e4m3"): the cross-attention keys/values of Eq. 1's encoder memory are stored as 8-bit floats
   (OCP FP8 E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest
@@ -361,6 +365,36 @@ class PipelinedDecoderOracle:
             x, _, _ = self._layer(l, x, meta, None, None, mask, bias, ctx)
         last = [meta.index((i, timestamp(i, G[i - 1].n_content, dt))) for i in active]
         return self._logits(x[last])
+
+    # ---- Eq. 6: the whole target in one teacher-forced pass under the dense mask
+    def teacher_forward(self, enc_mem: np.ndarray, ctx_len: int, subsequences: Sequence[Sequence[int]],
+                        terminators: Optional[Sequence[int]] = None):
+        """subsequences[i-1] = the content tokens of subsequence i.  Row (i, p), p = 0..m_i, has input bos
+        (p = 0) or content token p, timestamp (i-1) delta_t + p, and target content token p + 1 or, at
+        p = m_i, the subsequence's terminator (sep unless given).  Returns a dict: rows [(i, p)], targets,
+        logits [R, vocab], logprob [R] (log-softmax of the logits at the target) and loss = -sum(logprob)."""
+        hp = self.hp
+        dt = hp["delta_t"]
+        ctx = self.encode_context(enc_mem, ctx_len)
+        rows, toks, meta, targets = [], [], [], []
+        for i, sub in enumerate(subsequences, start=1):
+            term = hp["sep_id"] if terminators is None else int(terminators[i - 1])
+            seq = [hp["bos_id"]] + [int(t) for t in sub]
+            for p, tok in enumerate(seq):
+                rows.append((i, p))
+                toks.append(tok)
+                meta.append((i, timestamp(i, p, dt)))
+                targets.append(seq[p + 1] if p + 1 < len(seq) else term)
+        mask = self.visibility_matrix(meta, meta)
+        bias = self.position_bias(meta, meta) if self.pos_mode == POS_T5_BIAS else None
+        x = self.w["embed"][toks]
+        for l in range(self.L):
+            x, _, _ = self._layer(l, x, meta, None, None, mask, bias, ctx)
+        logits = self._logits(x)
+        mx = logits.max(axis=-1, keepdims=True)
+        lse = mx[:, 0] + np.log(np.exp(logits - mx).sum(axis=-1))
+        logprob = logits[np.arange(len(rows)), targets] - lse
+        return {"rows": rows, "targets": targets, "logits": logits, "logprob": logprob, "loss": float(-logprob.sum())}
 
     # ---- Algorithm 1 around either formulation
     def run(self, enc_mem: np.ndarray, ctx_len: int, forced_len: Optional[Sequence[int]] = None,

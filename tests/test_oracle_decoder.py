@@ -285,3 +285,49 @@ def test_workload_generator_is_deterministic_and_bf16_exact():
         c = W.CONFIGS[name]
         fl = W.make_forced_len(c)
         assert fl.shape == (c.batch, c.sub_max) and fl.min() >= 1 and fl.max() <= c.max_sub_len
+
+
+# ---------------------------------------------------------------- Eq. 6: the teacher-forced dense forward
+@pytest.mark.parametrize("pos_mode", [W.POS_T5_BIAS, W.POS_ROPE])
+def test_teacher_forward_equals_the_step_by_step_decode_under_teacher_forcing(pos_mode):
+    """Section 3.3: training sees the whole target at once under the dependency rule.  Every row's logits
+    must be the ones the step-by-step decode computes when it is fed the same tokens (the step at which
+    row (i, p) is the input of subsequence i is s_i + p), and the loss is the sum of the rows' negative
+    log-likelihoods of their targets, computed here with the library's cross-entropy."""
+    wl, wt, mem = build(SMALL, pos_mode=pos_mode)
+    o = O.PipelinedDecoderOracle(wt, wl.hyper())
+    fl = [4, 6, 3]
+    r = o.run(mem, wl.ctx, fl)
+    tf = o.teacher_forward(mem, wl.ctx, r["subsequences"])
+    assert [len(s) for s in r["subsequences"]] == fl and len(tf["rows"]) == sum(fl) + 3
+    by_step = {}
+    for s in r["trace"]:
+        for row, i in enumerate(s["active"]):
+            by_step[(i, s["t"] - r["starts"][i - 1])] = (s["logits"][row], s["appended"][i])
+    for k, (i, p) in enumerate(tf["rows"]):
+        lg, appended = by_step[(i, p)]
+        assert np.abs(tf["logits"][k] - lg).max() < 1e-10
+        assert tf["targets"][k] == appended                     # content token p + 1, or the separator at the end
+    want = F_cross_entropy(tf["logits"], tf["targets"])
+    assert abs(tf["loss"] - want) < 1e-9 * max(1.0, abs(want))
+    assert np.allclose(tf["logprob"].sum(), -tf["loss"])
+
+
+def F_cross_entropy(logits, targets):
+    return float(torch.nn.functional.cross_entropy(torch.as_tensor(logits, dtype=torch.float64),
+                                                   torch.as_tensor(targets, dtype=torch.long), reduction="sum"))
+
+
+def test_teacher_forward_of_a_single_subsequence_is_the_textbook_causal_forward():
+    wl, wt, mem = build(SMALL, sub_max=1, max_sub_len=24, time_max=64)
+    o = O.PipelinedDecoderOracle(wt, wl.hyper())
+    content = W.make_random_tokens(wl, (9,)).tolist()
+    tf = o.teacher_forward(mem, wl.ctx, [content], terminators=[wl.eos_id])
+    toks = [wl.bos_id] + content
+    want = textbook.causal_decoder_logits(wt, wl.hyper(), toks, [p + 1 for p in range(len(toks))], mem)
+    assert np.abs(tf["logits"] - want).max() < 1e-11
+    assert tf["targets"] == content + [wl.eos_id]
+    # an empty subsequence (the exploration that fails at once) is one row: bos -> terminator
+    tf2 = o.teacher_forward(mem, wl.ctx, [content, []])
+    assert tf2["rows"][-1] == (2, 0) and tf2["targets"][-1] == wl.sep_id
+    assert np.abs(tf2["logits"][:len(toks)] - tf["logits"]).max() < 1e-12       # later subsequences do not reach back
