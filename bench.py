@@ -301,6 +301,8 @@ def main():
     ap.add_argument("--no-sequential", action="store_true",
                     help="skip the sequential decoder (sub_max = 1 on the same targets), which is otherwise timed beside the "
                          "pipelined one at N = 1 for the speed-up the paper's tables report")
+    ap.add_argument("--no-teacher", action="store_true",
+                    help="skip the teacher-forced one-pass forward (Eq. 6) over the same targets")
     ap.add_argument("--no-queue", action="store_true",
                     help="skip the continuous-batching leg (a queue of 4 x batch sequences through the batch's rows)")
     ap.add_argument("--no-kv8", action="store_true",
@@ -506,6 +508,25 @@ def main():
     att = [r["frac"] for r in (roofline, roofline_self) if r]
     if att:
         line["roofline_min_attention_frac"] = min(att)
+    if rank == 0 and world == 1 and not args.no_teacher and wl.dtype == "bf16" and dec.rows_per_seq <= 32:
+        # the same targets scored in one teacher-forced pass (Section 3.3, Eq. 6) instead of decoded step by step
+        subs = [[res["tokens"][b, i, :res["lens"][b, i]].tolist() for i in range(int(res["n_sub"][b]))] for b in range(wl.batch)]
+        dec.encode_context(mem_dev, ctx_len, fl)
+        t_ms = []
+        for k in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(dec.stream)
+            lp, tf_loss, _ = dec.teacher_forward(subs)
+            b.record(dec.stream)
+            torch.cuda.synchronize()
+            if k >= 1:
+                t_ms.append(a.elapsed_time(b))
+        tf_ms = sum(t_ms) / len(t_ms)
+        line["teacher_forced_forward"] = {
+            "rows": int(len(lp)), "ms": tf_ms, "value": len(lp) / (tf_ms * 1e-3), "unit": "target tokens scored/s",
+            "loss_per_token": tf_loss / max(1, len(lp)), "speedup_over_decoding_them": (loss_ms_per_decode := loop_ms / args.steps) / tf_ms,
+            "note": "the decoded streams fed back as targets: every row's log-probability in one pass under the dense dependency "
+                    "rule (host tables up, log-probabilities down inside the timed region)"}
     if rank == 0 and world == 1 and not args.no_queue:
         line["continuous_batching"] = continuous_batching(dec, wl, mem_dev, ctx_len, fl, poll_every=4)
     if rank == 0 and world == 1 and not args.no_kv8 and wl.dtype == "bf16" and wl.ctx % 16 == 0 and dec.rows_per_seq <= 32:

@@ -191,6 +191,29 @@ PD_API pd_status pd_rows_done(pd_handle *h, int32_t *done, int32_t *steps);
 PD_API pd_status pd_collect_row(pd_handle *h, int32_t row, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags,
                                 int32_t *steps);
 
+/* The teacher-forced forward of Section 3.3 (Eq. 6): the whole target of every sequence in one pass instead of
+ * one time-step at a time.  Subsequence i of sequence b is given as its lens[b][i-1] content tokens; row (b, i, p),
+ * p = 0 .. lens, has the input <bos> (p = 0) or content token p, the timestamp (i-1)*delta_t + p, and attends to the
+ * rows the dependency rule lets it see (subsequence i' <= i, timestamp tau' <= tau - evaluated per pair, no mask is
+ * stored) and to the sequence's context; its target is content token p+1 or, at p = lens, the subsequence's
+ * terminator.  Row r's logits are the ones pd_step computes at step s_i + p when it is fed the same tokens.
+ * Uses the context keys/values of the last pd_encode_context (any kv_c_dtype); leaves the decode state untouched.
+ *   n_sub        host [batch]: subsequences of every sequence (0..sub_max; an empty one, lens = 0, is one row)
+ *   lens, tokens host [batch, sub_max], [batch, sub_max, max_sub_len]
+ *   terminators  host [batch, sub_max] or NULL (= sep_id everywhere)
+ *   scratch      device, 256-byte aligned, at least pd_teacher_forward_scratch_bytes(h, rows, own_logits) for the
+ *                sum over all subsequences of lens + 1 rows (own_logits = 1 when `logits` is NULL: the library then
+ *                works through the vocabulary projection in chunks of rows inside the scratch)
+ *   logprob      host [rows] or NULL: log P(target) per row, rows in (sequence, subsequence, position) order
+ *   logits       device fp32 [rows, vocab] or NULL: every row's logits (tests)
+ *   rows_out, loss_out  host or NULL: the row count, and Eq. 6's L = - sum of logprob
+ * bf16 path with at most 32 rows per sequence in pd_step (the tensor-core cross-attention kernel) only, else
+ * PD_ERR_UNSUPPORTED.  Synchronises. */
+PD_API size_t pd_teacher_forward_scratch_bytes(const pd_handle *h, int32_t max_rows, int32_t own_logits);
+PD_API pd_status pd_teacher_forward(pd_handle *h, const int32_t *n_sub, const int32_t *lens, const int32_t *tokens,
+                                    const int32_t *terminators, void *scratch, size_t scratch_bytes, float *logprob,
+                                    float *logits, int32_t *rows_out, double *loss_out);
+
 /* Whole Algorithm 1 from host buffers: copies enc_mem (host [batch, max_ctx, d_model], dtype;
  * pinned memory lets the copy overlap) to the device in chunks of sequences on a copy stream of
  * the handle's own while the context projection of the chunks already there runs on the handle's

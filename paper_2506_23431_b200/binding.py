@@ -58,6 +58,9 @@ _SIGS = {
     "pd_admit": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int32, _i32p]),
     "pd_rows_done": (C.c_int, [_H, _i32p, _i32p]),
     "pd_collect_row": (C.c_int, [_H, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "pd_teacher_forward_scratch_bytes": (C.c_size_t, [_H, C.c_int32, C.c_int32]),
+    "pd_teacher_forward": (C.c_int, [_H, _i32p, _i32p, _i32p, _i32p, C.c_void_p, C.c_size_t, C.POINTER(C.c_float), C.c_void_p,
+                                     _i32p, C.POINTER(C.c_double)]),
     "pd_generate_host": (C.c_int, [_H, C.c_void_p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "pd_get_trace": (C.c_int, [_H, C.POINTER(C.c_uint64)]),
     "pd_get_logits": (C.c_int, [_H, C.POINTER(C.c_float), _i32p]),
@@ -267,6 +270,38 @@ class PipelinedDecoder:
         n_sub, steps = np.empty((1,), np.int32), np.empty((1,), np.int32)
         self._check(_lib.pd_collect_row(self._h, int(row), _p(tokens), _p(lens), _p(n_sub), _p(flags), _p(steps)), "pd_collect_row")
         return {"tokens": tokens, "lens": lens, "n_sub": int(n_sub[0]), "flags": flags, "steps": int(steps[0])}
+
+    def teacher_forward(self, subsequences, terminators=None, want_logits: bool = False):
+        """Eq. 6 in one pass.  subsequences[b] = list of content-token lists of sequence b (after encode_context).
+        Returns (logprob float32 [rows], loss, logits torch CUDA float32 [rows, vocab] or None), rows in
+        (sequence, subsequence, position) order."""
+        torch = self.torch
+        sm, msl, B = self.cfg.sub_max, self.cfg.max_sub_len, self.batch
+        n_sub = np.zeros((B,), np.int32)
+        lens = np.zeros((B, sm), np.int32)
+        toks = np.zeros((B, sm, msl), np.int32)
+        term = None if terminators is None else np.zeros((B, sm), np.int32)
+        for b, subs in enumerate(subsequences):
+            n_sub[b] = len(subs)
+            for i, sub in enumerate(subs):
+                lens[b, i] = len(sub)
+                toks[b, i, :len(sub)] = sub
+                if term is not None:
+                    term[b, i] = terminators[b][i]
+        rows = int((lens + 1)[np.arange(sm)[None, :] < n_sub[:, None]].sum())
+        nbytes = int(_lib.pd_teacher_forward_scratch_bytes(self._h, max(rows, 1), 0 if want_logits else 1))
+        scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        sptr = (scratch.data_ptr() + 255) // 256 * 256
+        logits = torch.empty((max(rows, 1), self.cfg.vocab), dtype=torch.float32, device=self.device) if want_logits else None
+        lp = np.empty((max(rows, 1),), np.float32)
+        n_rows, loss = C.c_int32(0), C.c_double(0.0)
+        self.stream.wait_stream(torch.cuda.current_stream(self.device))
+        self._check(_lib.pd_teacher_forward(self._h, _p(n_sub), _p(lens), _p(toks), _p(term), C.c_void_p(sptr), C.c_size_t(nbytes),
+                                            lp.ctypes.data_as(C.POINTER(C.c_float)),
+                                            C.c_void_p(logits.data_ptr()) if want_logits else None, C.byref(n_rows), C.byref(loss)),
+                    "pd_teacher_forward")
+        assert n_rows.value == rows
+        return lp[:rows], loss.value, (logits[:rows] if want_logits else None)
 
     def generate_host(self, enc_mem_host, ctx_len, forced_len=None):
         """enc_mem_host: host buffer (torch CPU tensor, ideally pinned, or numpy array) of the model

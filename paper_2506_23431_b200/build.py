@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libpd.so")
-SOURCES = ["pd_api.cu", "kernels_misc.cu", "attn_core.cu", "cross_attn_tma.cu", "self_attn_tc.cu", "sched.cu", "attn_ops.cu", "attn_static.cu", "vocab_tc.cu", "vocab_ops.cu", "linear_tc.cu", "linear_ops.cu"]
+SOURCES = ["pd_api.cu", "kernels_misc.cu", "attn_core.cu", "cross_attn_tma.cu", "self_attn_tc.cu", "sched.cu", "attn_ops.cu", "attn_static.cu", "vocab_tc.cu", "vocab_ops.cu", "linear_tc.cu", "linear_ops.cu", "teacher_kernels.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

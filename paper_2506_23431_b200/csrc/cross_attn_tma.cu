@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(xthreads(FP8), 2) cross_attn_tma_kernel(const 
     if (lane == 0) n_aseq_s = n;
   }
   // rows of a sequence beyond its active ones come back as zeros (all heads)
-  for (int b = cta; b < batch; b += G) {
+  for (int b = cta; b < batch && a.row_base == nullptr; b += G) {
     const int S = nact_s[b];
     uint4 *z = reinterpret_cast<uint4 *>(out + (size_t)(b * dm.C + S) * dm.d);      // rows are d * 2 bytes, d a multiple of 64
     for (int idx = tid; idx < (dm.C - S) * dm.d / 8; idx += XTHREADS) z[idx] = make_uint4(0u, 0u, 0u, 0u);
@@ -320,13 +320,14 @@ __global__ void __launch_bounds__(xthreads(FP8), 2) cross_attn_tma_kernel(const 
         if (!mbar_wait(bar_empty + 8 * s, (u & 1u) ^ 1u)) { atomicExch(&a.st.hdr[HDR_STATUS], (int)PD_ERR_TIMEOUT); break; }
         mbar_expect_tx(bar_full + 8 * s, XSTAGE_BYTES);
         const uint32_t dst = base + s * XSTAGE_BYTES;
+        const int kv_b = a.kv_seq != nullptr ? a.kv_seq[cur.b] : cur.b;     // the sequence whose context this group reads
         if (FP8) {
           // block (layer, sequence, head) = max_ctx * 64 bytes of keys, then as many of transposed values
-          const int blk = (((a.layer * dm.B + cur.b) * H + cur.h) << 1);
+          const int blk = (((a.layer * dm.B + kv_b) * H + cur.h) << 1);
           tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, blk * (dm.ctx >> 1) + cur.tile * (XK / 2));    // 64 lines = 128 keys
           tma_load_3d(dst + XTILE_BYTES, &tmap_v, bar_full + 8 * s, cur.tile * XK, 0, blk + 1);       // 64 dims x 128 keys
         } else {
-          const int y = (int)(ctx_kv_offset(a.layer, dm.B, cur.b, H, cur.h, 0, dm.ctx) / kDh) + cur.tile * XK;
+          const int y = (int)(ctx_kv_offset(a.layer, dm.B, kv_b, H, cur.h, 0, dm.ctx) / kDh) + cur.tile * XK;
           tma_load_2d(dst, &tmap, bar_full + 8 * s, 0, y);                         // K tile
           tma_load_2d(dst + XTILE_BYTES, &tmap, bar_full + 8 * s, 0, y + dm.ctx);  // V tile
         }
@@ -350,10 +351,11 @@ __global__ void __launch_bounds__(xthreads(FP8), 2) cross_attn_tma_kernel(const 
     const int seg_start = H * pfx_s[b] + h * cur.nt, seg_end = seg_start + cur.nt;
     const int my_end = min(hi, seg_end);
     const int S = nact_s[b], ctx_len = min(max(a.st.ctx_len[b], 1), dm.ctx);
-    const int row0 = b * dm.C;
+    const int row0 = a.row_base != nullptr ? a.row_base[b] : b * dm.C;
     float seg_sl2 = sl2, seg_vscale = 1.f;          // 8-bit: the key scale joins the score scale, the value scale the final 1 / l
     if (FP8) {
-      const float2 sc2 = *reinterpret_cast<const float2 *>(a.kv_scale + ((((size_t)a.layer * dm.B + b) * H + h) << 1));
+      const int kv_b = a.kv_seq != nullptr ? a.kv_seq[b] : b;
+      const float2 sc2 = *reinterpret_cast<const float2 *>(a.kv_scale + ((((size_t)a.layer * dm.B + kv_b) * H + h) << 1));
       seg_sl2 = sl2 * sc2.x; seg_vscale = sc2.y;
     }
     uint32_t qf[MT][4][4];

@@ -6,6 +6,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -320,6 +321,7 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.qkv = h->ptr<void>(h->lay.qkv);
   a.fused_append = self && fused_append(h) ? 1 : 0;
   a.kv_scale = (!self && h->kv8) ? h->ptr<float>(h->lay.kv_scale) : nullptr;
+  a.kv_seq = nullptr; a.row_base = nullptr;
   return a;
 }
 
@@ -812,6 +814,160 @@ pd_status pd_collect_row(pd_handle *h, int32_t row, int32_t *tokens, int32_t *le
   if (flags) CU_TRY(h, cudaMemcpyAsync(flags, h->st.flag + r * dm.SM, (size_t)dm.SM * 4, cudaMemcpyDeviceToHost, s));
   if (steps) CU_TRY(h, cudaMemcpyAsync(steps, h->st.steps + r, 4, cudaMemcpyDeviceToHost, s));
   return device_status(h);
+}
+
+// ---- the teacher-forced forward of Eq. 6 -----------------------------------------------------------------
+namespace {
+constexpr int kTfGroup = 32;          // query rows per attention group
+constexpr int kTfCrossBatch = 256;    // groups per cross-attention launch
+struct TfLayout { size_t tables, x, hb, qkv, att, cq, co, ffn, logprob, part, tickets, logits, total; int logit_rows; };
+
+TfLayout tf_layout(const Dims &dm, size_t rows, bool own_logits) {
+  TfLayout L;
+  size_t off = 0;
+  auto reg = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, kAlign); return o; };
+  const size_t groups = rows / 1 + (size_t)dm.B;                     // generous: every sequence may end with a short group
+  L.tables = reg((4 * rows + 6 * groups) * sizeof(int32_t));
+  L.x = reg(rows * dm.d * 4);
+  L.hb = reg(rows * dm.d * 2);
+  L.qkv = reg(rows * 3 * dm.d * 4);
+  L.att = reg(rows * dm.d * 2);
+  L.cq = reg(rows * dm.d * 2);
+  L.co = reg(rows * dm.d * 2);
+  L.ffn = reg(rows * dm.ff * 2);
+  L.logprob = reg(rows * 4);
+  L.part = reg(cross_attn_tma_partial_bytes(kMaxCrossCtas, kTfGroup));
+  L.tickets = reg((size_t)kTfCrossBatch * dm.H * 4);
+  L.logit_rows = 0;
+  L.logits = off;
+  if (own_logits) {
+    size_t lr = ((size_t)256 << 20) / ((size_t)dm.V * 4);             // a logits chunk of about 256 MiB
+    if (lr < 1) lr = 1;
+    if (lr > rows) lr = rows;
+    L.logit_rows = (int)lr;
+    L.logits = reg(lr * dm.V * 4);
+  }
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t pd_teacher_forward_scratch_bytes(const pd_handle *h, int32_t max_rows, int32_t own_logits) {
+  if (!h || max_rows < 1) return 0;
+  return tf_layout(h->dm, (size_t)max_rows, own_logits != 0).total;
+}
+
+pd_status pd_teacher_forward(pd_handle *h, const int32_t *n_sub, const int32_t *lens, const int32_t *tokens,
+                             const int32_t *terminators, void *scratch, size_t scratch_bytes, float *logprob, float *logits,
+                             int32_t *rows_out, double *loss_out) {
+  if (!h) return PD_ERR_ARG;
+  if (!n_sub || !lens || !tokens || !scratch) return fail(h, PD_ERR_ARG, "pd_teacher_forward: null argument");
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_teacher_forward before pd_encode_context");
+  const Dims &dm = h->dm;
+  if (h->cfg.dtype != PD_DTYPE_BF16 || !h->have_tmap)
+    return fail(h, PD_ERR_UNSUPPORTED, "pd_teacher_forward runs on the bf16 path (tensor-core cross-attention) only");
+  if (reinterpret_cast<uintptr_t>(scratch) % kAlign != 0) return fail(h, PD_ERR_ARG, "pd_teacher_forward: misaligned scratch");
+  // ---- rows in (sequence, subsequence, position) order; groups of up to 32 rows inside a sequence
+  std::vector<int32_t> row_sub, row_tau, row_tok, row_tgt, g_row0, g_n, g_srow0, g_srows, g_seq, g_ctx;
+  std::vector<int32_t> ctx_len(h->batch);
+  CU_TRY(h, cudaMemcpyAsync(ctx_len.data(), h->st.ctx_len, (size_t)h->batch * 4, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));
+  for (int b = 0; b < h->batch; ++b) {
+    if (n_sub[b] < 0 || n_sub[b] > dm.SM) return fail(h, PD_ERR_ARG, "pd_teacher_forward: n_sub out of range");
+    const int srow0 = (int)row_sub.size();
+    for (int i = 1; i <= n_sub[b]; ++i) {
+      const int m = lens[b * dm.SM + i - 1];
+      if (m < 0 || m > dm.MSL) return fail(h, PD_ERR_ARG, "pd_teacher_forward: subsequence length out of range");
+      const int32_t *sub = tokens + ((size_t)b * dm.SM + i - 1) * dm.MSL;
+      const int term = terminators ? terminators[b * dm.SM + i - 1] : dm.sep;
+      for (int p = 0; p <= m; ++p) {
+        const int tok = p == 0 ? dm.bos : sub[p - 1], tgt = p < m ? sub[p] : term;
+        if (tok < 0 || tok >= dm.V || tgt < 0 || tgt >= dm.V) return fail(h, PD_ERR_ARG, "pd_teacher_forward: token id out of range");
+        row_sub.push_back(i); row_tau.push_back((i - 1) * dm.dt + p); row_tok.push_back(tok); row_tgt.push_back(tgt);
+      }
+    }
+    const int srows = (int)row_sub.size() - srow0;
+    if (srows > 0 && (n_sub[b] - 1) * dm.dt + dm.MSL + dm.SM >= dm.n_dist) return fail(h, PD_ERR_ARG, "pd_teacher_forward: positions beyond the tables");
+    for (int r = 0; r < srows; r += kTfGroup) {
+      g_row0.push_back(srow0 + r); g_n.push_back(std::min(kTfGroup, srows - r));
+      g_srow0.push_back(srow0); g_srows.push_back(srows); g_seq.push_back(b); g_ctx.push_back(ctx_len[b]);
+    }
+  }
+  const size_t R = row_sub.size(), G = g_row0.size();
+  if (rows_out) *rows_out = (int32_t)R;
+  if (loss_out) *loss_out = 0.0;
+  if (R == 0) return PD_OK;
+  const TfLayout L = tf_layout(dm, R, logits == nullptr);
+  if (scratch_bytes < L.total) return fail(h, PD_ERR_WORKSPACE, "pd_teacher_forward: scratch too small (pd_teacher_forward_scratch_bytes)");
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  cudaStream_t s = h->stream;
+  uint8_t *base = reinterpret_cast<uint8_t *>(scratch);
+  int32_t *tab = reinterpret_cast<int32_t *>(base + L.tables);
+  int32_t *d_sub = tab, *d_tau = tab + R, *d_tok = tab + 2 * R, *d_tgt = tab + 3 * R, *d_g = tab + 4 * R;
+  int32_t *d_grow0 = d_g, *d_gn = d_g + G, *d_gsrow0 = d_g + 2 * G, *d_gsrows = d_g + 3 * G, *d_gseq = d_g + 4 * G, *d_gctx = d_g + 5 * G;
+  auto up = [&](int32_t *dst, const std::vector<int32_t> &v) { return cudaMemcpyAsync(dst, v.data(), v.size() * 4, cudaMemcpyHostToDevice, s); };
+  CU_TRY(h, up(d_sub, row_sub)); CU_TRY(h, up(d_tau, row_tau)); CU_TRY(h, up(d_tok, row_tok)); CU_TRY(h, up(d_tgt, row_tgt));
+  CU_TRY(h, up(d_grow0, g_row0)); CU_TRY(h, up(d_gn, g_n)); CU_TRY(h, up(d_gsrow0, g_srow0)); CU_TRY(h, up(d_gsrows, g_srows));
+  CU_TRY(h, up(d_gseq, g_seq)); CU_TRY(h, up(d_gctx, g_ctx));
+  CU_TRY(h, cudaMemsetAsync(base + L.tickets, 0, (size_t)kTfCrossBatch * dm.H * 4, s));
+  CU_TRY(h, cudaStreamSynchronize(s));               // the host vectors may go
+
+  float *x = reinterpret_cast<float *>(base + L.x);
+  void *hb = base + L.hb, *qkv = base + L.qkv, *att = base + L.att, *cq = base + L.cq, *co = base + L.co, *ffn = base + L.ffn;
+  const int M = (int)R;
+  const bool rope = dm.pos_mode == PD_POS_ROPE;
+  OWN(h, PD_PROF_OTHER, launch_gather_rows(M, dm.d, d_tok, h->w.embed, x, s));
+  for (int l = 0; l < dm.L; ++l) {
+    const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, PD_DTYPE_BF16, x, lw[0], hb, s));
+    PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, rope, 0.f));
+    DenseAttnArgs da;
+    da.H = dm.H; da.d = dm.d; da.n_groups = (int)G; da.scale_log2e = dm.scale_log2e;
+    da.qkv = qkv; da.qkv_f32 = rope ? 1 : 0; da.out = reinterpret_cast<__nv_bfloat16 *>(att);
+    da.row_sub = d_sub; da.row_tau = d_tau; da.grp_row0 = d_grow0; da.grp_n = d_gn; da.grp_seq_row0 = d_gsrow0; da.grp_seq_rows = d_gsrows;
+    da.bias_tab = rope ? nullptr : h->ptr<float>(h->lay.bias_tab); da.n_dist = dm.n_dist;
+    da.rope_tab = rope ? h->ptr<float2>(h->lay.rope_tab) : nullptr;
+    OWN(h, PD_PROF_SELF_ATTN, launch_dense_self_attn(da, s));
+    PD_TRY(gemm(h, false, M, dm.d, dm.d, att, lw[2], x, true, 1.f));
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, PD_DTYPE_BF16, x, lw[3], hb, s));
+    PD_TRY(gemm(h, false, M, dm.d, dm.d, hb, lw[4], cq, false, 0.f));
+    for (size_t g0 = 0; g0 < G; g0 += kTfCrossBatch) {              // groups as "sequences" of the batched kernel, 256 at a time
+      AttnArgs a = attn_args(h, l, false);
+      a.dm.C = kTfGroup;
+      a.batch = (int)std::min<size_t>(kTfCrossBatch, G - g0);
+      a.q = cq; a.out = co;
+      a.st.n_active = d_gn + g0; a.st.ctx_len = d_gctx + g0;
+      a.kv_seq = d_gseq + g0; a.row_base = d_grow0 + g0;
+      a.part_o = reinterpret_cast<float *>(base + L.part);
+      a.tickets = reinterpret_cast<int32_t *>(base + L.tickets);
+      OWN(h, PD_PROF_CROSS_ATTN, launch_cross_attn_tma(a, h->tmap_kvc, h->kv8 ? h->tmap_kvc_v : h->tmap_kvc, h->cross_ctas, s));
+    }
+    PD_TRY(gemm(h, false, M, dm.d, dm.d, co, lw[6], x, true, 1.f));
+    OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, PD_DTYPE_BF16, x, lw[7], hb, s));
+    PD_TRY(gemm(h, false, M, dm.ff, dm.d, hb, lw[8], ffn, false, 0.f));
+    OWN(h, PD_PROF_OTHER, launch_relu(PD_DTYPE_BF16, ffn, (size_t)M * dm.ff, s));
+    PD_TRY(gemm(h, false, M, dm.d, dm.ff, ffn, lw[9], x, true, 1.f));
+  }
+  OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, PD_DTYPE_BF16, x, h->w.final_norm, hb, s));
+  float *d_lp = reinterpret_cast<float *>(base + L.logprob);
+  if (logits != nullptr) {
+    PD_TRY(gemm(h, true, M, dm.V, dm.d, hb, h->w.lm_head, logits, true, 0.f));
+    OWN(h, PD_PROF_OTHER, launch_target_logprob(M, dm.V, logits, d_tgt, d_lp, s));
+  } else {
+    float *chunk = reinterpret_cast<float *>(base + L.logits);
+    for (int r0 = 0; r0 < M; r0 += L.logit_rows) {
+      const int n = std::min(L.logit_rows, M - r0);
+      PD_TRY(gemm(h, true, n, dm.V, dm.d, reinterpret_cast<uint8_t *>(hb) + (size_t)r0 * dm.d * 2, h->w.lm_head, chunk, true, 0.f));
+      OWN(h, PD_PROF_OTHER, launch_target_logprob(n, dm.V, chunk, d_tgt + r0, d_lp + r0, s));
+    }
+  }
+  std::vector<float> lp(R);
+  CU_TRY(h, cudaMemcpyAsync(lp.data(), d_lp, R * 4, cudaMemcpyDeviceToHost, s));
+  PD_TRY(device_status(h));
+  double loss = 0.0;
+  for (size_t r = 0; r < R; ++r) { loss -= (double)lp[r]; if (logprob) logprob[r] = lp[r]; }
+  if (loss_out) *loss_out = loss;
+  return PD_OK;
 }
 
 pd_status pd_generate_host(pd_handle *h, const void *enc_mem_host, const int32_t *ctx_len, int32_t batch,

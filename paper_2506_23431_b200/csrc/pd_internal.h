@@ -104,7 +104,28 @@ struct AttnArgs {
   int fused_append;
   // cross-attention over 8-bit keys/values: [layer][sequence][head][keys | values] fp32 scales (else null)
   const float *kv_scale;
+  // cross-attention over row groups that are not one per sequence (the teacher-forced forward: many rows per
+  // sequence, in groups of up to 32): the sequence whose context group g reads, and the group's first row;
+  // null = group g is sequence g with rows g * C ...
+  const int32_t *kv_seq;
+  const int32_t *row_base;
 };
+
+// ---- teacher-forced dense forward (teacher_kernels.cu) ------------------------------------------------
+struct DenseAttnArgs {
+  int H, d, n_groups;
+  float scale_log2e;
+  const void *qkv; int qkv_f32;          // [rows][3 d]: bf16, or fp32 (rotary mode: rotated here)
+  __nv_bfloat16 *out;                    // [rows][d]
+  const int32_t *row_sub, *row_tau;      // [rows] subsequence i and timestamp tau of every row
+  const int32_t *grp_row0, *grp_n;       // [groups] first row and number of rows (<= 32) of a query group
+  const int32_t *grp_seq_row0, *grp_seq_rows;   // [groups] first row and row count of the group's sequence (its keys)
+  const float *bias_tab; int n_dist;     // T5 mode: [H][n_dist], log2(e)-scaled; else null
+  const float2 *rope_tab;                // rotary mode: [n_dist][32] (cos, sin); else null
+};
+cudaError_t launch_dense_self_attn(const DenseAttnArgs &a, cudaStream_t s);
+cudaError_t launch_gather_rows(int rows, int d, const int32_t *row_tok, const void *embed, float *x, cudaStream_t s);
+cudaError_t launch_target_logprob(int rows, int V, const float *logits, const int32_t *targets, float *logprob, cudaStream_t s);
 
 // ---- launchers (each enqueues on `s`; returns cudaGetLastError()) ------------------------
 cudaError_t launch_reset_state(const Dims &dm, const DecState &st, int batch, const int32_t *ctx_len_dev,
