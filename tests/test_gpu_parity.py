@@ -146,6 +146,36 @@ def test_bf16_long_page_lists():
     dec.close()
 
 
+def test_bf16_free_running_cap_and_time_max():
+    """No forced lengths on the bf16 path: subsequences run into the max_sub_len cap (ended with sep, flag capped) and
+    time_max cuts the rest (flag truncated); every step replayed against the oracle."""
+    wl = W.CONFIGS["summarisation"].scaled(name="bf16_cap", batch=3, ctx=80, sub_max=6, delta_t=2, max_sub_len=7, time_max=15,
+                                           **SMALL_BF16)
+    weights, mem, ctx_len, dec, rows = make(wl, ragged=True)
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, None)
+    assert any(f & 4 for r in runs.values() for f in r["flags"]) and any(f & 2 for r in runs.values() for f in r["flags"])
+    s = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, None, runs)
+    assert s["max_err"] < 2e-2
+    dec.close()
+
+
+@pytest.mark.parametrize("pos_mode", [W.POS_T5_BIAS, W.POS_ROPE])
+def test_bf16_one_row_per_sequence_one_sequence_tiny_context(pos_mode):
+    """delta_t beyond every length: at most one subsequence is open at a time (one row per sequence, the smallest row
+    block), a batch of one, and a context shorter than a key tile."""
+    wl = W.CONFIGS["bart_base"].scaled(name="bf16_one_row", batch=1, ctx=16, sub_max=4, delta_t=12, max_sub_len=10,
+                                       length_dist=("uniform", 6, 10), time_max=60, pos_mode=pos_mode, **SMALL_BF16)
+    weights, mem, _, dec, rows = make(wl)
+    assert dec.rows_per_seq == 1
+    ctx_len = np.array([11], dtype=np.int32)
+    fl = W.make_forced_len(wl)
+    runs = parity.oracle_runs(wl, weights, {0: mem[0]}, ctx_len, fl)
+    s = parity.replay_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    assert s["max_err"] < 2e-2 and s["choices"] > 0
+    parity.free_run_compare(dec, wl, dec.device_memory(mem), ctx_len, fl, runs)
+    dec.close()
+
+
 def test_steps_after_the_end_are_no_ops():
     from paper_2506_23431_b200.binding import PipelinedDecoder
     wl = TINY.scaled(vocab=300)
