@@ -36,6 +36,12 @@ What follows the paper and what is a reading of it:
                          (every subsequence as [bos, Y_i], inputs given) under the dense dependency
                          mask; returns the logits of every position and the loss
                          L = - sum_(i,t) log P(target_i^(t+1) | targets seen under the rule; H^E).
+* start plans          - an option of this build for Section 6's "new subsequences adaptively rather
+                         than at fixed time intervals": `decode`, `run` and `teacher_forward` take the
+                         start step of every subsequence (increasing, the first one 1) instead of
+                         deriving it from delta_t; entry p of a subsequence started at s carries the
+                         timestamp s - 1 + p, which is Eq. 2's (i-1) delta_t + p for the fixed plan
+                         s_i = (i-1) delta_t + 1.  Everything else (rule, distance, stop test) is unchanged.
 * `e4m3_round`, `quantize_context_kv` - an option of this build, not of the paper (hp["kv_c_dtype"] =
   "e4m3"): the cross-attention keys/values of Eq. 1's encoder memory are stored as 8-bit floats
   (OCP FP8 E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest
@@ -64,6 +70,11 @@ FLAG_CAPPED = 4      # terminator imposed because max_sub_len content tokens wer
 def timestamp(i: int, p: int, delta_t: int) -> int:
     """Step at which entry p of subsequence i was generated (p = 0 is bos).  Eq. 2 prose."""
     return (i - 1) * delta_t + p
+
+
+def fixed_plan(delta_t: int, sub_max: int) -> List[int]:
+    """Eq. 2's start steps: s_i = (i-1) delta_t + 1."""
+    return [(i - 1) * delta_t + 1 for i in range(1, sub_max + 1)]
 
 
 def visible(i_q: int, tau_q: int, i_k: int, tau_k: int) -> bool:
@@ -104,7 +115,7 @@ class Sub:
 
 
 def decode(step_fn: Callable[[List[Sub], int, List[int]], Dict[int, int]], delta_t: int, time_max: int,
-           sub_max: int, bos: int, terminators: Sequence[int]):
+           sub_max: int, bos: int, terminators: Sequence[int], start_plan: Optional[Sequence[int]] = None):
     """The decoding procedure of Section 3.4.  `step_fn(G, t, active)` plays Decoder(G, H^E): it returns
     the new token of every active (not yet ended) subsequence.  Returns (G, steps_used, trace) where
     trace[t-1] = (active list, {i: token}) and G keeps bos (callers strip with `strip`).
@@ -112,16 +123,24 @@ def decode(step_fn: Callable[[List[Sub], int, List[int]], Dict[int, int]], delta
     The schedule comes from Eq. 2: while the procedure runs, the number of subsequences at step t is
     k(t) = min(sub_max, ceil(t / delta_t)), so subsequence i appears exactly at s_i = (i-1) delta_t + 1;
     k(t) grows by at most one per step, which is the paper's "a new subsequence every delta_t steps while
-    fewer than sub_max exist"."""
+    fewer than sub_max exist".  With `start_plan` (increasing start steps, the first one 1, at most sub_max of them)
+    subsequence i appears at start_plan[i-1] instead: k(t) = number of planned starts <= t."""
+    if start_plan is not None:
+        plan = [int(x) for x in start_plan][:sub_max]
+        if not plan or plan[0] != 1 or any(b <= a for a, b in zip(plan, plan[1:])):
+            raise ValueError("a start plan begins at step 1 and increases")
     G: List[Sub] = []
     trace = []
     t = 0
     while t < time_max:
         t += 1
-        k_t = min(sub_max, -(-t // delta_t))                 # Eq. 2, capped
+        if start_plan is None:
+            k_t = min(sub_max, -(-t // delta_t))             # Eq. 2, capped
+        else:
+            k_t = sum(1 for s_i in plan if s_i <= t)
         if len(G) < k_t:
             i = len(G) + 1
-            assert k_t == i and (i - 1) * delta_t + 1 == t   # one at a time, at its start step
+            assert k_t == i and (plan[i - 1] if start_plan is not None else (i - 1) * delta_t + 1) == t   # one at a time, at its start step
             G.append(Sub(i, t, bos))
         active = [s.index for s in G if not s.ended]
         new = step_fn(G, t, active)
@@ -357,24 +376,24 @@ class PipelinedDecoderOracle:
         for s in G:
             for p, tok in enumerate(s.tokens):
                 toks.append(tok)
-                meta.append((s.index, timestamp(s.index, p, dt)))
+                meta.append((s.index, s.start - 1 + p))
         mask = self.visibility_matrix(meta, meta)
         bias = self.position_bias(meta, meta) if self.pos_mode == POS_T5_BIAS else None
         x = self.w["embed"][toks]
         for l in range(self.L):
             x, _, _ = self._layer(l, x, meta, None, None, mask, bias, ctx)
-        last = [meta.index((i, timestamp(i, G[i - 1].n_content, dt))) for i in active]
+        last = [meta.index((i, G[i - 1].start - 1 + G[i - 1].n_content)) for i in active]
         return self._logits(x[last])
 
     # ---- Eq. 6: the whole target in one teacher-forced pass under the dense mask
     def teacher_forward(self, enc_mem: np.ndarray, ctx_len: int, subsequences: Sequence[Sequence[int]],
-                        terminators: Optional[Sequence[int]] = None):
+                        terminators: Optional[Sequence[int]] = None, start_plan: Optional[Sequence[int]] = None):
         """subsequences[i-1] = the content tokens of subsequence i.  Row (i, p), p = 0..m_i, has input bos
         (p = 0) or content token p, timestamp (i-1) delta_t + p, and target content token p + 1 or, at
         p = m_i, the subsequence's terminator (sep unless given).  Returns a dict: rows [(i, p)], targets,
         logits [R, vocab], logprob [R] (log-softmax of the logits at the target) and loss = -sum(logprob)."""
         hp = self.hp
-        dt = hp["delta_t"]
+        starts = fixed_plan(hp["delta_t"], len(subsequences)) if start_plan is None else [int(x) for x in start_plan]
         ctx = self.encode_context(enc_mem, ctx_len)
         rows, toks, meta, targets = [], [], [], []
         for i, sub in enumerate(subsequences, start=1):
@@ -383,7 +402,7 @@ class PipelinedDecoderOracle:
             for p, tok in enumerate(seq):
                 rows.append((i, p))
                 toks.append(tok)
-                meta.append((i, timestamp(i, p, dt)))
+                meta.append((i, starts[i - 1] - 1 + p))
                 targets.append(seq[p + 1] if p + 1 < len(seq) else term)
         mask = self.visibility_matrix(meta, meta)
         bias = self.position_bias(meta, meta) if self.pos_mode == POS_T5_BIAS else None
@@ -399,7 +418,7 @@ class PipelinedDecoderOracle:
     # ---- Algorithm 1 around either formulation
     def run(self, enc_mem: np.ndarray, ctx_len: int, forced_len: Optional[Sequence[int]] = None,
             teacher: Optional[Callable[[int, int], Optional[int]]] = None, formulation: str = "B",
-            keep_logits: bool = True):
+            keep_logits: bool = True, start_plan: Optional[Sequence[int]] = None):
         """Decode one sequence.  `teacher(i, t)`, when given and not None for that (i, t),
         replaces the chosen token as the one appended (the oracle's own choice is still
         recorded).  A subsequence that already holds max_sub_len content tokens ends with sep
@@ -417,7 +436,8 @@ class PipelinedDecoderOracle:
             if formulation == "B":
                 rows = [(i, t - 1, G[i - 1].tokens[-1]) for i in active]
                 for (i, tau, _) in rows:
-                    assert tau == timestamp(i, G[i - 1].n_content, dt)
+                    assert tau == G[i - 1].start - 1 + G[i - 1].n_content
+                    assert start_plan is not None or tau == timestamp(i, G[i - 1].n_content, dt)
                 logits = self.step_incremental(cache, rows, ctx)
             elif formulation == "A":
                 logits = self.step_dense(G, active, ctx)
@@ -442,7 +462,7 @@ class PipelinedDecoderOracle:
             return appended
 
         G, steps, _ = decode(step_fn, dt, hp["time_max"], hp["sub_max"], hp["bos_id"],
-                             (hp["eos_id"], hp["sep_id"]))
+                             (hp["eos_id"], hp["sep_id"]), start_plan)
         for i in capped:
             G[i - 1].flag |= FLAG_CAPPED
         return {"subsequences": strip(G), "flags": [s.flag for s in G], "n_sub": len(G), "steps": steps,

@@ -331,3 +331,33 @@ def test_teacher_forward_of_a_single_subsequence_is_the_textbook_causal_forward(
     tf2 = o.teacher_forward(mem, wl.ctx, [content, []])
     assert tf2["rows"][-1] == (2, 0) and tf2["targets"][-1] == wl.sep_id
     assert np.abs(tf2["logits"][:len(toks)] - tf["logits"]).max() < 1e-12       # later subsequences do not reach back
+
+
+def test_start_plan_equal_to_eq_2_changes_nothing_and_an_uneven_one_keeps_the_reductions():
+    """Timestamps follow the start steps: with Eq. 2's plan every logit is the fixed-interval one; with an uneven plan the
+    dense and the incremental formulation still agree, the teacher-forced forward still equals the step-by-step decode,
+    and later subsequences still do not reach back."""
+    wl, wt, mem = build(SMALL)
+    o = O.PipelinedDecoderOracle(wt, wl.hyper())
+    fl = [4, 6, 3]
+    base = o.run(mem, wl.ctx, fl)
+    same = o.run(mem, wl.ctx, fl, start_plan=O.fixed_plan(wl.delta_t, wl.sub_max))
+    assert base["subsequences"] == same["subsequences"] and base["steps"] == same["steps"]
+    for x, y in zip(base["trace"], same["trace"]):
+        assert x["active"] == y["active"] and np.array_equal(x["logits"], y["logits"])
+    plan = [1, 2, 6]
+    a = o.run(mem, wl.ctx, fl, formulation="A", start_plan=plan)
+    b = o.run(mem, wl.ctx, fl, formulation="B", start_plan=plan)
+    assert a["starts"] == plan and b["starts"] == plan and a["steps"] == b["steps"] == 9
+    for x, y in zip(a["trace"], b["trace"]):
+        assert x["active"] == y["active"] and np.abs(x["logits"] - y["logits"]).max() < 1e-10
+    assert any(not np.array_equal(x["logits"], y["logits"]) for x, y in zip(b["trace"][1:], base["trace"][1:]))
+    tf = o.teacher_forward(mem, wl.ctx, b["subsequences"], start_plan=plan)
+    by_step = {(i, s["t"] - b["starts"][i - 1]): s["logits"][row] for s in b["trace"] for row, i in enumerate(s["active"])}
+    for k, (i, p) in enumerate(tf["rows"]):
+        assert np.abs(tf["logits"][k] - by_step[(i, p)]).max() < 1e-10
+    # non-interference under the plan: subsequence 1's logits do not depend on what the later ones are taught
+    c = o.run(mem, wl.ctx, fl, start_plan=plan, teacher=lambda i, t: (7 if i > 1 else None))
+    for x, y in zip(b["trace"], c["trace"]):
+        if 1 in x["active"]:
+            assert np.array_equal(x["logits"][x["active"].index(1)], y["logits"][y["active"].index(1)])

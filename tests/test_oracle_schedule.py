@@ -122,3 +122,32 @@ def test_select_token_rules():
     assert O.select_token(logits, 0, 3, 4, 1, 2) == (3, False)             # terminators barred, tie -> lowest id
     assert O.select_token(logits, 3, 3, 4, 1, 2) == (2, False)             # (m+1)-th emission is sep
     assert O.select_token(np.array([1.0, 1.0, 1.0]), 0, None, 4, 7, 8)[0] == 0
+
+
+# ---------------------------------------------------------------- start plans (subsequences not at fixed intervals)
+def test_the_fixed_plan_is_eq_2_and_gives_the_same_decode():
+    """A plan equal to Eq. 2's start steps must reproduce the fixed-interval procedure exactly; an uneven plan starts
+    every subsequence at its planned step, still one per step, and stops by the same rule."""
+    def scripted(lengths):
+        def step_fn(G, t, active):
+            return {i: (2 if G[i - 1].n_content >= lengths[i - 1] else 10 + i) for i in active}
+        return step_fn
+    for delta_t, sub_max in ((1, 4), (2, 5), (3, 3)):
+        lengths = [5, 2, 6, 1, 4][:sub_max]
+        plan = O.fixed_plan(delta_t, sub_max)
+        assert plan == [(i - 1) * delta_t + 1 for i in range(1, sub_max + 1)]
+        a = O.decode(scripted(lengths), delta_t, 60, sub_max, 0, (1, 2))
+        b = O.decode(scripted(lengths), delta_t, 60, sub_max, 0, (1, 2), start_plan=plan)
+        assert O.strip(a[0]) == O.strip(b[0]) and a[1] == b[1] and a[2] == b[2]
+        assert [s.start for s in a[0]] == [s.start for s in b[0]]
+    G, steps, trace = O.decode(scripted([6, 6, 2]), 2, 60, 3, 0, (1, 2), start_plan=[1, 2, 6])
+    assert [s.start for s in G] == [1, 2, 6]
+    assert [a for a, _ in trace][:6] == [[1], [1, 2], [1, 2], [1, 2], [1, 2], [1, 2, 3]]
+    assert steps == 8 and O.strip(G) == [[11] * 6, [12] * 6, [13] * 2]
+    # the plan's later starts do not keep a finished sequence alive (the stop test sees only what it holds)
+    G, steps, _ = O.decode(scripted([1, 9, 9]), 2, 60, 3, 0, (1, 2), start_plan=[1, 5, 9])
+    assert steps == 2 and len(G) == 1
+    with pytest.raises(ValueError):
+        O.decode(scripted([1]), 2, 10, 3, 0, (1, 2), start_plan=[2, 3])
+    with pytest.raises(ValueError):
+        O.decode(scripted([1]), 2, 10, 3, 0, (1, 2), start_plan=[1, 1])
