@@ -169,6 +169,17 @@ PD_API pd_status pd_done(pd_handle *h, int32_t *all_done);
 PD_API pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_sub, int32_t *flags,
                      int32_t *steps);
 
+/* Start steps that are not at fixed intervals (Section 6 names "new subsequences adaptively rather than at fixed time
+ * intervals" as future work; the policy is the caller's, the library takes its outcome): plan[b][i-1] = the step of
+ * sequence b's own clock at which subsequence i is admitted, instead of Eq. 2's (i-1)*delta_t + 1.  Host
+ * [batch, sub_max]; every plan starts at 1 and its start steps are at least cfg.delta_t apart (which keeps the bound on
+ * concurrently open subsequences the workspace is sized for), else PD_ERR_ARG.  Entry p of a subsequence started at s
+ * carries the timestamp s - 1 + p; the dependency rule, the Manhattan distance and the stop test are unchanged (a
+ * sequence whose held subsequences have all ended stops, later planned starts or not).  Call it after
+ * pd_encode_context and before the first pd_step (PD_ERR_STATE otherwise); pd_encode_context and pd_admit put the
+ * fixed-interval plan back.  pd_teacher_forward uses the plan in force.  Synchronises. */
+PD_API pd_status pd_set_start_plan(pd_handle *h, const int32_t *plan);
+
 /* Continuous batching: a new sequence in a row whose sequence has ended, between two steps (Algorithm 1
  * runs per sequence; rows only share the step clock).  The row starts over as pd_encode_context would leave
  * it - state cleared, subsequence 1 admitted, its own step counter at 1 for the coming pd_step, its pages its

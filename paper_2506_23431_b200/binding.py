@@ -55,6 +55,7 @@ _SIGS = {
     "pd_run": (C.c_int, [_H, C.c_int32, _i32p]),
     "pd_done": (C.c_int, [_H, _i32p]),
     "pd_collect": (C.c_int, [_H, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "pd_set_start_plan": (C.c_int, [_H, _i32p]),
     "pd_admit": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int32, _i32p]),
     "pd_rows_done": (C.c_int, [_H, _i32p, _i32p]),
     "pd_collect_row": (C.c_int, [_H, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
@@ -245,6 +246,11 @@ class PipelinedDecoder:
         steps = np.empty((b,), np.int32)
         self._check(_lib.pd_collect(self._h, _p(tokens), _p(lens), _p(n_sub), _p(flags), _p(steps)), "pd_collect")
         return {"tokens": tokens, "lens": lens, "n_sub": n_sub, "flags": flags, "steps": steps}
+
+    def set_start_plan(self, plan):
+        """plan [batch, sub_max]: start step of every subsequence (after encode_context, before the first step)."""
+        pl = _np_i32(plan, (self.batch, self.cfg.sub_max))
+        self._check(_lib.pd_set_start_plan(self._h, _p(pl)), "pd_set_start_plan")
 
     def admit(self, row: int, enc_mem, ctx_len: int, forced_len=None):
         """A new sequence in `row` (whose sequence has ended): enc_mem torch CUDA tensor [ctx, d] of the model dtype."""

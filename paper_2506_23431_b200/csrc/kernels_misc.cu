@@ -28,6 +28,7 @@ __global__ void reset_state_kernel(Dims dm, DecState st, int batch, const int32_
   for (size_t i = gid; i < (size_t)batch * dm.SM; i += stride) {
     st.forced_len[i] = forced_len ? forced_len[i] : -1;
     st.last_tok[i] = dm.bos;
+    st.plan[i] = (int)(i % dm.SM) * dm.dt + 1;          // Eq. 2: s_i = (i-1) delta_t + 1
   }
   for (size_t i = gid; i < (size_t)dm.B * dm.SM * (dm.MSL + 1); i += stride) st.chosen[i] = -1;
   for (size_t i = gid; i < (size_t)dm.B * dm.SM * dm.MSL; i += stride) st.tokens[i] = -1;
@@ -63,6 +64,7 @@ __global__ void admit_row_kernel(Dims dm, DecState st, int b, int ctx_len, const
     const int sidx = b * SM + i;
     st.forced_len[sidx] = forced_len ? forced_len[i] : -1;
     st.last_tok[sidx] = dm.bos;
+    st.plan[sidx] = i * dm.dt + 1;
     st.start[sidx] = i == 0 ? 1 : 0; st.len[sidx] = 0; st.state[sidx] = i == 0 ? SUB_ACTIVE : SUB_NONE; st.flag[sidx] = 0;
   }
   for (int i = tid; i < SM * (dm.MSL + 1); i += n) st.chosen[(size_t)b * SM * (dm.MSL + 1) + i] = -1;

@@ -24,7 +24,7 @@ struct Region { size_t off = 0, bytes = 0; };
 struct Layout {
   // integer state (offsets in int32 words from the start of the state block)
   size_t w_hdr, w_stats, w_k, w_done, w_steps, w_nact, w_ctx, w_ticket, w_start, w_len, w_state, w_flag, w_last,
-      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, w_crow, w_t0, state_words;
+      w_forced, w_row, w_prow, w_rtok, w_ptab, w_tokens, w_chosen, w_trace, w_plist_n, w_xtick, w_crow, w_t0, w_plan, state_words;
   Region state, plist, row_meta, bias_tab, ctx_len_in, forced_in, teacher, dist_bucket, rope_tab, x, hbuf, qkv, qbuf, self_out, cq, cross_out,
       ffn, logits, vpart_val, vpart_idx, vterm, part_o, part_ml, kv_c, kv_scale, kv_pool, enc_stage, proj_stage, cublas_ws;
   size_t total = 0;
@@ -93,7 +93,7 @@ void make_layout(const pd_config &c, const Dims &dm, int max_splits, Layout &L) 
   L.w_t0 = take(B);
   L.w_k = take(B); L.w_done = take(B); L.w_steps = take(B); L.w_nact = take(B); L.w_ctx = take(B); L.w_ticket = take(B);
   L.w_start = take(B * SM); L.w_len = take(B * SM); L.w_state = take(B * SM); L.w_flag = take(B * SM);
-  L.w_last = take(B * SM); L.w_forced = take(B * SM);
+  L.w_last = take(B * SM); L.w_forced = take(B * SM); L.w_plan = take(B * SM);
   L.w_row = take(B * C); L.w_prow = take(B * C); L.w_rtok = take(B * C);
   L.w_ptab = take(B * SM * dm.PPS);
   L.w_tokens = take(B * SM * dm.MSL);
@@ -546,7 +546,7 @@ pd_status pd_init(const pd_config *cfg, const pd_weights *weights, void *workspa
   st.ctx_len = sb + L.w_ctx; st.seq_ticket = sb + L.w_ticket; st.crow = sb + L.w_crow; st.t0 = sb + L.w_t0;
   st.plist_n = sb + L.w_plist_n; st.plist = h->ptr<int4>(L.plist); st.row_meta = h->ptr<int4>(L.row_meta);
   st.start = sb + L.w_start; st.len = sb + L.w_len; st.state = sb + L.w_state; st.flag = sb + L.w_flag;
-  st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced;
+  st.last_tok = sb + L.w_last; st.forced_len = sb + L.w_forced; st.plan = sb + L.w_plan;
   st.row_sub = sb + L.w_row; st.prev_row_sub = sb + L.w_prow; st.row_tok = sb + L.w_rtok;
   st.page_table = sb + L.w_ptab; st.tokens = sb + L.w_tokens; st.chosen = sb + L.w_chosen;
 
@@ -775,6 +775,23 @@ pd_status pd_collect(pd_handle *h, int32_t *tokens, int32_t *lens, int32_t *n_su
   return device_status(h);
 }
 
+pd_status pd_set_start_plan(pd_handle *h, const int32_t *plan) {
+  if (!h || !plan) return PD_ERR_ARG;
+  if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_set_start_plan before pd_encode_context");
+  if (h->steps_enqueued != 0) return fail(h, PD_ERR_STATE, "pd_set_start_plan after the first pd_step");
+  const Dims &dm = h->dm;
+  for (int b = 0; b < h->batch; ++b)
+    for (int i = 0; i < dm.SM; ++i) {
+      const int s_i = plan[b * dm.SM + i];
+      if (i == 0 ? s_i != 1 : s_i - plan[b * dm.SM + i - 1] < dm.dt)
+        return fail(h, PD_ERR_ARG, "pd_set_start_plan: a plan starts at step 1 and its start steps are at least delta_t apart");
+    }
+  CU_TRY(h, cudaSetDevice(h->cfg.device));
+  CU_TRY(h, cudaMemcpyAsync(h->st.plan, plan, (size_t)h->batch * dm.SM * 4, cudaMemcpyHostToDevice, h->stream));
+  CU_TRY(h, cudaStreamSynchronize(h->stream));          // the host array may go
+  return PD_OK;
+}
+
 pd_status pd_admit(pd_handle *h, int32_t row, const void *enc_mem, int32_t ctx_len, const int32_t *forced_len) {
   if (!h) return PD_ERR_ARG;
   if (!h->encoded) return fail(h, PD_ERR_STATE, "pd_admit before pd_encode_context");
@@ -869,8 +886,9 @@ pd_status pd_teacher_forward(pd_handle *h, const int32_t *n_sub, const int32_t *
   if (reinterpret_cast<uintptr_t>(scratch) % kAlign != 0) return fail(h, PD_ERR_ARG, "pd_teacher_forward: misaligned scratch");
   // ---- rows in (sequence, subsequence, position) order; groups of up to 32 rows inside a sequence
   std::vector<int32_t> row_sub, row_tau, row_tok, row_tgt, g_row0, g_n, g_srow0, g_srows, g_seq, g_ctx;
-  std::vector<int32_t> ctx_len(h->batch);
+  std::vector<int32_t> ctx_len(h->batch), plan((size_t)h->batch * dm.SM);
   CU_TRY(h, cudaMemcpyAsync(ctx_len.data(), h->st.ctx_len, (size_t)h->batch * 4, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(h, cudaMemcpyAsync(plan.data(), h->st.plan, plan.size() * 4, cudaMemcpyDeviceToHost, h->stream));
   CU_TRY(h, cudaStreamSynchronize(h->stream));
   for (int b = 0; b < h->batch; ++b) {
     if (n_sub[b] < 0 || n_sub[b] > dm.SM) return fail(h, PD_ERR_ARG, "pd_teacher_forward: n_sub out of range");
@@ -883,11 +901,12 @@ pd_status pd_teacher_forward(pd_handle *h, const int32_t *n_sub, const int32_t *
       for (int p = 0; p <= m; ++p) {
         const int tok = p == 0 ? dm.bos : sub[p - 1], tgt = p < m ? sub[p] : term;
         if (tok < 0 || tok >= dm.V || tgt < 0 || tgt >= dm.V) return fail(h, PD_ERR_ARG, "pd_teacher_forward: token id out of range");
-        row_sub.push_back(i); row_tau.push_back((i - 1) * dm.dt + p); row_tok.push_back(tok); row_tgt.push_back(tgt);
+        row_sub.push_back(i); row_tau.push_back(plan[(size_t)b * dm.SM + i - 1] - 1 + p); row_tok.push_back(tok); row_tgt.push_back(tgt);
       }
     }
     const int srows = (int)row_sub.size() - srow0;
-    if (srows > 0 && (n_sub[b] - 1) * dm.dt + dm.MSL + dm.SM >= dm.n_dist) return fail(h, PD_ERR_ARG, "pd_teacher_forward: positions beyond the tables");
+    if (srows > 0 && plan[(size_t)b * dm.SM + n_sub[b] - 1] - 1 + dm.MSL + dm.SM >= dm.n_dist)
+      return fail(h, PD_ERR_ARG, "pd_teacher_forward: positions beyond the tables");
     for (int r = 0; r < srows; r += kTfGroup) {
       g_row0.push_back(srow0 + r); g_n.push_back(std::min(kTfGroup, srows - r));
       g_srow0.push_back(srow0); g_srows.push_back(srows); g_seq.push_back(b); g_ctx.push_back(ctx_len[b]);

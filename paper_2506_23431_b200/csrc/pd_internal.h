@@ -76,6 +76,7 @@ struct DecState {
   int4 *row_meta;               // [B*C] per row: (page, slot in it, position tau + i) of the entry the coming step appends, subsequence i (0 = unused row)
   int4 *plist;                  // [B][SM*PPS] (page, entries in it, subsequence i', distance base t - (tau' + i') of entry 0)
   int32_t *start, *len, *state, *flag, *last_tok, *forced_len;        // [B*SM]
+  int32_t *plan;                // [B*SM] step (of the sequence's own clock) at which subsequence i is to start; Eq. 2's (i-1) delta_t + 1 unless set
   int32_t *row_sub, *prev_row_sub, *row_tok;                          // [B*C]
   int32_t *page_table;          // [B*SM*PPS]
   int32_t *tokens;              // [B*SM*MSL]

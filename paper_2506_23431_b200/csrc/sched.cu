@@ -22,13 +22,13 @@ __device__ __forceinline__ void better(float &bv, int &bi, float v, int i) {
 // its threads instead.  Indices are local to the sequence: subsequence i at [i - 1], row c at [c].
 struct SeqStage {
   int32_t *row_sub, *row_tok;                                        // [C]
-  int32_t *len, *forced_len, *state, *flag, *start, *last_tok, *teacher;   // [SM]
+  int32_t *len, *forced_len, *state, *flag, *start, *last_tok, *teacher, *plan;   // [SM]
   int32_t *page_table;                                               // [SM * PPS]
   int4 *row_meta;                                                    // [C]
   int4 *plist;                                                       // [SM * PPS]
 };
 __host__ __device__ inline size_t seq_stage_bytes(const Dims &dm) {
-  return ((size_t)(2 * dm.C + 7 * dm.SM + dm.SM * dm.PPS + 3) / 4 * 4) * sizeof(int32_t) + ((size_t)dm.C + (size_t)dm.SM * dm.PPS) * sizeof(int4);
+  return ((size_t)(2 * dm.C + 8 * dm.SM + dm.SM * dm.PPS + 3) / 4 * 4) * sizeof(int32_t) + ((size_t)dm.C + (size_t)dm.SM * dm.PPS) * sizeof(int4);
 }
 
 // Scalars of the sequence that only its own scheduler changes, read at the top of the kernel.
@@ -41,9 +41,9 @@ __device__ __forceinline__ SeqStage seq_stage_views(const Dims &dm, uint8_t *sme
   v.row_sub = w; w += C;
   v.row_tok = w; w += C;
   v.len = w; w += SM; v.forced_len = w; w += SM; v.state = w; w += SM; v.flag = w; w += SM;
-  v.start = w; w += SM; v.last_tok = w; w += SM; v.teacher = w; w += SM;
+  v.start = w; w += SM; v.last_tok = w; w += SM; v.teacher = w; w += SM; v.plan = w; w += SM;
   v.page_table = w; w += NPT;
-  w = reinterpret_cast<int32_t *>(smem) + (size_t)(2 * C + 7 * SM + NPT + 3) / 4 * 4;     // 16-byte aligned
+  w = reinterpret_cast<int32_t *>(smem) + (size_t)(2 * C + 8 * SM + NPT + 3) / 4 * 4;     // 16-byte aligned
   v.row_meta = reinterpret_cast<int4 *>(w);
   v.plist = v.row_meta + C;
   return v;
@@ -64,6 +64,7 @@ __device__ __forceinline__ SeqScalars stage_in(const Dims &dm, const DecState &s
     v.len[i] = st.len[sidx]; v.forced_len[i] = st.forced_len[sidx]; v.state[i] = st.state[sidx]; v.flag[i] = st.flag[sidx];
     v.start[i] = st.start[sidx]; v.last_tok[i] = st.last_tok[sidx];
     v.teacher[i] = teacher != nullptr ? teacher[sidx] : -1;
+    v.plan[i] = st.plan[sidx];
   }
   for (int i = tid; i < NPT; i += nthr) v.page_table[i] = st.page_table[(size_t)b * NPT + i];
   return sc;
@@ -149,7 +150,7 @@ __device__ void schedule_sequence(const Dims &dm, const DecState &st, const SeqS
     done = true;                                   // time_max reached with subsequences still open
     for (int i = lane + 1; i <= k; i += 32)
       if (v.state[i - 1] == SUB_ACTIVE) v.flag[i - 1] |= PD_FLAG_TRUNCATED;
-  } else if (t % dm.dt == 0 && k < SM) {           // step t+1 satisfies (t+1-1) mod delta_t == 0
+  } else if (k < SM && v.plan[k] == t + 1) {       // the next subsequence starts at step t + 1 (Eq. 2: (t+1-1) mod delta_t == 0 unless a plan was set)
     if (lane == 0) {
       st.k[b] = k + 1;
       v.start[k] = t + 1;

@@ -15,13 +15,15 @@ TOL = {"fp32": 1e-4, "bf16": 2e-2}   # max-abs logit error allowed per storage t
 
 
 def oracle_runs(wl: W.Workload, weights, mem_rows: Dict[int, np.ndarray], ctx_len, forced_len,
-                keep_logits: bool = True) -> Dict[int, dict]:
-    """Decode the given batch rows with the oracle (formulation B).  mem_rows: {b: [ctx, d]}."""
+                keep_logits: bool = True, start_plan=None) -> Dict[int, dict]:
+    """Decode the given batch rows with the oracle (formulation B).  mem_rows: {b: [ctx, d]}; start_plan
+    [batch, sub_max] or None (Eq. 2's fixed intervals)."""
     orc = O.PipelinedDecoderOracle(weights, wl.hyper())
     out = {}
     for b, mem in mem_rows.items():
         fl = None if forced_len is None else forced_len[b]
-        out[b] = orc.run(mem, int(ctx_len[b]), fl, keep_logits=keep_logits)
+        plan = None if start_plan is None else [int(x) for x in start_plan[b]]
+        out[b] = orc.run(mem, int(ctx_len[b]), fl, keep_logits=keep_logits, start_plan=plan)
     return out
 
 
@@ -34,7 +36,7 @@ def _margin(logits: np.ndarray, barred: Sequence[int]) -> float:
 
 
 def replay_compare(dec, wl: W.Workload, mem_dev, ctx_len, forced_len, runs: Dict[int, dict],
-                   tol: Optional[float] = None, max_steps: Optional[int] = None, use_logits: bool = True) -> dict:
+                   tol: Optional[float] = None, max_steps: Optional[int] = None, use_logits: bool = True, start_plan=None) -> dict:
     """Teacher-forced replay: the library consumes the oracle's appended tokens on the rows the
     oracle decoded (other rows run free), so every step's logits stay comparable.  Asserts:
     active sets bit-exact, logits within tol, own greedy choice equal where the oracle's margin
@@ -47,6 +49,8 @@ def replay_compare(dec, wl: W.Workload, mem_dev, ctx_len, forced_len, runs: Dict
     tol = TOL[wl.dtype] if tol is None else tol
     hp = wl.hyper()
     dec.encode_context(mem_dev, ctx_len, forced_len)
+    if start_plan is not None:
+        dec.set_start_plan(start_plan)
     batch, sm = dec.batch, wl.sub_max
     t_end = max(r["steps"] for r in runs.values())
     stats = {"max_err": 0.0, "logits": 0, "choices": 0, "low_margin": 0, "steps": 0}

@@ -176,6 +176,62 @@ def test_bf16_one_row_per_sequence_one_sequence_tiny_context(pos_mode):
     dec.close()
 
 
+def uneven_plan(wl, seed):
+    """Start steps at least delta_t apart, with seeded extra gaps (what an adaptive policy might decide)."""
+    g = np.random.Generator(np.random.Philox(key=np.array([seed, 808], dtype=np.uint64)))
+    gaps = wl.delta_t + g.integers(0, 4, size=(wl.batch, wl.sub_max))
+    gaps[:, 0] = 1
+    return np.cumsum(gaps, axis=1).astype(np.int32)
+
+
+@pytest.mark.parametrize("kind", ["bf16_t5", "bf16_rope", "fp32"])
+def test_start_plans_not_at_fixed_intervals(kind):
+    """Subsequences admitted at planned steps instead of every delta_t: the oracle decodes with the same plan; active
+    sets, logits, choices, streams and the trace must agree step by step, and the teacher-forced forward must use the
+    plan's timestamps too."""
+    if kind == "fp32":
+        wl = TINY.scaled(batch=2, ctx=64, sub_max=4, delta_t=2, max_sub_len=9, length_dist=("uniform", 2, 9), time_max=60,
+                         vocab=300, norm_gain_std=0.1)
+    else:
+        wl = W.CONFIGS["bart_base"].scaled(name="plan", batch=3, ctx=150, sub_max=6, delta_t=2, max_sub_len=24,
+                                           length_dist=("uniform", 1, 24), time_max=90,
+                                           pos_mode=W.POS_T5_BIAS if kind == "bf16_t5" else W.POS_ROPE, **SMALL_BF16)
+    weights, mem, ctx_len, dec, rows = make(wl, ragged=True)
+    fl = W.make_forced_len(wl)
+    plan = uneven_plan(wl, 3)
+    assert (np.diff(plan, axis=1) >= wl.delta_t).all() and (np.diff(plan, axis=1) > wl.delta_t).any()
+    runs = parity.oracle_runs(wl, weights, {b: mem[b] for b in rows}, ctx_len, fl, start_plan=plan)
+    assert all(r["starts"] == plan[b, :r["n_sub"]].tolist() for b, r in runs.items())
+    mem_dev = dec.device_memory(mem)
+    s = parity.replay_compare(dec, wl, mem_dev, ctx_len, fl, runs, start_plan=plan)
+    assert s["choices"] > 0
+    # the fixed plan comes back with the next pd_encode_context
+    base = parity.oracle_runs(wl, weights, {0: mem[0]}, ctx_len, fl)
+    parity.replay_compare(dec, wl, mem_dev, ctx_len, fl, base)
+    if kind != "fp32":
+        from oracle import pipelined_decoder as O
+        dec.encode_context(mem_dev, ctx_len, fl)
+        dec.set_start_plan(plan)
+        subs = [runs[b]["subsequences"] for b in range(wl.batch)]
+        lp, loss, logits = dec.teacher_forward(subs, want_logits=True)
+        ref = O.PipelinedDecoderOracle(weights, wl.hyper()).teacher_forward(mem[0], int(ctx_len[0]), subs[0],
+                                                                           start_plan=plan[0, :len(subs[0])].tolist())
+        got = logits[:len(ref["rows"])].cpu().numpy().astype(np.float64)
+        assert np.abs(got - ref["logits"]).max() <= 2e-2
+    # plans the workspace is not sized for are refused
+    from paper_2506_23431_b200.binding import PdError
+    dec.encode_context(mem_dev, ctx_len, fl)
+    bad = plan.copy(); bad[0, 1] = bad[0, 0] + wl.delta_t - 1
+    with pytest.raises(PdError) as e:
+        dec.set_start_plan(bad)
+    assert e.value.status == -1
+    dec.step()
+    with pytest.raises(PdError) as e:
+        dec.set_start_plan(plan)
+    assert e.value.status == -2
+    dec.close()
+
+
 def test_steps_after_the_end_are_no_ops():
     from paper_2506_23431_b200.binding import PipelinedDecoder
     wl = TINY.scaled(vocab=300)
