@@ -301,8 +301,16 @@ bool make_ff_plan(pd_handle *h, int M, int N, int K) {
   } while (0)
 
 bool self_tc(const pd_handle *h) { return h->cfg.dtype == PD_DTYPE_BF16 && self_attn_tc_supported(h->dm); }
-// Nothing to rotate: the projection rounds to bf16 itself and the attention kernel places the new cache entries.
-bool fused_append(const pd_handle *h) { return self_tc(h) && h->dm.pos_mode != PD_POS_ROPE; }
+// The tensor-core attention kernel places the new cache entries itself: from the projection's bf16 output when
+// nothing is rotated (1), from its fp32 output, rotating queries and keys first, in rotary mode (2).
+// In rotary mode the fused form pays one more dependent fetch for every page that receives a new entry, which is
+// most pages when a subsequence fits one page (measured on the keyphrase shape: 20.6 us against 16.7 + 2.0 us for the
+// append launch); there the append kernel stays.
+int fused_append(const pd_handle *h) {
+  if (!self_tc(h)) return 0;
+  if (h->dm.pos_mode != PD_POS_ROPE) return 1;
+  return h->dm.PPS >= 2 ? 2 : 0;
+}
 
 AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   AttnArgs a;
@@ -319,7 +327,8 @@ AttnArgs attn_args(pd_handle *h, int layer, bool self) {
   a.tickets = h->ptr<int32_t>(h->lay.state) + h->lay.w_xtick;
   a.bias_tab = h->cfg.pos_mode == PD_POS_T5_BIAS ? h->ptr<float>(h->lay.bias_tab) : nullptr;
   a.qkv = h->ptr<void>(h->lay.qkv);
-  a.fused_append = self && fused_append(h) ? 1 : 0;
+  a.fused_append = self ? fused_append(h) : 0;
+  a.rope_tab = h->ptr<float2>(h->lay.rope_tab);
   a.kv_scale = (!self && h->kv8) ? h->ptr<float>(h->lay.kv_scale) : nullptr;
   a.kv_seq = nullptr; a.row_base = nullptr;
   return a;
@@ -373,10 +382,10 @@ pd_status enqueue_step(pd_handle *h) {
   for (int l = 0; l < dm.L; ++l) {
     const void *const *lw = &h->layer_w[(size_t)l * kLayerTensors];
     if (l > 0) OWN(h, PD_PROF_OTHER, launch_rmsnorm(dm, M, dt, x, lw[0], hb, s));
-    if (fused_append(h)) {
-      // the attention kernel takes queries, keys and values straight from the projection's bf16 output and
-      // appends the new cache entries itself
-      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, false, 0.f));
+    if (fused_append(h) != 0) {
+      // the attention kernel takes queries, keys and values straight from the projection's output (bf16, or fp32
+      // where it has to rotate them) and appends the new cache entries itself
+      PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, fused_append(h) == 2, 0.f));
     } else if (dt == PD_DTYPE_BF16 && dm.pos_mode != PD_POS_ROPE) {
       // nothing to rotate: the projection rounds to bf16 itself and the append only places the rows
       PD_TRY(gemm(h, false, M, 3 * dm.d, dm.d, hb, lw[1], qkv, false, 0.f));

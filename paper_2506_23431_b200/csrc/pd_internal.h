@@ -99,10 +99,11 @@ struct AttnArgs {
   int rel_buckets;
   const float *bias_tab;       // [H, n_dist]: rel_bias[h][bucket(dist)] * log2(e), or null
   int32_t *tickets;            // one arrival counter per (sequence, head), zero between launches
-  // tensor-core self-attention with the step's KV-append inside it (fused_append): the projection's
-  // output [rows][3 d] in bf16
+  // tensor-core self-attention with the step's KV-append inside it: the projection's output [rows][3 d] in
+  // bf16 (fused_append = 1) or in fp32, to be rotated with rope_tab (fused_append = 2); 0 = the append kernel ran
   const void *qkv;
   int fused_append;
+  const float2 *rope_tab;
   // cross-attention over 8-bit keys/values: [layer][sequence][head][keys | values] fp32 scales (else null)
   const float *kv_scale;
   // cross-attention over row groups that are not one per sequence (the teacher-forced forward: many rows per

@@ -26,8 +26,11 @@
 // head straight from the projection's output into its ring slot (asynchronously, like the rest of
 // the page) and, once they have landed, on into the cache - every (page, head) block is met by
 // exactly one warp of the launch, so the cache is written once, without a race, and no separate
-// append launch exists.  Queries come from the same projection output.  In rotary mode the append
-// kernel rotates queries and keys first and this kernel reads the cache alone.
+// append launch exists.  Queries come from the same projection output.  In rotary mode the
+// projection's output is fp32 and has to be rotated: the CTA's warps first rotate and round the rows'
+// new keys (and values) of this head into the cache, each warp rotates its query fragments, and after
+// the CTA's barrier the new entries are fetched from the cache like any other (everything that needs a
+// dependent load happens once, in the prologue, never inside the page walk).
 //
 // Splits: the number of splits in use follows the list's length (a CTA whose split is not needed
 // leaves at once).  Warps merge through shared memory; split CTAs leave a partial record, take a
@@ -103,11 +106,12 @@ __host__ __device__ constexpr int self_attn_tc_ring_bytes(int P, int mt) {
                                                                                       : SW * 16 * mt * (SMROW + 2) * 4;
 }
 
-// MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens; FUSED = the launch appends the
-// step's keys/values itself (queries, keys, values in a.qkv) instead of following the append kernel (queries in a.q)
+// MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens; MODE 0 = the launch follows the append
+// kernel (queries in a.q); 1 = it appends the step's keys/values itself from the projection's bf16 output a.qkv;
+// 2 = the same from an fp32 output that it rotates by the rows' positions first (rotary mode)
 // OCC = CTAs per SM the register budget is set for: four leave the compiler 128 registers (nothing spills),
 // five 96 (more CTAs resident, which wins when there are more (sequence, head) pairs than four per SM)
-template <int MT, int P, bool FUSED, int OCC>
+template <int MT, int P, int MODE, int OCC>
 __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kernel(AttnArgs a) {
   constexpr int BK = P > SKEYS ? P : SKEYS; // keys per batch
   constexpr int PB = BK / P;               // pages per batch
@@ -147,7 +151,8 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   int my_rsub = 0;
   if (tid < dm.C) my_rsub = a.st.row_sub[row0 + tid];
   // (page, slot, position tau + i, subsequence) of the entry row `lane` of this sequence appends at this step
-  const int4 meta = (FUSED && lane < dm.C) ? a.st.row_meta[row0 + lane] : make_int4(-1, 0, 0, 0);
+  constexpr bool FUSED = MODE == 1;
+  const int4 meta = (MODE != 0 && lane < dm.C) ? a.st.row_meta[row0 + lane] : make_int4(-1, 0, 0, 0);
   const bool use_bias = a.bias_tab != nullptr;
   float my_bias[SBIAS_PER_THREAD];
 #pragma unroll
@@ -165,6 +170,7 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
     const __nv_bfloat16 *q_hi = qsrc + (size_t)(row0 + r_hi) * qstride + h * kDh + 2 * tig;
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
+      if (MODE == 2) continue;               // rotary mode: loaded as fp32 and rotated below, once the rows' positions are known
       qf[mt][kk][0] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
       qf[mt][kk][1] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
       qf[mt][kk][2] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
@@ -183,18 +189,77 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   }
   if (split >= n_eff) return;
 
+  const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
+  const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
+  if (MODE == 2) {
+    const float *qkv32 = reinterpret_cast<const float *>(a.qkv);
+    // (a) the rows' new entries: warp w takes rows w, w + SW, ...; lane l columns 2 l, 2 l + 1 of the key (rotated by the
+    // row's position) and of the value, rounded to bf16 and written to the row's cache slot.  All loads first.
+    {
+      float2 kf[(16 * MT + SW - 1) / SW], vf[(16 * MT + SW - 1) / SW], cs[(16 * MT + SW - 1) / SW];
+#pragma unroll
+      for (int j = 0; j < (16 * MT + SW - 1) / SW; ++j) {
+        const int c = warp + j * SW;
+        if (c < S) {
+          const int pos = __shfl_sync(0xffffffffu, meta.z, c);
+          const float *src = qkv32 + (size_t)(row0 + c) * 3 * dm.d + dm.d + (size_t)h * kDh + 2 * lane;
+          kf[j] = *reinterpret_cast<const float2 *>(src);
+          vf[j] = *reinterpret_cast<const float2 *>(src + dm.d);
+          cs[j] = a.rope_tab[(size_t)pos * (kDh / 2) + lane];
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < (16 * MT + SW - 1) / SW; ++j) {
+        const int c = warp + j * SW;
+        if (c < S) {
+          const int page = __shfl_sync(0xffffffffu, meta.x, c), slot = __shfl_sync(0xffffffffu, meta.y, c);
+          const float kx = kf[j].x * cs[j].x - kf[j].y * cs[j].y, ky = kf[j].x * cs[j].y + kf[j].y * cs[j].x;
+          __nv_bfloat16 *cache = const_cast<__nv_bfloat16 *>(pool_lh) + page * page_stride + kv_entry_offset<__nv_bfloat16>(slot, 2 * lane, 0);
+          *reinterpret_cast<uint32_t *>(cache) = s_pack_bf16(kx, ky);
+          *reinterpret_cast<uint32_t *>(cache + kDh) = s_pack_bf16(vf[j].x, vf[j].y);   // the value row follows the key row of the same entry
+        }
+      }
+    }
+    // (b) this warp's query fragments, rotated likewise
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int r = mt * 16 + g + 8 * hh;
+        const int pos = __shfl_sync(0xffffffffu, meta.z, r & 31);
+        float2 v[8], c2[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {         // columns kk * 16 + 2 tig (+ 8): j = 2 kk + half
+          const int col = (j >> 1) * 16 + 2 * tig + (j & 1) * 8;
+          v[j] = make_float2(0.f, 0.f); c2[j] = make_float2(1.f, 0.f);
+          if (r < S) {
+            v[j] = *reinterpret_cast<const float2 *>(qkv32 + (size_t)(row0 + r) * 3 * dm.d + (size_t)h * kDh + col);
+            c2[j] = a.rope_tab[(size_t)pos * (kDh / 2) + col / 2];
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          qf[mt][j >> 1][hh + 2 * (j & 1)] = s_pack_bf16(v[j].x * c2[j].x - v[j].y * c2[j].y, v[j].x * c2[j].y + v[j].y * c2[j].x);
+      }
+    }
+  }
+
   const int W = n_eff * SW;
   const int n_mine = n_batches > g0 ? (n_batches - g0 + W - 1) / W : 0;
   const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SSLOT;
-  const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
-  const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
 
   // One page of a batch: the entries the cache holds are copied; if a row appends to this page at this step
   // (its entry is the page's last), that entry comes from the projection's output: 8 + 8 chunks of 16 bytes.
-  auto fetch_page = [&](uint32_t dst, int4 e) {
+  // (`early`: before the CTA's barrier.  In rotary mode a new entry is then still on its way into the cache: the
+  // entries before it are copied, the entry itself after the barrier.)
+  auto fetch_page = [&](uint32_t dst, int4 e, bool early) {
     if (e.y <= 0) return;
     const __nv_bfloat16 *blk = pool_lh + e.x * page_stride;
     int n_copy = e.y;
+    if (MODE == 2 && early) {
+      const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
+      if (hit != 0u) n_copy = __shfl_sync(0xffffffffu, meta.y, __ffs(hit) - 1);
+    }
     if (FUSED) {
       const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
       if (hit != 0u) {
@@ -212,23 +277,23 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   };
   // batch n of this warp = list entries PB * (g0 + n W) ...; `list` = the list in global memory (before the
   // CTA's copy is complete) or in shared memory
-  auto fetch = [&](int n, const int4 *list) {
+  auto fetch = [&](int n, const int4 *list, bool early) {
     const int first = PB * (g0 + n * W);
     const uint32_t dst = my_ring + (n & 1) * SSLOT;
 #pragma unroll
     for (int pb = 0; pb < PB; ++pb) {
       const int4 e = first + pb < n_list ? list[first + pb] : make_int4(0, 0, 0, 0);
-      fetch_page(dst + pb * P * 256, e);
+      fetch_page(dst + pb * P * 256, e, early);
     }
   };
   // Nothing is ever cleared: what a slot holds beyond a page's entries (anything) gets score -inf, and
   // the value fragments of those keys are zeroed in registers after ldmatrix.
   if (n_mine > 0) {
 #pragma unroll
-    for (int pb = 0; pb < PB; ++pb) fetch_page(my_ring + pb * P * 256, PB * g0 + pb < n_list ? e_first[pb] : make_int4(0, 0, 0, 0));
+    for (int pb = 0; pb < PB; ++pb) fetch_page(my_ring + pb * P * 256, PB * g0 + pb < n_list ? e_first[pb] : make_int4(0, 0, 0, 0), true);
   }
   s_cp_async_commit();
-  if (n_mine > 1) fetch(1, pl);
+  if (n_mine > 1) fetch(1, pl, true);
   s_cp_async_commit();
   if (tid < list_cap) plist_s[tid] = my_entry;
   for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
@@ -237,6 +302,27 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   for (int k = 0; k < SBIAS_PER_THREAD; ++k)
     if (use_bias && k * STHREADS + tid < dm.n_dist) bias_s[k * STHREADS + tid] = my_bias[k];
   __syncthreads();
+  if (MODE == 2) {
+    // the new entries are in the cache now (written by this CTA's warps before the barrier): those of the two batches
+    // already on their way follow them into the ring
+    for (int n = 0; n < 2 && n < n_mine; ++n) {
+#pragma unroll
+      for (int pb = 0; pb < PB; ++pb) {
+        const int idx = PB * (g0 + n * W) + pb;
+        const int4 e = idx < n_list ? plist_s[idx] : make_int4(0, 0, 0, 0);
+        const unsigned hit = __ballot_sync(0xffffffffu, e.y > 0 && lane < S && meta.x == e.x);
+        if (hit != 0u) {
+          const int slot = __shfl_sync(0xffffffffu, meta.y, __ffs(hit) - 1);
+          if (lane < 16) {
+            const uint32_t off = s_swz(slot, lane & 7) + (lane < 8 ? 0u : 128u);
+            s_cp_async16(my_ring + (n & 1) * SSLOT + pb * P * 256 + off,
+                         reinterpret_cast<const uint8_t *>(pool_lh + e.x * page_stride) + off);
+          }
+        }
+      }
+    }
+    s_cp_async_commit();
+  }
 
   int rs[MT][2];                     // subsequence of rows g and g + 8 of every query tile
   int tile_last[MT];                 // subsequence of the tile's last active row (rows are sorted)
@@ -259,7 +345,8 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   const float sl2 = dm.scale_log2e;
 
   for (int n = 0; n < n_mine; ++n) {
-    s_cp_async_wait<1>();              // everything but the newest group has landed: batch n is in its slot
+    if (MODE == 2 && n == 0) s_cp_async_wait<0>();     // the first batches' new entries were requested last
+    else s_cp_async_wait<1>();         // everything but the newest group has landed: batch n is in its slot
     __syncwarp();                      // (and the appended entries the lanes stored themselves are visible)
     // per page of the batch: entries that exist, subsequence, distance base of its first entry
     int nv[PB], ksub[PB], d0[PB];
@@ -415,7 +502,7 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
       }
     }
     __syncwarp();   // every lane is done reading the slot
-    if (n + 2 < n_mine) fetch(n + 2, plist_s);
+    if (n + 2 < n_mine) fetch(n + 2, plist_s, false);
     s_cp_async_commit();
   }
   s_cp_async_wait<0>();
@@ -551,10 +638,12 @@ int self_attn_tc_splits(const Dims &dm, int pairs, int sms) {
 template <int MT, int P>
 static cudaError_t prepare_one() {
   const int smem = self_attn_tc_max_smem(P, MT);
-  cudaError_t e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, false, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, true, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaError_t e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 0, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 0, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 2, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   return e;
 }
 
@@ -566,8 +655,8 @@ cudaError_t self_attn_tc_prepare() {
   return e;
 }
 
-// a.fused_append: a.qkv = the projection's output [rows][3 d] in bf16 (else a.q = the queries the append
-// kernel left), a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed), a.part_o /
+// a.fused_append 1: a.qkv = the projection's output [rows][3 d] in bf16; 2: in fp32, rotated here with a.rope_tab;
+// 0: a.q = the queries the append kernel left.  a.tickets one zeroed int32 per (sequence, head) (the kernel leaves them zeroed), a.part_o /
 // a.part_ml sized for a.splits records per (row, head).
 cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s) {
   dim3 grid(a.splits, a.dm.H, a.batch);
@@ -578,10 +667,12 @@ cudaError_t launch_self_attn_tc(const AttnArgs &a, cudaStream_t s) {
   const bool roomy = (long long)a.splits * a.dm.H * a.batch <= 4LL * sms;      // all CTAs resident at four per SM
 #define PD_SELF_LAUNCH(MT_, P_)                                                                            \
   do {                                                                                                   \
-    if (a.fused_append && roomy) self_attn_tc_kernel<MT_, P_, true, 4><<<grid, STHREADS, smem, s>>>(a);   \
-    else if (a.fused_append) self_attn_tc_kernel<MT_, P_, true, 5><<<grid, STHREADS, smem, s>>>(a);       \
-    else if (roomy) self_attn_tc_kernel<MT_, P_, false, 4><<<grid, STHREADS, smem, s>>>(a);               \
-    else self_attn_tc_kernel<MT_, P_, false, 5><<<grid, STHREADS, smem, s>>>(a);                          \
+    if (a.fused_append == 1 && roomy) self_attn_tc_kernel<MT_, P_, 1, 4><<<grid, STHREADS, smem, s>>>(a);        \
+    else if (a.fused_append == 1) self_attn_tc_kernel<MT_, P_, 1, 5><<<grid, STHREADS, smem, s>>>(a);            \
+    else if (a.fused_append == 2 && roomy) self_attn_tc_kernel<MT_, P_, 2, 4><<<grid, STHREADS, smem, s>>>(a);   \
+    else if (a.fused_append == 2) self_attn_tc_kernel<MT_, P_, 2, 5><<<grid, STHREADS, smem, s>>>(a);            \
+    else if (roomy) self_attn_tc_kernel<MT_, P_, 0, 4><<<grid, STHREADS, smem, s>>>(a);                          \
+    else self_attn_tc_kernel<MT_, P_, 0, 5><<<grid, STHREADS, smem, s>>>(a);                                     \
   } while (0)
   if (mt == 1 && a.dm.P == 16) PD_SELF_LAUNCH(1, 16);
   else if (mt == 2 && a.dm.P == 16) PD_SELF_LAUNCH(2, 16);
