@@ -110,3 +110,18 @@ def test_rows_per_sequence_bound():
                 worst = max(worst, n)
         assert worst <= rows
     assert min(32, 8 // 1 + 1) == 9          # keyphrase config: 9 rows per sequence, not 32
+
+
+def test_pure_host_helpers_of_the_stand_alone_ops():
+    """Sizing helpers that need no GPU: the projection kernel's tile plan (the number of partial sums-of-squares it
+    writes = column slices x CTAs along K), scratch sizes, and their refusals."""
+    lib = B._lib
+    assert lib.pd_linear_sumsq_parts(1024, 1024) == 128          # 16 slices of 64 columns x 8 CTAs along K
+    assert lib.pd_linear_sumsq_parts(4096, 1024) == 128
+    assert lib.pd_linear_sumsq_parts(1024, 4096) > 0 and lib.pd_linear_sumsq_parts(768, 2304) > 0
+    assert lib.pd_linear_sumsq_parts(96, 64) == 0 and lib.pd_linear_sumsq_parts(64, 8) == 0     # d_in % 64, d_out % 16
+    assert lib.pd_linear_scratch_bytes(1024, 1024) >= 1024 * 1024 * 2 and lib.pd_linear_scratch_bytes(96, 64) == 0
+    assert lib.pd_vocab_argmax_scratch_bytes(128, 32128) > 0
+    assert lib.pd_cross_attention_scratch_bytes(4, 16, 8, 2) > 0 and lib.pd_cross_attention_scratch_bytes(4, 65, 8, 2) == 0
+    assert lib.pd_teacher_forward_scratch_bytes(None, 100, 1) == 0
+    assert lib.pd_cross_attention_static_max_bytes() == 8 << 20
