@@ -1,7 +1,7 @@
 // Pipelined self-attention for bf16 storage (sm_100a): decode attention of all active
 // subsequences of a sequence over the paged per-subsequence KV cache, with the dependency rule
 // of Section 3.2 (a query of subsequence i sees subsequences i' <= i as generated so far)
-// evaluated per page from (subsequence, first position) metadata - no mask is ever stored -
+// evaluated per key from (subsequence, position) metadata - no mask is ever stored -
 // and the step's KV-append with its positional write (Eq. 2: the entry's position is tau + i)
 // done by the same launch.
 //
@@ -10,29 +10,25 @@
 // up with HBM, so scores and P.V run on tensor cores (mma.sync m16n8k16, bf16 in, fp32
 // accumulate) with the visibility rule and the T5 bias applied to the accumulator fragment.
 //
-// The scheduler leaves, once per step, a list of the sequence's pages (page, entries, subsequence,
-// first position) that every layer and head reuses.  One CTA = one (split, head, sequence); each of
-// its warps is an independent worker that takes every W-th BATCH of the list (32 keys: two 16-token
-// pages, or one 32-token page; W = splits in use * warps), copies exactly the entries that exist -
-// one contiguous run per page, key row and value row per entry - into its private two-slot ring
-// with 16-byte cp.async and runs scores, softmax and P.V over the whole batch at once (twice the
-// independent tensor-core work per dependent chain of a single page).  Pages are stored
-// pre-swizzled (16-byte chunk c of a row of entry e at chunk c ^ (e & 7)), so a linear copy lands
-// in the bank-conflict-free layout ldmatrix wants.
+// What a launch costs is set by the number of iterations of its busiest warp, and an iteration costs
+// the same whether its 16 key slots are full or not.  Pages are per subsequence, so most of a sequence's
+// pages are partly filled (a 21-entry subsequence holds two pages): walking pages made a warp do up to
+// three times the iterations its keys needed.  The kernel therefore walks KEYS: from the page list the
+// scheduler leaves once per step (page, entries, subsequence, first position) the CTA builds, in shared
+// memory, the flat list of the entries that exist - where each lies (page, slot), its subsequence and
+// its distance base - and its warps take tiles of 16 consecutive keys of that list, whatever pages
+// they come from.  A tile is gathered into the warp's private two-slot ring with 16-byte cp.async
+// (the cache rows are stored pre-swizzled by their slot; the copy re-swizzles them by their place in
+// the tile, so that ldmatrix reads without bank conflicts); one CTA = one (split, head, sequence).
 //
-// Fused append (when nothing has to be rotated, i.e. with the T5 bias; the projection then writes
-// bf16 itself): the entry a row feeds at this step is the last one of its subsequence's last page
-// and is not in the cache yet.  The warp that meets that page copies the row's key and value of this
-// head straight from the projection's output into its ring slot (asynchronously, like the rest of
-// the page) and, once they have landed, on into the cache - every (page, head) block is met by
-// exactly one warp of the launch, so the cache is written once, without a race, and no separate
-// append launch exists.  Queries come from the same projection output.  In rotary mode the
-// projection's output is fp32 and has to be rotated: the CTA's warps first rotate and round the rows'
-// new keys (and values) of this head into the cache, each warp rotates its query fragments, and after
-// the CTA's barrier the new entries are fetched from the cache like any other (everything that needs a
-// dependent load happens once, in the prologue, never inside the page walk).
+// Fused append: the entries the rows feed at this step are written to the cache by the same launch,
+// in its prologue: warp w takes rows w, w + 4, ...; their keys and values of this head come straight from
+// the projection's output (bf16 when nothing is rotated; fp32, rotated by the position tau + i and
+// rounded, in rotary mode), requested in the first round of loads and stored once the rows' slots are
+// known.  After the CTA's barrier they are cache entries like any other.  Queries come from the same
+// projection output (rotated likewise).  Split CTAs of one (sequence, head) write the same bits.
 //
-// Splits: the number of splits in use follows the list's length (a CTA whose split is not needed
+// Splits: the number of splits in use follows the key list's length (a CTA whose split is not needed
 // leaves at once).  Warps merge through shared memory; split CTAs leave a partial record, take a
 // ticket, and the last one to arrive merges the records in split order (deterministic) and writes
 // the output - no merge launch, and no CTA ever waits for another.
@@ -42,14 +38,15 @@ namespace pd {
 
 constexpr int SW = 4;                      // worker warps per CTA
 constexpr int STHREADS = SW * 32;
-constexpr int SDEPTH = 2;                  // ring slots per warp: the batch in use and the next one
-constexpr int SKEYS = 16;                  // keys per batch: one 16-token page (a 32-token page is a batch of its own)
+constexpr int SDEPTH = 2;                  // ring slots per warp: the tile in use and the next one
+constexpr int STK = 16;                    // keys per tile
+constexpr uint32_t SSLOT = STK * 256u;     // keys + values of one tile of one head (4 KB)
 constexpr int SMAXLIST = 256;              // page-list entries of one sequence held in shared memory
 constexpr int SMAXDIST = 512;
 constexpr int SMROW = kDh + 8;             // row stride of the merge scratch in floats (spreads the eight fragment rows over the banks)
-// Pages a warp walks before another split is used: a page costs a warp ~0.75 us, a split ~4 us of fixed cost
-// (partial records, fence, ticket, the last CTA's read-back), so a split pays once it saves about six pages per warp.
-constexpr int SBATCHES_PER_WARP = 10;
+// Tiles a warp walks before another split is used: a tile costs a warp ~0.75 us, a split ~4 us of fixed cost
+// (partial records, fence, ticket, the last CTA's read-back), so a split pays once it saves about six tiles per warp.
+constexpr int STILES_PER_WARP = 10;
 constexpr int SBIAS_PER_THREAD = (SMAXDIST + STHREADS - 1) / STHREADS;
 
 __device__ __forceinline__ uint32_t s_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -89,21 +86,9 @@ __device__ __forceinline__ uint32_t s_pack_bf16(float lo, float hi) {
 // swizzle phase (row & 7) of an entry is the same in the slot as in its page.
 __device__ __forceinline__ uint32_t s_swz(int row, int chunk) { return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4)); }
 
-// All lanes: copy the first n entries of one (page, head) block - n * 256 contiguous bytes, key row
-// then value row per entry - to `dst`.
-template <int P>
-__device__ __forceinline__ void s_fetch_run(uint32_t dst, const __nv_bfloat16 *blk, int n, int lane) {
-  const uint8_t *src = reinterpret_cast<const uint8_t *>(blk) + lane * 16;
-  const int nchunks = n * 16;                    // 16-byte chunks of the run
-#pragma unroll
-  for (int k = 0; k < P / 2; ++k)                // P * 16 chunks over 32 lanes
-    if (k * 32 + lane < nchunks) s_cp_async16(dst + lane * 16 + k * 512, src + k * 512);
-}
-
 // Bytes of the rings (or of the merge scratch that reuses them, whichever is larger).
-__host__ __device__ constexpr int self_attn_tc_ring_bytes(int P, int mt) {
-  return SW * SDEPTH * (P > SKEYS ? P : SKEYS) * 256 > SW * 16 * mt * (SMROW + 2) * 4 ? SW * SDEPTH * (P > SKEYS ? P : SKEYS) * 256
-                                                                                      : SW * 16 * mt * (SMROW + 2) * 4;
+__host__ __device__ constexpr int self_attn_tc_ring_bytes(int mt) {
+  return SW * SDEPTH * (int)SSLOT > SW * 16 * mt * (SMROW + 2) * 4 ? SW * SDEPTH * (int)SSLOT : SW * 16 * mt * (SMROW + 2) * 4;
 }
 
 // MT = 16-row query tiles (rows per sequence <= 16 * MT); P = page_tokens; MODE 0 = the launch follows the append
@@ -113,16 +98,12 @@ __host__ __device__ constexpr int self_attn_tc_ring_bytes(int P, int mt) {
 // five 96 (more CTAs resident, which wins when there are more (sequence, head) pairs than four per SM)
 template <int MT, int P, int MODE, int OCC>
 __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kernel(AttnArgs a) {
-  constexpr int BK = P > SKEYS ? P : SKEYS; // keys per batch
-  constexpr int PB = BK / P;               // pages per batch
-  constexpr int NT = BK / 8;               // 8-key score tiles per batch
-  constexpr int KS = BK / 16;              // 16-key steps of P.V per batch
-  constexpr uint32_t SSLOT = BK * 256u;    // keys + values of one batch of one head
-  // dynamic shared memory: the warps' rings (reused as merge scratch), then the sequence's page list
-  // (page, entries, subsequence i', distance base of entry 0), then this head's bias row
+  // dynamic shared memory: the warps' rings (reused as merge scratch), the sequence's page list, the exclusive
+  // prefix of its entry counts, the flat key list (where the key lies; its subsequence and distance base), and
+  // this head's bias row
   extern __shared__ __align__(128) uint8_t s_ring_raw[];
   __shared__ int rsub_s[16 * MT];          // subsequence of row r
-  __shared__ int last_s;
+  __shared__ int last_s, n_keys_s;
 
   const Dims &dm = a.dm;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -130,28 +111,25 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   const int row0 = b * dm.C;
   __nv_bfloat16 *out = (__nv_bfloat16 *)a.out;
   const int g = lane >> 2, tig = lane & 3;
+  const int list_cap = dm.SM * dm.PPS;
+  int4 *plist_s = reinterpret_cast<int4 *>(s_ring_raw + self_attn_tc_ring_bytes(MT));
+  int *off_s = reinterpret_cast<int *>(plist_s + list_cap);                  // [list_cap + 1]
+  int2 *key_s = reinterpret_cast<int2 *>(off_s + ((list_cap + 1 + 1) & ~1));   // [list_cap * P]: (page * 32 + slot, subsequence | (distance base + 1024) << 8)
+  float *bias_s = reinterpret_cast<float *>(key_s + (size_t)list_cap * P);
 
-  // ---- ONE round of independent global loads, none waiting for another: active-row count, page
-  // list (first STHREADS entries), row -> subsequence, where every row's new entry goes, bias row of
-  // this head, query fragments.  What turns out to be unused (rows beyond the active ones) is masked afterwards.
+  // ---- ONE round of independent global loads, none waiting for another: active-row count, page list, row ->
+  // subsequence, where every row's new entry goes, bias row of this head, query fragments, and (fused modes) the
+  // new keys/values of the rows this warp appends.  What turns out to be unused is masked afterwards.
   const int S = a.st.n_active[b];
   const int n_list = a.st.plist_n[b];
-  const int list_cap = dm.SM * dm.PPS;
   const int4 *pl = a.st.plist + (size_t)b * list_cap;
-  int4 *plist_s = reinterpret_cast<int4 *>(s_ring_raw + self_attn_tc_ring_bytes(P, MT));
-  float *bias_s = reinterpret_cast<float *>(plist_s + list_cap);
-  int4 my_entry = make_int4(0, 0, 0, 0);
-  if (tid < list_cap) my_entry = pl[tid];
-  // the entries of this warp's first batch, so that its copies can start before the CTA has assembled
-  // the list in shared memory (its index does not depend on how many splits are in use)
-  const int g0 = split * SW + warp;
-  int4 e_first[PB];
+  int4 my_entry[(SMAXLIST + STHREADS - 1) / STHREADS];
 #pragma unroll
-  for (int pb = 0; pb < PB; ++pb) e_first[pb] = PB * g0 + pb < list_cap ? pl[PB * g0 + pb] : make_int4(0, 0, 0, 0);
+  for (int k = 0; k < (SMAXLIST + STHREADS - 1) / STHREADS; ++k)
+    my_entry[k] = k * STHREADS + tid < list_cap ? pl[k * STHREADS + tid] : make_int4(0, 0, 0, 0);
   int my_rsub = 0;
   if (tid < dm.C) my_rsub = a.st.row_sub[row0 + tid];
   // (page, slot, position tau + i, subsequence) of the entry row `lane` of this sequence appends at this step
-  constexpr bool FUSED = MODE == 1;
   const int4 meta = (MODE != 0 && lane < dm.C) ? a.st.row_meta[row0 + lane] : make_int4(-1, 0, 0, 0);
   const bool use_bias = a.bias_tab != nullptr;
   float my_bias[SBIAS_PER_THREAD];
@@ -160,67 +138,74 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
     const int dd = k * STHREADS + tid;
     my_bias[k] = (use_bias && dd < dm.n_dist) ? a.bias_tab[h * dm.n_dist + dd] : 0.f;
   }
-  const __nv_bfloat16 *qsrc = FUSED ? (const __nv_bfloat16 *)a.qkv : (const __nv_bfloat16 *)a.q;
-  const size_t qstride = FUSED ? 3 * (size_t)dm.d : (size_t)dm.d;
   uint32_t qf[MT][4][4];
+  if (MODE != 2) {
+    const __nv_bfloat16 *qsrc = MODE == 1 ? (const __nv_bfloat16 *)a.qkv : (const __nv_bfloat16 *)a.q;
+    const size_t qstride = MODE == 1 ? 3 * (size_t)dm.d : (size_t)dm.d;
 #pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
-    const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
-    const __nv_bfloat16 *q_lo = qsrc + (size_t)(row0 + r_lo) * qstride + h * kDh + 2 * tig;
-    const __nv_bfloat16 *q_hi = qsrc + (size_t)(row0 + r_hi) * qstride + h * kDh + 2 * tig;
+    for (int mt = 0; mt < MT; ++mt) {
+      const int r_lo = mt * 16 + g, r_hi = r_lo + 8;
+      const __nv_bfloat16 *q_lo = qsrc + (size_t)(row0 + r_lo) * qstride + h * kDh + 2 * tig;
+      const __nv_bfloat16 *q_hi = qsrc + (size_t)(row0 + r_hi) * qstride + h * kDh + 2 * tig;
 #pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      if (MODE == 2) continue;               // rotary mode: loaded as fp32 and rotated below, once the rows' positions are known
-      qf[mt][kk][0] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
-      qf[mt][kk][1] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
-      qf[mt][kk][2] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
-      qf[mt][kk][3] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
+      for (int kk = 0; kk < 4; ++kk) {
+        qf[mt][kk][0] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16) : 0u;
+        qf[mt][kk][1] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16) : 0u;
+        qf[mt][kk][2] = r_lo < dm.C ? *reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8) : 0u;
+        qf[mt][kk][3] = r_hi < dm.C ? *reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8) : 0u;
+      }
+    }
+  }
+  // the new entries this warp appends (rows warp, warp + SW, ...): lane l holds columns 2 l, 2 l + 1 of key and value
+  constexpr int APW = (16 * MT + SW - 1) / SW;
+  uint32_t new_k[APW], new_v[APW];
+  float2 new_kf[MODE == 2 ? APW : 1], new_vf[MODE == 2 ? APW : 1];
+  if (MODE == 1) {
+#pragma unroll
+    for (int j = 0; j < APW; ++j) {
+      const int c = warp + j * SW;
+      new_k[j] = new_v[j] = 0u;
+      if (c < dm.C) {
+        const __nv_bfloat16 *src = (const __nv_bfloat16 *)a.qkv + (size_t)(row0 + c) * 3 * dm.d + dm.d + (size_t)h * kDh + 2 * lane;
+        new_k[j] = *reinterpret_cast<const uint32_t *>(src);
+        new_v[j] = *reinterpret_cast<const uint32_t *>(src + dm.d);
+      }
+    }
+  } else if (MODE == 2) {
+#pragma unroll
+    for (int j = 0; j < APW; ++j) {
+      const int c = warp + j * SW;
+      new_kf[j] = new_vf[j] = make_float2(0.f, 0.f);
+      if (c < dm.C) {
+        const float *src = (const float *)a.qkv + (size_t)(row0 + c) * 3 * dm.d + dm.d + (size_t)h * kDh + 2 * lane;
+        new_kf[j] = *reinterpret_cast<const float2 *>(src);
+        new_vf[j] = *reinterpret_cast<const float2 *>(src + dm.d);
+      }
     }
   }
 
-  // splits in use: enough that a warp gets about SBATCHES_PER_WARP batches, at most the launched ones
-  const int n_batches = (n_list + PB - 1) / PB;
-  const int n_eff = min(a.splits, max(1, (n_batches + SW * SBATCHES_PER_WARP - 1) / (SW * SBATCHES_PER_WARP)));
   if (S == 0) {   // nothing active: keep the output rows of this head defined
     if (split == 0)
       for (int idx = tid; idx < dm.C * kDh; idx += STHREADS)
         out[(size_t)(row0 + idx / kDh) * dm.d + h * kDh + idx % kDh] = __float2bfloat16_rn(0.f);
     return;
   }
-  if (split >= n_eff) return;
-
   const __nv_bfloat16 *pool_lh = (const __nv_bfloat16 *)a.kv + kv_block_offset(a.layer, dm.pool, 0, dm.H, h, P);
   const size_t page_stride = (size_t)dm.H * 2 * P * kDh;      // elements from one page's block of this head to the next page's
+
+  // ---- append (every CTA of the (sequence, head) pair writes the same bits) and, in rotary mode, the queries
   if (MODE == 2) {
     const float *qkv32 = reinterpret_cast<const float *>(a.qkv);
-    // (a) the rows' new entries: warp w takes rows w, w + SW, ...; lane l columns 2 l, 2 l + 1 of the key (rotated by the
-    // row's position) and of the value, rounded to bf16 and written to the row's cache slot.  All loads first.
-    {
-      float2 kf[(16 * MT + SW - 1) / SW], vf[(16 * MT + SW - 1) / SW], cs[(16 * MT + SW - 1) / SW];
 #pragma unroll
-      for (int j = 0; j < (16 * MT + SW - 1) / SW; ++j) {
-        const int c = warp + j * SW;
-        if (c < S) {
-          const int pos = __shfl_sync(0xffffffffu, meta.z, c);
-          const float *src = qkv32 + (size_t)(row0 + c) * 3 * dm.d + dm.d + (size_t)h * kDh + 2 * lane;
-          kf[j] = *reinterpret_cast<const float2 *>(src);
-          vf[j] = *reinterpret_cast<const float2 *>(src + dm.d);
-          cs[j] = a.rope_tab[(size_t)pos * (kDh / 2) + lane];
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < (16 * MT + SW - 1) / SW; ++j) {
-        const int c = warp + j * SW;
-        if (c < S) {
-          const int page = __shfl_sync(0xffffffffu, meta.x, c), slot = __shfl_sync(0xffffffffu, meta.y, c);
-          const float kx = kf[j].x * cs[j].x - kf[j].y * cs[j].y, ky = kf[j].x * cs[j].y + kf[j].y * cs[j].x;
-          __nv_bfloat16 *cache = const_cast<__nv_bfloat16 *>(pool_lh) + page * page_stride + kv_entry_offset<__nv_bfloat16>(slot, 2 * lane, 0);
-          *reinterpret_cast<uint32_t *>(cache) = s_pack_bf16(kx, ky);
-          *reinterpret_cast<uint32_t *>(cache + kDh) = s_pack_bf16(vf[j].x, vf[j].y);   // the value row follows the key row of the same entry
-        }
+    for (int j = 0; j < APW; ++j) {
+      const int c = warp + j * SW;
+      if (c < S) {
+        const int pos = __shfl_sync(0xffffffffu, meta.z, c);
+        const float2 cs = a.rope_tab[(size_t)pos * (kDh / 2) + lane];
+        new_k[j] = s_pack_bf16(new_kf[j].x * cs.x - new_kf[j].y * cs.y, new_kf[j].x * cs.y + new_kf[j].y * cs.x);
+        new_v[j] = s_pack_bf16(new_vf[j].x, new_vf[j].y);
       }
     }
-    // (b) this warp's query fragments, rotated likewise
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -243,84 +228,81 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
       }
     }
   }
-
-  const int W = n_eff * SW;
-  const int n_mine = n_batches > g0 ? (n_batches - g0 + W - 1) / W : 0;
-  const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SSLOT;
-
-  // One page of a batch: the entries the cache holds are copied; if a row appends to this page at this step
-  // (its entry is the page's last), that entry comes from the projection's output: 8 + 8 chunks of 16 bytes.
-  // (`early`: before the CTA's barrier.  In rotary mode a new entry is then still on its way into the cache: the
-  // entries before it are copied, the entry itself after the barrier.)
-  auto fetch_page = [&](uint32_t dst, int4 e, bool early) {
-    if (e.y <= 0) return;
-    const __nv_bfloat16 *blk = pool_lh + e.x * page_stride;
-    int n_copy = e.y;
-    if (MODE == 2 && early) {
-      const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
-      if (hit != 0u) n_copy = __shfl_sync(0xffffffffu, meta.y, __ffs(hit) - 1);
-    }
-    if (FUSED) {
-      const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
-      if (hit != 0u) {
-        const int c = __ffs(hit) - 1;
-        const int slot = __shfl_sync(0xffffffffu, meta.y, c);
-        n_copy = slot;                                         // the entries before the new one
-        if (lane < 16) {                                       // lanes 0-7: the key row's chunks, 8-15: the value row's
-          const __nv_bfloat16 *src = (const __nv_bfloat16 *)a.qkv + (size_t)(row0 + c) * 3 * dm.d + (lane < 8 ? 1 : 2) * (size_t)dm.d +
-                                     (size_t)h * kDh + (lane & 7) * 8;
-          s_cp_async16(dst + s_swz(slot, lane & 7) + (lane < 8 ? 0u : 128u), src);
-        }
+  if (MODE != 0) {
+#pragma unroll
+    for (int j = 0; j < APW; ++j) {
+      const int c = warp + j * SW;
+      if (c < S) {
+        const int page = __shfl_sync(0xffffffffu, meta.x, c), slot = __shfl_sync(0xffffffffu, meta.y, c);
+        __nv_bfloat16 *cache = const_cast<__nv_bfloat16 *>(pool_lh) + page * page_stride + kv_entry_offset<__nv_bfloat16>(slot, 2 * lane, 0);
+        *reinterpret_cast<uint32_t *>(cache) = new_k[j];
+        *reinterpret_cast<uint32_t *>(cache + kDh) = new_v[j];      // the value row follows the key row of the same entry
       }
     }
-    s_fetch_run<P>(dst, blk, n_copy, lane);
-  };
-  // batch n of this warp = list entries PB * (g0 + n W) ...; `list` = the list in global memory (before the
-  // CTA's copy is complete) or in shared memory
-  auto fetch = [&](int n, const int4 *list, bool early) {
-    const int first = PB * (g0 + n * W);
-    const uint32_t dst = my_ring + (n & 1) * SSLOT;
-#pragma unroll
-    for (int pb = 0; pb < PB; ++pb) {
-      const int4 e = first + pb < n_list ? list[first + pb] : make_int4(0, 0, 0, 0);
-      fetch_page(dst + pb * P * 256, e, early);
-    }
-  };
-  // Nothing is ever cleared: what a slot holds beyond a page's entries (anything) gets score -inf, and
-  // the value fragments of those keys are zeroed in registers after ldmatrix.
-  if (n_mine > 0) {
-#pragma unroll
-    for (int pb = 0; pb < PB; ++pb) fetch_page(my_ring + pb * P * 256, PB * g0 + pb < n_list ? e_first[pb] : make_int4(0, 0, 0, 0), true);
   }
-  s_cp_async_commit();
-  if (n_mine > 1) fetch(1, pl, true);
-  s_cp_async_commit();
-  if (tid < list_cap) plist_s[tid] = my_entry;
-  for (int i = tid + STHREADS; i < n_list; i += STHREADS) plist_s[i] = pl[i];   // lists longer than one round
+
+  // ---- the page list in shared memory, the exclusive prefix of its entry counts, the flat key list
+#pragma unroll
+  for (int k = 0; k < (SMAXLIST + STHREADS - 1) / STHREADS; ++k)
+    if (k * STHREADS + tid < list_cap) plist_s[k * STHREADS + tid] = my_entry[k];
   if (tid < 16 * MT) rsub_s[tid] = my_rsub;
 #pragma unroll
   for (int k = 0; k < SBIAS_PER_THREAD; ++k)
     if (use_bias && k * STHREADS + tid < dm.n_dist) bias_s[k * STHREADS + tid] = my_bias[k];
-  __syncthreads();
-  if (MODE == 2) {
-    // the new entries are in the cache now (written by this CTA's warps before the barrier): those of the two batches
-    // already on their way follow them into the ring
-    for (int n = 0; n < 2 && n < n_mine; ++n) {
+  __syncthreads();          // (also: this CTA's appended entries are in the cache for all its warps)
+  if (warp == 0) {
+    int carry = 0;
+    for (int j0 = 0; j0 < n_list; j0 += 32) {
+      const int nv = j0 + lane < n_list ? plist_s[j0 + lane].y : 0;
+      int incl = nv;
 #pragma unroll
-      for (int pb = 0; pb < PB; ++pb) {
-        const int idx = PB * (g0 + n * W) + pb;
-        const int4 e = idx < n_list ? plist_s[idx] : make_int4(0, 0, 0, 0);
-        const unsigned hit = __ballot_sync(0xffffffffu, e.y > 0 && lane < S && meta.x == e.x);
-        if (hit != 0u) {
-          const int slot = __shfl_sync(0xffffffffu, meta.y, __ffs(hit) - 1);
-          if (lane < 16) {
-            const uint32_t off = s_swz(slot, lane & 7) + (lane < 8 ? 0u : 128u);
-            s_cp_async16(my_ring + (n & 1) * SSLOT + pb * P * 256 + off,
-                         reinterpret_cast<const uint8_t *>(pool_lh + e.x * page_stride) + off);
-          }
-        }
+      for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += u; }
+      if (j0 + lane < n_list) off_s[j0 + lane] = carry + incl - nv;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) n_keys_s = carry;
+  }
+  __syncthreads();
+  for (int j = tid; j < n_list; j += STHREADS) {
+    const int4 e = plist_s[j];
+    const int o0 = off_s[j];
+    for (int k = 0; k < e.y; ++k)      // entry k of the page: its distance base is the page's minus its offset
+      key_s[o0 + k] = make_int2(e.x * 32 + k, e.z | ((e.w - k + 1024) << 8));
+  }
+  __syncthreads();
+  const int n_keys = n_keys_s;
+
+  // splits in use: enough that a warp gets about STILES_PER_WARP tiles, at most the launched ones
+  const int n_tiles = (n_keys + STK - 1) / STK;
+  const int n_eff = min(a.splits, max(1, (n_tiles + SW * STILES_PER_WARP - 1) / (SW * STILES_PER_WARP)));
+  if (split >= n_eff) return;
+  const int W = n_eff * SW, g0 = split * SW + warp;
+  const int n_mine = n_tiles > g0 ? (n_tiles - g0 + W - 1) / W : 0;
+  const uint32_t my_ring = s_smem_u32(s_ring_raw) + warp * SDEPTH * SSLOT;
+
+  // Tile n of this warp = keys 16 (g0 + n W) ... of the flat list.  Lane l copies, in eight rounds, one 16-byte chunk
+  // each: round k covers keys 2 k and 2 k + 1, chunks 0-7 = the key row, 8-15 = the value row.  A cache row's chunk c
+  // lies at place c ^ (slot & 7) of its row; in the tile it goes to place c ^ (row in tile & 7).
+  auto fetch = [&](int n) {
+    const int first = STK * (g0 + n * W);
+    const uint32_t dst = my_ring + (n % SDEPTH) * SSLOT;
+#pragma unroll
+    for (int k = 0; k < STK / 2; ++k) {
+      const int r = 2 * k + (lane >> 4), p = lane & 15;
+      if (first + r < n_keys) {
+        const int src = key_s[first + r].x;
+        const int page = src >> 5, slot = src & 31;
+        const uint8_t *from = reinterpret_cast<const uint8_t *>(pool_lh + page * page_stride) + slot * 256 + p * 16;
+        const int place = (p & 7) ^ (slot & 7) ^ (r & 7);
+        s_cp_async16(dst + r * 256 + (p & 8) * 16 + place * 16, from);
       }
     }
+  };
+  // Nothing is ever cleared: what a slot holds beyond the list's last key (anything) gets score -inf, and the value
+  // fragments of those keys are zeroed in registers after ldmatrix.
+#pragma unroll
+  for (int n = 0; n < SDEPTH; ++n) {
+    if (n < n_mine) fetch(n);
     s_cp_async_commit();
   }
 
@@ -332,7 +314,7 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
     rs[mt][1] = rsub_s[min(mt * 16 + g + 8, S - 1)];
     tile_last[mt] = 16 * mt < S ? rsub_s[min(16 * mt + 15, S - 1)] : 0;
   }
-  const int sub_first = rsub_s[0];   // the smallest active subsequence: a page it sees, every row sees
+  const int sub_first = rsub_s[0];   // the smallest active subsequence: a key it sees, every row sees
   float o[MT][8][4];
   float m_run[MT][2], l_run[MT][2];
 #pragma unroll
@@ -345,51 +327,35 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
   const float sl2 = dm.scale_log2e;
 
   for (int n = 0; n < n_mine; ++n) {
-    if (MODE == 2 && n == 0) s_cp_async_wait<0>();     // the first batches' new entries were requested last
-    else s_cp_async_wait<1>();         // everything but the newest group has landed: batch n is in its slot
-    __syncwarp();                      // (and the appended entries the lanes stored themselves are visible)
-    // per page of the batch: entries that exist, subsequence, distance base of its first entry
-    int nv[PB], ksub[PB], d0[PB];
-    const int first = PB * (g0 + n * W);
+    s_cp_async_wait<SDEPTH - 1>();     // everything but the newest group has landed: tile n is in its slot
+    __syncwarp();
+    const int first = STK * (g0 + n * W);
+    const int nv = min(STK, n_keys - first);           // keys of this tile that exist
+    // this thread's four keys of the tile (two per 8-key score tile): subsequence and distance base
+    int ksub[2][2], kd[2][2];
 #pragma unroll
-    for (int pb = 0; pb < PB; ++pb) {
-      const int4 e = first + pb < n_list ? plist_s[first + pb] : make_int4(0, 0, 0x7fffffff, 0);
-      nv[pb] = e.y; ksub[pb] = e.z; d0[pb] = e.w;
-      if (FUSED && e.y > 0) {
-        // the entry a row appended to this page has landed in the slot: on into the cache (same swizzled place)
-        const unsigned hit = __ballot_sync(0xffffffffu, lane < S && meta.x == e.x);
-        if (hit != 0u) {
-          const int slot = __shfl_sync(0xffffffffu, meta.y, __ffs(hit) - 1);
-          if (lane < 16) {
-            const uint32_t off = s_swz(slot, lane & 7) + (lane < 8 ? 0u : 128u);
-            uint4 v;
-            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                         : "r"(my_ring + (n & 1) * SSLOT + pb * P * 256 + off));
-            uint8_t *cache = reinterpret_cast<uint8_t *>(const_cast<__nv_bfloat16 *>(pool_lh + e.x * page_stride)) + off;
-            *reinterpret_cast<uint4 *>(cache) = v;
-          }
-        }
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int x = 0; x < 2; ++x) {
+        const int e = nt * 8 + 2 * tig + x;
+        const int m = e < nv ? key_s[first + e].y : 0x7f;     // absent: a subsequence no row reaches
+        ksub[nt][x] = m & 0xff; kd[nt][x] = (m >> 8) - 1024;
       }
-    }
-    const uint32_t kbase = my_ring + (n & 1) * SSLOT, vbase = kbase + 128u;
-    // Dependency rule: a row of subsequence i sees a page iff i' <= i (every stored entry was
-    // generated before the current step).  The list is sorted by subsequence: a query tile none
-    // of whose rows sees the batch's first page is skipped; a batch of full pages that every row sees
-    // needs no masking at all.
+    const int k_first = key_s[first].y & 0xff, k_last = key_s[first + nv - 1].y & 0xff;   // keys are sorted by subsequence
+    const uint32_t kbase = my_ring + (n % SDEPTH) * SSLOT, vbase = kbase + 128u;
+    // Dependency rule: a row of subsequence i sees a key iff i' <= i (every stored entry was generated
+    // before the current step).  A query tile none of whose rows sees the tile's first key is skipped;
+    // a full tile that every row sees needs no masking at all.
     bool act[MT];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) act[mt] = tile_last[mt] >= ksub[0];
-    bool plain = true;
-#pragma unroll
-    for (int pb = 0; pb < PB; ++pb) plain = plain && nv[pb] == P && sub_first >= ksub[pb];
+    for (int mt = 0; mt < MT; ++mt) act[mt] = tile_last[mt] >= k_first;
+    const bool plain = nv == STK && sub_first >= k_last;
 
-    // ---- scores: Q (16 x 64) . K^T (64 x 32 keys); two accumulators per tile halve the mma chain
-    float sc[MT][NT][4];
+    // ---- scores: Q (16 x 64) . K^T (64 x 16 keys); two accumulators per tile halve the mma chain
+    float sc[MT][2][4];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      constexpr int per_page = P / 8;                    // score tiles per page
-      const int pb = nt / per_page, within = (nt % per_page) * 8;
-      if (within < nv[pb]) {
+    for (int nt = 0; nt < 2; ++nt) {
+      if (nt * 8 < nv) {
         const int key = nt * 8 + (lane & 7);
         uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
         s_ldsm_x4(kbase + s_swz(key, (lane >> 3)), b0, b1, b2, b3);        // dims 0..31
@@ -412,37 +378,25 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
           for (int x = 0; x < 4; ++x) sc[mt][nt][x] = 0.f;
       }
     }
-    // ---- scale, positional bias on the Manhattan distance, visibility, online softmax (log2 domain)
-    uint32_t pf[MT][KS][4];
+    // ---- scale, positional bias on the Manhattan distance (the key's distance base + the row's subsequence),
+    // visibility, online softmax (log2 domain)
+    uint32_t pf[MT][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       if (!act[mt]) continue;
       float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        constexpr int per_page = P / 8;
-        const int pb = nt / per_page, within = (nt % per_page) * 8 + 2 * tig;    // this thread's first key of the tile, inside its page
-        // distance of rows g / g + 8 to the page's entry 0, minus the key's offset in the page
-        const float *bp0 = bias_s + (d0[pb] + rs[mt][0] - within);
-        const float *bp1 = bias_s + (d0[pb] + rs[mt][1] - within);
-        if (plain) {
+      for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const float bias = use_bias ? ((x & 2) ? bp1 : bp0)[-(x & 1)] : 0.f;
-            sc[mt][nt][x] = fmaf(sc[mt][nt][x], sl2, bias);
+        for (int x = 0; x < 4; ++x) {
+          const int kx = x & 1, hh = x >> 1;
+          const bool vis = plain || (ksub[nt][kx] <= rs[mt][hh]);       // (an absent key's subsequence is beyond every row)
+          float v = -INFINITY;
+          if (vis) {
+            const float bias = use_bias ? bias_s[kd[nt][kx] + rs[mt][hh]] : 0.f;
+            v = fmaf(sc[mt][nt][x], sl2, bias);
           }
-        } else {
-          const bool see0 = rs[mt][0] >= ksub[pb], see1 = rs[mt][1] >= ksub[pb];
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const bool vis = within + (x & 1) < nv[pb] && ((x & 2) ? see1 : see0);
-            float v = -INFINITY;
-            if (vis) {
-              const float bias = use_bias ? ((x & 2) ? bp1 : bp0)[-(x & 1)] : 0.f;
-              v = fmaf(sc[mt][nt][x], sl2, bias);
-            }
-            sc[mt][nt][x] = v;
-          }
+          sc[mt][nt][x] = v;
         }
         mx0 = fmaxf(mx0, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
         mx1 = fmaxf(mx1, fmaxf(sc[mt][nt][2], sc[mt][nt][3]));
@@ -457,12 +411,12 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
       m_run[mt][0] = mn0; m_run[mt][1] = mn1;
       float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
+      for (int nt = 0; nt < 2; ++nt) {
         float p0 = s_ex2(sc[mt][nt][0] - ref0), p1 = s_ex2(sc[mt][nt][1] - ref0);
         float p2 = s_ex2(sc[mt][nt][2] - ref1), p3 = s_ex2(sc[mt][nt][3] - ref1);
         s0 += p0 + p1; s1 += p2 + p3;
-        pf[mt][nt >> 1][(nt & 1) * 2 + 0] = s_pack_bf16(p0, p1);
-        pf[mt][nt >> 1][(nt & 1) * 2 + 1] = s_pack_bf16(p2, p3);
+        pf[mt][nt * 2 + 0] = s_pack_bf16(p0, p1);
+        pf[mt][nt * 2 + 1] = s_pack_bf16(p2, p3);
       }
       l_run[mt][0] = l_run[mt][0] * cr0 + s0;
       l_run[mt][1] = l_run[mt][1] * cr1 + s1;
@@ -471,38 +425,33 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
         for (int dn = 0; dn < 8; ++dn) { o[mt][dn][0] *= cr0; o[mt][dn][1] *= cr0; o[mt][dn][2] *= cr1; o[mt][dn][3] *= cr1; }
       }
     }
-    // ---- O += P (16 x 32 keys) . V (32 keys x 64)
+    // ---- O += P (16 x 16 keys) . V (16 keys x 64)
+    {
+      const int vkey = ((lane >> 3) & 1) * 8 + (lane & 7);
+      // this lane's fragment halves hold keys k0, k0 + 1 (b0, b2) and k0 + 8, k0 + 9 (b1, b3) of the tile;
+      // keys that do not exist have weight exactly 0 and must not contribute whatever the slot holds
+      const bool ragged = nv < STK;
+      uint32_t keep_a = 0xffffffffu, keep_b = 0xffffffffu;
+      if (ragged) {
+        const int k0 = 2 * tig;
+        keep_a = (k0 < nv ? 0x0000ffffu : 0u) | (k0 + 1 < nv ? 0xffff0000u : 0u);
+        keep_b = (k0 + 8 < nv ? 0x0000ffffu : 0u) | (k0 + 9 < nv ? 0xffff0000u : 0u);
+      }
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      constexpr int per_page = P / 16;                   // 16-key steps per page
-      const int pb = ks / per_page, within = (ks % per_page) * 16;
-      if (within < nv[pb]) {
-        const int vkey = ks * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-        // this lane's fragment halves hold keys k0, k0 + 1 (b0, b2) and k0 + 8, k0 + 9 (b1, b3) of the page;
-        // keys that do not exist have weight exactly 0 and must not contribute whatever the slot holds
-        const bool ragged = nv[pb] < within + 16;
-        uint32_t keep_a = 0xffffffffu, keep_b = 0xffffffffu;
-        if (ragged) {
-          const int k0 = within + 2 * tig;
-          keep_a = (k0 < nv[pb] ? 0x0000ffffu : 0u) | (k0 + 1 < nv[pb] ? 0xffff0000u : 0u);
-          keep_b = (k0 + 8 < nv[pb] ? 0x0000ffffu : 0u) | (k0 + 9 < nv[pb] ? 0xffff0000u : 0u);
-        }
+      for (int dp = 0; dp < 4; ++dp) {
+        uint32_t b0, b1, b2, b3;
+        s_ldsm_x4_t(vbase + s_swz(vkey, dp * 2 + (lane >> 4)), b0, b1, b2, b3);
+        if (ragged) { b0 &= keep_a; b1 &= keep_b; b2 &= keep_a; b3 &= keep_b; }
 #pragma unroll
-        for (int dp = 0; dp < 4; ++dp) {
-          uint32_t b0, b1, b2, b3;
-          s_ldsm_x4_t(vbase + s_swz(vkey, dp * 2 + (lane >> 4)), b0, b1, b2, b3);
-          if (ragged) { b0 &= keep_a; b1 &= keep_b; b2 &= keep_a; b3 &= keep_b; }
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            if (!act[mt]) continue;
-            s_mma_bf16(o[mt][2 * dp], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b0, b1);
-            s_mma_bf16(o[mt][2 * dp + 1], pf[mt][ks][0], pf[mt][ks][1], pf[mt][ks][2], pf[mt][ks][3], b2, b3);
-          }
+        for (int mt = 0; mt < MT; ++mt) {
+          if (!act[mt]) continue;
+          s_mma_bf16(o[mt][2 * dp], pf[mt][0], pf[mt][1], pf[mt][2], pf[mt][3], b0, b1);
+          s_mma_bf16(o[mt][2 * dp + 1], pf[mt][0], pf[mt][1], pf[mt][2], pf[mt][3], b2, b3);
         }
       }
     }
     __syncwarp();   // every lane is done reading the slot
-    if (n + 2 < n_mine) fetch(n + 2, plist_s, false);
+    if (n + SDEPTH < n_mine) fetch(n + SDEPTH);
     s_cp_async_commit();
   }
   s_cp_async_wait<0>();
@@ -609,24 +558,23 @@ __global__ void __launch_bounds__(STHREADS, MT == 1 ? OCC : 2) self_attn_tc_kern
 }
 
 static int self_attn_tc_smem(const Dims &dm) {
-  const int mt = (dm.C + 15) / 16;
-  return self_attn_tc_ring_bytes(dm.P, mt) + dm.SM * dm.PPS * (int)sizeof(int4) + (dm.pos_mode == PD_POS_T5_BIAS ? dm.n_dist * 4 : 0);
+  const int mt = (dm.C + 15) / 16, list_cap = dm.SM * dm.PPS;
+  return self_attn_tc_ring_bytes(mt) + list_cap * (int)sizeof(int4) + ((list_cap + 2) & ~1) * 4 + list_cap * dm.P * (int)sizeof(int2) +
+         (dm.pos_mode == PD_POS_T5_BIAS ? dm.n_dist * 4 : 0);
 }
-static int self_attn_tc_max_smem(int P, int mt) { return self_attn_tc_ring_bytes(P, mt) + SMAXLIST * (int)sizeof(int4) + SMAXDIST * 4; }
 
 bool self_attn_tc_supported(const Dims &dm) {
-  return dm.C <= 32 && (dm.P == 16 || dm.P == 32) && dm.SM * dm.PPS <= SMAXLIST &&
-         (dm.pos_mode != PD_POS_T5_BIAS || dm.n_dist <= SMAXDIST);
+  return dm.C <= 32 && (dm.P == 16 || dm.P == 32) && dm.SM * dm.PPS <= SMAXLIST && dm.SM <= 127 &&
+         (dm.pos_mode != PD_POS_T5_BIAS || dm.n_dist <= SMAXDIST) && self_attn_tc_smem(dm) <= 200 * 1024;
 }
 
 // Splits to launch for `pairs` (sequence, head) pairs on a device with `sms` SMs: enough for the
-// longest page list a sequence can have (CTAs whose split the current lists do not need leave at
+// longest key list a sequence can have (CTAs whose split the current lists do not need leave at
 // once), but never more CTAs than are resident at the same time - a second wave costs a whole
 // CTA lifetime, a longer walk per warp a fraction of one.
 int self_attn_tc_splits(const Dims &dm, int pairs, int sms) {
-  const int per = dm.P > SKEYS ? 1 : SKEYS / dm.P;       // pages per batch
-  const int batches = (dm.SM * dm.PPS + per - 1) / per;
-  int s = (batches + SW * SBATCHES_PER_WARP - 1) / (SW * SBATCHES_PER_WARP);
+  const int tiles = (dm.SM * (dm.MSL + 2) + STK - 1) / STK;
+  int s = (tiles + SW * STILES_PER_WARP - 1) / (SW * STILES_PER_WARP);
   // CTAs an SM holds: five by registers (two with 32 rows), and what 227 KB of shared memory allow
   const int by_smem = (227 * 1024) / (self_attn_tc_smem(dm) + 1024 + 256);
   const int per_sm = dm.C <= 16 ? (by_smem < 5 ? by_smem : 5) : (by_smem < 2 ? by_smem : 2);
@@ -637,7 +585,7 @@ int self_attn_tc_splits(const Dims &dm, int pairs, int sms) {
 
 template <int MT, int P>
 static cudaError_t prepare_one() {
-  const int smem = self_attn_tc_max_smem(P, MT);
+  const int smem = 200 * 1024;
   cudaError_t e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 0, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(self_attn_tc_kernel<MT, P, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
